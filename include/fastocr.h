@@ -1,0 +1,189 @@
+/*
+ * fastocr.h - C ABI of the FastOCR decode-step attention hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, for one transformer layer at a time (and, with
+ * fastocr_decode_step, for a whole decode step), the attention work of the
+ * paper's Algorithm 1 after warm-up:
+ *   - focal layers attend the full KV cache and score every image token
+ *     (Section 3.1.2, Eq. 2 first case),
+ *   - the ceil(tau*N) best-scored image tokens become the focal-token set F,
+ *   - all other layers attend only K = T u F, all text tokens plus F
+ *     (Eq. 2 second case), the set being inherited from the nearest preceding
+ *     focal layer (Cross-Layer Propagation) or from the previous decode step
+ *     (Cross-Step Fixation Reuse, Section 3.2),
+ * and never modifies, compacts or frees the cache (Section 2: no physical eviction).
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory owned by the caller and valid on
+ *     the context's device; "host" pointers are ordinary host memory. The
+ *     library allocates device memory only inside fastocr_create.
+ *   - All tensor arguments are dense row-major with the index order written in
+ *     brackets; bf16 means the 16-bit brain-float bit pattern.
+ *   - Every compute call is asynchronous on `stream` (a cudaStream_t passed as
+ *     void*, NULL = the legacy default stream), performs no allocation and no
+ *     host-device synchronisation, and may be captured into a CUDA graph.
+ *   - Calls on one context must not overlap on the GPU (they share its
+ *     workspace): issue them on one stream, or order the streams.
+ *   - Return value: FASTOCR_OK or an error code; on error nothing was launched
+ *     and fastocr_last_error(ctx) describes the problem. Argument checks are
+ *     host-side only; the contents of device arrays (lengths, indices, page
+ *     ids) cannot be validated without a synchronisation: indices outside
+ *     [0, vis_len) are clamped on the device and counted in a status word
+ *     readable with fastocr_device_faults.
+ *   - head_dim must be 128 and num_q_heads / num_kv_heads (the GQA group size)
+ *     one of 1, 2, 4, 7, 8; query head h reads KV head h / group size.
+ */
+#ifndef FASTOCR_H_
+#define FASTOCR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum fastocr_status {
+  FASTOCR_OK = 0,
+  FASTOCR_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, inconsistent shapes            */
+  FASTOCR_ERR_UNSUPPORTED = 2, /* head_dim != 128, group size, page size, vis_len too large   */
+  FASTOCR_ERR_WORKSPACE = 3,   /* the call exceeds the limits given to fastocr_create         */
+  FASTOCR_ERR_CUDA = 4         /* a CUDA runtime call failed; see fastocr_last_error          */
+} fastocr_status;
+
+typedef struct fastocr_ctx fastocr_ctx; /* opaque; owns the workspace; bound to one device */
+
+/* Upper bounds used to size the workspace once. */
+typedef struct fastocr_limits {
+  int32_t max_batch;    /* sequences per call                                   */
+  int32_t num_q_heads;  /* H                                                     */
+  int32_t num_kv_heads; /* H_kv                                                  */
+  int32_t max_seq_len;  /* cached tokens per sequence (text + image)            */
+  int32_t max_vis_len;  /* image tokens per sequence, N; at most 32768          */
+} fastocr_limits;
+
+/*
+ * Read-only view of ONE layer's KV cache for a (possibly ragged) batch.
+ * The image tokens of sequence b occupy the contiguous position span
+ * [vis_start[b], vis_start[b] + vis_len[b]); every other position is text
+ * (system, prompt, generated and the current token) and is always attended.
+ */
+typedef struct fastocr_kv_view {
+  int32_t batch;        /* B                                                                     */
+  int32_t num_q_heads;  /* H                                                                     */
+  int32_t num_kv_heads; /* H_kv, divides H                                                       */
+  int32_t head_dim;     /* 128                                                                   */
+  int32_t page_size;    /* 0: contiguous cache; otherwise tokens per page (a power of two)       */
+  int32_t max_seq_len;  /* host-known upper bound on seq_len[b]; sizes the launch                */
+  const void* k;        /* device bf16. contiguous: [B][seq_stride_tokens][H_kv][128]            */
+  const void* v;        /*              paged:      [num_pages][page_size][H_kv][128]            */
+  int64_t seq_stride_tokens;  /* contiguous only: tokens between consecutive sequences           */
+  const int32_t* block_table; /* paged only: device [B][max_pages], physical page of each logical page */
+  int32_t max_pages;          /* paged only: row length of block_table                           */
+  const int32_t* seq_len;     /* device [B]: S_b, number of cached tokens                        */
+  const int32_t* vis_start;   /* device [B]: first image position                                */
+  const int32_t* vis_len;     /* device [B]: N_b, number of image tokens                         */
+  float sm_scale;             /* softmax scale, 1/sqrt(head_dim) (Appendix B)                    */
+} fastocr_kv_view;
+
+/* Creates a context on `device` with workspace for the given limits (cudaMalloc happens here and
+ * only here). *out is set on success. Not thread-safe per context. */
+fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limits* limits);
+void fastocr_destroy(fastocr_ctx* ctx);
+/* Message of the last failed call on this context (owned by the context; "" if none). */
+const char* fastocr_last_error(const fastocr_ctx* ctx);
+/* Synchronises the device and returns how many out-of-range indices kernels have clamped since
+ * the last call (diagnostic; not for the hot path). Negative on CUDA error. */
+int64_t fastocr_device_faults(fastocr_ctx* ctx);
+
+/* |F| = ceil(tau * N) clamped to [0, N] (Section 3.1.2). tau = 0 keeps no image token,
+ * tau >= 1 keeps all. Host-only. */
+int32_t fastocr_kept_count(int32_t n_vis, double tau);
+
+/*
+ * Dense decode attention over the whole cache: Eq. 2 first case, Attn = softmax(q K^T * sm_scale) V
+ * (Appendix B), for every query head of every sequence. This is the focal-layer path and the
+ * unpruned baseline.
+ *   q          device bf16 [B][H][128]
+ *   out        device [B][H][128], bf16, or fp32 when out_is_fp32 != 0
+ *   scores_out NULL, or device fp32 [B][n_stride]: additionally receives the head-averaged image
+ *              attention of fastocr_focal_scores from the same pass over K (entries
+ *              [vis_len[b], n_stride) are left untouched); n_stride >= max vis_len.
+ */
+fastocr_status fastocr_dense_decode_attn(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, void* out,
+                                         int out_is_fp32, float* scores_out, int32_t n_stride, void* stream);
+
+/*
+ * Focal scores: for image token i of sequence b, the attention weight from the current query to
+ * that token, softmax taken over the FULL cache, averaged over all H query heads (the a-bar of
+ * Section 3.1.1 that Eq. 2's TopK ranks). Reads K only.
+ *   scores_out     device fp32 [B][n_stride]
+ *   image_mass_out NULL, or device fp32 [B]: sum_i scores = Eq. 1's image-attention ratio r
+ */
+fastocr_status fastocr_focal_scores(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, float* scores_out,
+                                    int32_t n_stride, float* image_mass_out, void* stream);
+
+/*
+ * TopK of Eq. 2: for each sequence the k[b] image tokens with the largest scores. Larger score
+ * wins; equal scores: the lower index wins; -0 equals +0; NaN ranks below every number. Indices
+ * are relative to vis_start and written in ascending order to idx_out[b][0..k[b]); the rest of the
+ * row is left untouched.
+ *   scores  device fp32 [B][n_stride]      vis_len device int32 [B]
+ *   k       device int32 [B], 0 <= k[b] <= vis_len[b] (larger values are clamped)
+ *   idx_out device int32 [B][k_stride]
+ *   max_vis_len host-known bound on vis_len[b] (<= 32768)
+ */
+fastocr_status fastocr_select_topk(fastocr_ctx* ctx, const float* scores, int32_t n_stride, const int32_t* vis_len,
+                                   const int32_t* k, int32_t batch, int32_t max_vis_len, int32_t* idx_out,
+                                   int32_t k_stride, void* stream);
+
+/*
+ * Pruned decode attention: Eq. 2 second case. Softmax and weighted sum run over the kept set
+ * K = T u F only: every text position plus positions vis_start + idx[b][i], i < k[b].
+ *   idx device int32 [B][k_stride] (values in [0, vis_len[b]); need not be sorted, must be distinct)
+ *   k   device int32 [B]
+ *   max_kept host-known bound on k[b] + seq_len[b] - vis_len[b] (0: use kv->max_seq_len)
+ * A sequence whose kept set is empty yields zeros.
+ */
+fastocr_status fastocr_sparse_decode_attn(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q,
+                                          const int32_t* idx, const int32_t* k, int32_t k_stride, int32_t max_kept,
+                                          void* out, int out_is_fp32, void* stream);
+
+/*
+ * One post-warm-up decode step of Algorithm 1 over L layers (Cross-Step Fixation Reuse followed by
+ * Cross-Layer Propagation), all launches on `stream`:
+ *   layer 0 reuses `fixation` when it is not focal and has_fixation != 0, otherwise it attends the
+ *   full cache and selects (the fallback); each later focal layer attends the full cache and
+ *   refreshes the set; every other layer attends text + the current set. On return (in stream
+ *   order) `fixation` holds the set of the deepest focal layer: the F_last of the next step.
+ *   layers   host array [L] of views (all with the same batch / heads / spans)
+ *   q, out   device [L][B][H][128]; out bf16 or fp32
+ *   is_focal host uint8 [L]: membership in the focal layer set C
+ *   k        device int32 [B]; fixation device int32 [B][k_stride] (in/out)
+ *   max_vis_len, max_kept: host bounds as above
+ * Returns through *has_fixation_out (may be NULL) whether `fixation` is valid afterwards.
+ */
+fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
+                                   const void* q, void* out, int out_is_fp32, const uint8_t* is_focal,
+                                   const int32_t* k, int32_t* fixation, int32_t k_stride, int has_fixation,
+                                   int32_t max_vis_len, int32_t max_kept, int* has_fixation_out, void* stream);
+
+/*
+ * Focal Layer Selection (Section 3.1.1; Algorithm 1, profiling block), host-only: rank layers by
+ * mean image-attention ratio (descending; equal ratios: lower layer first) and accept greedily
+ * while fewer than floor(rho*L) are chosen and the candidate is more than `gap` layers from every
+ * accepted one. mean_ratio host [L]; focal_out host int32 [L] receives the set in ascending order.
+ * Returns the number of focal layers, or -1 on invalid arguments.
+ */
+int32_t fastocr_focal_layers(const double* mean_ratio, int32_t num_layers, double rho, int32_t gap,
+                             int32_t* focal_out);
+
+/* Appendix B: self-attention FLOPs of one decode step, b*l*(8h^2 + 4hs). Host-only. */
+double fastocr_attn_flops(double batch, double layers, double hidden, double seq_len);
+
+/* Number of kernels this library has launched on any context since load (for bench accounting). */
+int64_t fastocr_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTOCR_H_ */

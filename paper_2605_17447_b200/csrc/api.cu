@@ -1,0 +1,394 @@
+// C ABI of the FastOCR decode-attention library: context, argument checks, split planning and the
+// per-layer / per-step launch sequences. All arithmetic lives in attn.cu and topk.cu.
+#include "../../include/fastocr.h"
+
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kernels.h"
+
+namespace fastocr {
+static std::atomic<long long> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+cudaError_t configure_topk();
+}  // namespace fastocr
+
+using fastocr::AttnLaunch;
+
+struct fastocr_ctx {
+  int device = 0;
+  int sm_count = 148;
+  fastocr_limits lim{};
+  int64_t cap_items = 0;        // (sequence, KV head, split) partial slots
+  float* part_acc = nullptr;    // [cap_items][8][128]
+  float* part_ml = nullptr;     // [cap_items][8][2]
+  float* logits = nullptr;      // [max_batch][H][max_vis_len]
+  float* stats = nullptr;       // [max_batch][H][2]
+  float* scores = nullptr;      // [max_batch][max_vis_len] (decode_step scratch)
+  unsigned long long* faults = nullptr;
+  int target_items = 0;         // tuning: desired number of CTAs per attention launch
+  int min_chunk = 0;            // tuning: smallest split, tokens
+  char err[512] = {0};
+};
+
+namespace {
+
+fastocr_status fail(fastocr_ctx* ctx, fastocr_status code, const char* fmt, ...) {
+  if (ctx != nullptr) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(ctx->err, sizeof ctx->err, fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+bool group_supported(int G) { return G == 1 || G == 2 || G == 4 || G == 7 || G == 8; }
+
+int env_int(const char* name, int dflt) {
+  const char* v = std::getenv(name);
+  return (v != nullptr && *v != 0) ? std::atoi(v) : dflt;
+}
+
+int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// Split planning: how many tokens one CTA streams. Enough CTAs to keep every SM busy with a few
+// resident CTAs and to even out the tail, but no smaller than min_chunk tokens so that the
+// prologue (query load, row table, pipeline fill) is amortised.
+void plan_split(const fastocr_ctx* ctx, int batch, int num_kv_heads, int max_len, int* chunk_tokens,
+                int* max_chunks) {
+  const int64_t units = static_cast<int64_t>(batch) * num_kv_heads;
+  int64_t nch = (ctx->target_items + units - 1) / units;
+  const int min_chunk = units >= 64 ? ctx->min_chunk : 32;
+  const int64_t by_min = max_len / min_chunk > 0 ? max_len / min_chunk : 1;
+  if (nch > by_min) nch = by_min;
+  const int64_t by_cap = ctx->cap_items / units > 0 ? ctx->cap_items / units : 1;
+  if (nch > by_cap) nch = by_cap;
+  if (nch < 1) nch = 1;
+  int chunk = round_up(static_cast<int>((max_len + nch - 1) / nch), fastocr::kTokensPerCtaIter);
+  if (chunk > fastocr::kMaxChunk) chunk = fastocr::kMaxChunk;
+  if (chunk < fastocr::kTokensPerCtaIter) chunk = fastocr::kTokensPerCtaIter;
+  *chunk_tokens = chunk;
+  *max_chunks = (max_len + chunk - 1) / chunk;
+  if (*max_chunks < 1) *max_chunks = 1;
+}
+
+fastocr_status check_view(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, bool need_v) {
+  if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
+  if (kv == nullptr || q == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL view or query pointer");
+  if (kv->k == nullptr || (need_v && kv->v == nullptr)) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL cache pointer");
+  if (kv->seq_len == nullptr || kv->vis_start == nullptr || kv->vis_len == nullptr)
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL seq_len / vis_start / vis_len");
+  if (kv->batch <= 0 || kv->num_q_heads <= 0 || kv->num_kv_heads <= 0 || kv->max_seq_len <= 0)
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "batch, head counts and max_seq_len must be positive");
+  if (kv->head_dim != fastocr::kHeadDim) return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "head_dim %d (only 128)", kv->head_dim);
+  if (kv->num_q_heads % kv->num_kv_heads != 0)
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "num_q_heads %d not a multiple of num_kv_heads %d", kv->num_q_heads, kv->num_kv_heads);
+  if (!group_supported(kv->num_q_heads / kv->num_kv_heads))
+    return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "GQA group size %d (supported: 1, 2, 4, 7, 8)", kv->num_q_heads / kv->num_kv_heads);
+  if (kv->page_size < 0 || (kv->page_size & (kv->page_size - 1)) != 0)
+    return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "page_size %d is not 0 or a power of two", kv->page_size);
+  if (kv->page_size > 0) {
+    if (kv->block_table == nullptr || kv->max_pages <= 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "paged view without block_table");
+    if (static_cast<int64_t>(kv->max_pages) * kv->page_size < kv->max_seq_len)
+      return fail(ctx, FASTOCR_ERR_INVALID_ARG, "max_pages * page_size < max_seq_len");
+  } else if (kv->seq_stride_tokens < kv->max_seq_len) {
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "seq_stride_tokens < max_seq_len");
+  }
+  if (!(kv->sm_scale > 0.f) || !std::isfinite(kv->sm_scale)) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "sm_scale must be positive");
+  if (kv->batch > ctx->lim.max_batch || kv->num_q_heads > ctx->lim.num_q_heads ||
+      kv->num_kv_heads > ctx->lim.num_kv_heads || kv->max_seq_len > ctx->lim.max_seq_len)
+    return fail(ctx, FASTOCR_ERR_WORKSPACE, "view (B=%d H=%d Hkv=%d S<=%d) exceeds the context limits (B=%d H=%d Hkv=%d S<=%d)",
+                kv->batch, kv->num_q_heads, kv->num_kv_heads, kv->max_seq_len, ctx->lim.max_batch, ctx->lim.num_q_heads,
+                ctx->lim.num_kv_heads, ctx->lim.max_seq_len);
+  return FASTOCR_OK;
+}
+
+AttnLaunch make_launch(const fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, bool with_v, int max_len) {
+  AttnLaunch a{};
+  a.k = kv->k;
+  a.v = with_v ? kv->v : nullptr;
+  a.seq_stride_tokens = kv->seq_stride_tokens;
+  a.block_table = kv->block_table;
+  a.max_pages = kv->max_pages;
+  a.page_size = kv->page_size;
+  a.seq_len = kv->seq_len;
+  a.vis_start = kv->vis_start;
+  a.vis_len = kv->vis_len;
+  a.batch = kv->batch;
+  a.num_q_heads = kv->num_q_heads;
+  a.num_kv_heads = kv->num_kv_heads;
+  a.sm_scale = kv->sm_scale;
+  a.q = q;
+  a.part_acc = ctx->part_acc;
+  a.part_ml = ctx->part_ml;
+  a.fault_counter = ctx->faults;
+  plan_split(ctx, kv->batch, kv->num_kv_heads, max_len, &a.chunk_tokens, &a.max_chunks);
+  return a;
+}
+
+fastocr_status cuda_fail(fastocr_ctx* ctx, cudaError_t e, const char* what) {
+  return fail(ctx, FASTOCR_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define FASTOCR_TRY_CUDA(expr, what)                         \
+  do {                                                       \
+    cudaError_t e_ = (expr);                                 \
+    if (e_ != cudaSuccess) return cuda_fail(ctx, e_, what);  \
+  } while (0)
+
+// dense pass (+ optional fused scoring) without re-validating the view
+fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, void* out, int out_is_fp32,
+                          float* scores_out, int32_t n_stride, int32_t max_vis, cudaStream_t s) {
+  AttnLaunch a = make_launch(ctx, kv, q, /*with_v=*/out != nullptr, kv->max_seq_len);
+  const bool want_scores = scores_out != nullptr;
+  if (want_scores) {
+    a.logits = ctx->logits;
+    a.n_stride = ctx->lim.max_vis_len;
+  }
+  FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
+  FASTOCR_TRY_CUDA(fastocr::launch_attn_combine(a, out, out_is_fp32, want_scores ? ctx->stats : nullptr, s), "combine launch");
+  if (want_scores)
+    FASTOCR_TRY_CUDA(fastocr::launch_scores_finalize(ctx->logits, ctx->stats, kv->vis_len, kv->batch, kv->num_q_heads,
+                                                     ctx->lim.max_vis_len, max_vis, scores_out, n_stride, s),
+                     "score finalisation launch");
+  return FASTOCR_OK;
+}
+
+fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, const int32_t* idx,
+                           const int32_t* k, int32_t k_stride, int32_t max_kept, void* out, int out_is_fp32,
+                           cudaStream_t s) {
+  const int max_len = (max_kept > 0 && max_kept < kv->max_seq_len) ? max_kept : kv->max_seq_len;
+  AttnLaunch a = make_launch(ctx, kv, q, true, max_len);
+  a.idx = idx;
+  a.kcount = k;
+  a.k_stride = k_stride;
+  FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
+  FASTOCR_TRY_CUDA(fastocr::launch_attn_combine(a, out, out_is_fp32, nullptr, s), "combine launch");
+  return FASTOCR_OK;
+}
+
+fastocr_status check_scores_args(fastocr_ctx* ctx, const fastocr_kv_view* kv, const float* scores_out, int32_t n_stride) {
+  if (scores_out == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL scores_out");
+  if (n_stride <= 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "n_stride must be positive");
+  (void)kv;
+  return FASTOCR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limits* lim) {
+  if (out == nullptr || lim == nullptr) return FASTOCR_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (lim->max_batch <= 0 || lim->num_q_heads <= 0 || lim->num_kv_heads <= 0 || lim->max_seq_len <= 0 ||
+      lim->max_vis_len < 0 || lim->num_q_heads % lim->num_kv_heads != 0)
+    return FASTOCR_ERR_INVALID_ARG;
+  if (lim->max_vis_len > fastocr::kTopkMaxN) return FASTOCR_ERR_UNSUPPORTED;
+  fastocr_ctx* ctx = new (std::nothrow) fastocr_ctx();
+  if (ctx == nullptr) return FASTOCR_ERR_WORKSPACE;
+  ctx->device = device;
+  ctx->lim = *lim;
+  cudaError_t e = cudaSetDevice(device);
+  int sm = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess) e = fastocr::configure_kernels();
+  if (e == cudaSuccess) e = fastocr::configure_topk();
+  if (e != cudaSuccess) {
+    delete ctx;
+    return FASTOCR_ERR_CUDA;
+  }
+  ctx->sm_count = sm > 0 ? sm : 148;
+  ctx->target_items = env_int("FASTOCR_TARGET_ITEMS", ctx->sm_count * 3 * 8);
+  ctx->min_chunk = env_int("FASTOCR_MIN_CHUNK", 128);
+  if (ctx->min_chunk < fastocr::kTokensPerCtaIter) ctx->min_chunk = fastocr::kTokensPerCtaIter;
+  const int64_t units = static_cast<int64_t>(lim->max_batch) * lim->num_kv_heads;
+  const int64_t min_chunks = (lim->max_seq_len + fastocr::kMaxChunk - 1) / fastocr::kMaxChunk;
+  ctx->cap_items = units * min_chunks;
+  if (ctx->cap_items < 2 * ctx->target_items) ctx->cap_items = 2 * ctx->target_items;
+  const int64_t nvis = lim->max_vis_len > 0 ? lim->max_vis_len : 1;
+  const size_t bytes_acc = static_cast<size_t>(ctx->cap_items) * fastocr::kMaxGroup * fastocr::kHeadDim * sizeof(float);
+  const size_t bytes_ml = static_cast<size_t>(ctx->cap_items) * fastocr::kMaxGroup * 2 * sizeof(float);
+  const size_t bytes_logits = static_cast<size_t>(lim->max_batch) * lim->num_q_heads * nvis * sizeof(float);
+  const size_t bytes_stats = static_cast<size_t>(lim->max_batch) * lim->num_q_heads * 2 * sizeof(float);
+  const size_t bytes_scores = static_cast<size_t>(lim->max_batch) * nvis * sizeof(float);
+  if ((e = cudaMalloc(&ctx->part_acc, bytes_acc)) != cudaSuccess || (e = cudaMalloc(&ctx->part_ml, bytes_ml)) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->logits, bytes_logits)) != cudaSuccess || (e = cudaMalloc(&ctx->stats, bytes_stats)) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->scores, bytes_scores)) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->faults, sizeof(unsigned long long))) != cudaSuccess ||
+      (e = cudaMemset(ctx->faults, 0, sizeof(unsigned long long))) != cudaSuccess) {
+    fastocr_destroy(ctx);
+    return e == cudaErrorMemoryAllocation ? FASTOCR_ERR_WORKSPACE : FASTOCR_ERR_CUDA;
+  }
+  *out = ctx;
+  return FASTOCR_OK;
+}
+
+void fastocr_destroy(fastocr_ctx* ctx) {
+  if (ctx == nullptr) return;
+  cudaSetDevice(ctx->device);
+  cudaFree(ctx->part_acc);
+  cudaFree(ctx->part_ml);
+  cudaFree(ctx->logits);
+  cudaFree(ctx->stats);
+  cudaFree(ctx->scores);
+  cudaFree(ctx->faults);
+  delete ctx;
+}
+
+const char* fastocr_last_error(const fastocr_ctx* ctx) { return ctx != nullptr ? ctx->err : "NULL context"; }
+
+int64_t fastocr_device_faults(fastocr_ctx* ctx) {
+  if (ctx == nullptr) return -1;
+  unsigned long long v = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+  if (cudaMemcpy(&v, ctx->faults, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  if (cudaMemset(ctx->faults, 0, sizeof v) != cudaSuccess) return -1;
+  return static_cast<int64_t>(v);
+}
+
+int32_t fastocr_kept_count(int32_t n_vis, double tau) {
+  if (n_vis <= 0 || !(tau > 0.0)) return 0;
+  if (tau >= 1.0) return n_vis;
+  const double c = std::ceil(tau * static_cast<double>(n_vis) - 1e-9);
+  if (c <= 0.0) return 0;
+  return c >= static_cast<double>(n_vis) ? n_vis : static_cast<int32_t>(c);
+}
+
+fastocr_status fastocr_dense_decode_attn(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, void* out,
+                                         int out_is_fp32, float* scores_out, int32_t n_stride, void* stream) {
+  fastocr_status st = check_view(ctx, kv, q, true);
+  if (st != FASTOCR_OK) return st;
+  if (out == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL out");
+  int32_t max_vis = 0;
+  if (scores_out != nullptr) {
+    if ((st = check_scores_args(ctx, kv, scores_out, n_stride)) != FASTOCR_OK) return st;
+    max_vis = n_stride < ctx->lim.max_vis_len ? n_stride : ctx->lim.max_vis_len;
+    if (ctx->lim.max_vis_len <= 0) return fail(ctx, FASTOCR_ERR_WORKSPACE, "context was created with max_vis_len = 0");
+  }
+  return dense_impl(ctx, kv, q, out, out_is_fp32, scores_out, n_stride, max_vis, static_cast<cudaStream_t>(stream));
+}
+
+fastocr_status fastocr_focal_scores(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, float* scores_out,
+                                    int32_t n_stride, float* image_mass_out, void* stream) {
+  fastocr_status st = check_view(ctx, kv, q, false);
+  if (st != FASTOCR_OK) return st;
+  if ((st = check_scores_args(ctx, kv, scores_out, n_stride)) != FASTOCR_OK) return st;
+  if (ctx->lim.max_vis_len <= 0) return fail(ctx, FASTOCR_ERR_WORKSPACE, "context was created with max_vis_len = 0");
+  const int32_t max_vis = n_stride < ctx->lim.max_vis_len ? n_stride : ctx->lim.max_vis_len;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = dense_impl(ctx, kv, q, nullptr, 0, scores_out, n_stride, max_vis, s);
+  if (st != FASTOCR_OK) return st;
+  if (image_mass_out != nullptr)
+    FASTOCR_TRY_CUDA(fastocr::launch_image_mass(scores_out, n_stride, kv->vis_len, kv->batch, image_mass_out, s), "image mass launch");
+  return FASTOCR_OK;
+}
+
+fastocr_status fastocr_select_topk(fastocr_ctx* ctx, const float* scores, int32_t n_stride, const int32_t* vis_len,
+                                   const int32_t* k, int32_t batch, int32_t max_vis_len, int32_t* idx_out,
+                                   int32_t k_stride, void* stream) {
+  if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
+  if (scores == nullptr || vis_len == nullptr || k == nullptr || idx_out == nullptr)
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL pointer argument");
+  if (batch <= 0 || n_stride <= 0 || k_stride <= 0 || max_vis_len <= 0 || max_vis_len > n_stride)
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "need batch, n_stride, k_stride > 0 and 0 < max_vis_len <= n_stride");
+  if (max_vis_len > fastocr::kTopkMaxN)
+    return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "max_vis_len %d exceeds %d", max_vis_len, fastocr::kTopkMaxN);
+  FASTOCR_TRY_CUDA(fastocr::launch_select_topk(scores, n_stride, vis_len, k, batch, max_vis_len, idx_out, k_stride,
+                                               static_cast<cudaStream_t>(stream)),
+                   "top-k launch");
+  return FASTOCR_OK;
+}
+
+fastocr_status fastocr_sparse_decode_attn(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q,
+                                          const int32_t* idx, const int32_t* k, int32_t k_stride, int32_t max_kept,
+                                          void* out, int out_is_fp32, void* stream) {
+  fastocr_status st = check_view(ctx, kv, q, true);
+  if (st != FASTOCR_OK) return st;
+  if (idx == nullptr || k == nullptr || out == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL idx, k or out");
+  if (k_stride <= 0 || max_kept < 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "k_stride must be positive, max_kept non-negative");
+  return sparse_impl(ctx, kv, q, idx, k, k_stride, max_kept, out, out_is_fp32, static_cast<cudaStream_t>(stream));
+}
+
+fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
+                                   const void* q, void* out, int out_is_fp32, const uint8_t* is_focal,
+                                   const int32_t* k, int32_t* fixation, int32_t k_stride, int has_fixation,
+                                   int32_t max_vis_len, int32_t max_kept, int* has_fixation_out, void* stream) {
+  if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
+  if (num_layers <= 0 || layers == nullptr || q == nullptr || out == nullptr || is_focal == nullptr || k == nullptr ||
+      fixation == nullptr)
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL pointer or num_layers <= 0");
+  if (k_stride <= 0 || max_vis_len <= 0 || max_vis_len > ctx->lim.max_vis_len)
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "k_stride / max_vis_len out of range (context max_vis_len %d)", ctx->lim.max_vis_len);
+  for (int l = 0; l < num_layers; ++l) {
+    fastocr_status st = check_view(ctx, &layers[l], q, true);
+    if (st != FASTOCR_OK) return st;
+    if (layers[l].batch != layers[0].batch || layers[l].num_q_heads != layers[0].num_q_heads ||
+        layers[l].num_kv_heads != layers[0].num_kv_heads)
+      return fail(ctx, FASTOCR_ERR_INVALID_ARG, "layer %d has a different batch / head geometry", l);
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t per_layer = static_cast<int64_t>(layers[0].batch) * layers[0].num_q_heads * fastocr::kHeadDim;
+  const size_t q_bytes = per_layer * 2, o_bytes = per_layer * (out_is_fp32 ? 4 : 2);
+  bool have = has_fixation != 0;
+  for (int l = 0; l < num_layers; ++l) {
+    const void* ql = static_cast<const char*>(q) + l * q_bytes;
+    void* ol = static_cast<char*>(out) + l * o_bytes;
+    const bool focal = is_focal[l] != 0;
+    fastocr_status st;
+    if (focal || (l == 0 && !have)) {
+      // full attention + scoring + selection; the refreshed set replaces the current one
+      st = dense_impl(ctx, &layers[l], ql, ol, out_is_fp32, ctx->scores, ctx->lim.max_vis_len, max_vis_len, s);
+      if (st != FASTOCR_OK) return st;
+      FASTOCR_TRY_CUDA(fastocr::launch_select_topk(ctx->scores, ctx->lim.max_vis_len, layers[l].vis_len, k, layers[l].batch,
+                                                   max_vis_len, fixation, k_stride, s),
+                       "top-k launch");
+      have = true;
+    } else {
+      st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, s);
+      if (st != FASTOCR_OK) return st;
+    }
+  }
+  if (has_fixation_out != nullptr) *has_fixation_out = have ? 1 : 0;
+  return FASTOCR_OK;
+}
+
+int32_t fastocr_focal_layers(const double* mean_ratio, int32_t num_layers, double rho, int32_t gap, int32_t* focal_out) {
+  if (mean_ratio == nullptr || focal_out == nullptr || num_layers <= 0 || gap < 0 || !(rho >= 0.0)) return -1;
+  const int budget = static_cast<int>(std::floor(rho * num_layers + 1e-9));
+  std::vector<char> used(num_layers, 0), chosen(num_layers, 0);
+  int count = 0;
+  // walk the layers from the highest mean ratio down (selection sort keeps ties in layer order)
+  for (int step = 0; step < num_layers && count < budget; ++step) {
+    int best = -1;
+    for (int l = 0; l < num_layers; ++l)
+      if (!used[l] && (best < 0 || mean_ratio[l] > mean_ratio[best])) best = l;
+    used[best] = 1;
+    bool far_enough = true;
+    for (int l = 0; l < num_layers; ++l)
+      if (chosen[l] && std::abs(l - best) <= gap) far_enough = false;
+    if (far_enough) {
+      chosen[best] = 1;
+      ++count;
+    }
+  }
+  int n = 0;
+  for (int l = 0; l < num_layers; ++l)
+    if (chosen[l]) focal_out[n++] = l;
+  return n;
+}
+
+double fastocr_attn_flops(double batch, double layers, double hidden, double seq_len) {
+  return batch * layers * (8.0 * hidden * hidden + 4.0 * hidden * seq_len);
+}
+
+int64_t fastocr_launch_count(void) { return fastocr::g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,68 @@
+// Internal launch interface between the C ABI (api.cu) and the kernels. Not installed.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fastocr {
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxGroup = 8;          // query heads per KV head handled by one CTA
+constexpr int kAttnWarps = 4;         // warps per attention CTA
+constexpr int kQuad = 4;              // tokens one warp consumes per pipeline stage
+constexpr int kTokensPerCtaIter = kAttnWarps * kQuad;
+constexpr int kMaxChunk = 4096;       // tokens per split (row table lives in shared memory)
+constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
+
+struct AttnLaunch {
+  // cache view
+  const void* k;
+  const void* v;              // nullptr: keys only (scores pass)
+  int64_t seq_stride_tokens;
+  const int32_t* block_table;
+  int32_t max_pages;
+  int32_t page_size;          // 0 = contiguous
+  const int32_t* seq_len;
+  const int32_t* vis_start;
+  const int32_t* vis_len;
+  int32_t batch, num_q_heads, num_kv_heads;
+  float sm_scale;
+  const void* q;
+  // pruned mode (idx != nullptr)
+  const int32_t* idx;
+  const int32_t* kcount;
+  int32_t k_stride;
+  // split geometry
+  int32_t chunk_tokens;       // multiple of kTokensPerCtaIter, <= kMaxChunk
+  int32_t max_chunks;         // grid.x
+  // workspace
+  float* part_acc;            // [B][Hkv][max_chunks][G][128]
+  float* part_ml;             // [B][Hkv][max_chunks][G][2]  (max, sum) in the log2 domain
+  float* logits;              // nullptr or [B][H][n_stride], log2-domain logits of image tokens
+  int32_t n_stride;
+  unsigned long long* fault_counter;
+};
+
+cudaError_t launch_attn_partial(const AttnLaunch& a, cudaStream_t s);
+
+// Merges the per-split partials of every (sequence, head): writes out (bf16 / fp32) unless out is
+// nullptr, and the global (max, sum) per head to stats [B][H][2] unless stats is nullptr.
+cudaError_t launch_attn_combine(const AttnLaunch& a, void* out, int out_is_fp32, float* stats, cudaStream_t s);
+
+// scores[b][i] = (1/H) sum_h 2^(logit[b][h][i] - max_h) / sum_h  for i < vis_len[b].
+cudaError_t launch_scores_finalize(const float* logits, const float* stats, const int32_t* vis_len, int32_t batch,
+                                   int32_t num_q_heads, int32_t n_stride_logits, int32_t max_vis_len, float* scores,
+                                   int32_t n_stride, cudaStream_t s);
+
+// mass[b] = sum_{i < vis_len[b]} scores[b][i], fixed summation order.
+cudaError_t launch_image_mass(const float* scores, int32_t n_stride, const int32_t* vis_len, int32_t batch,
+                              float* mass, cudaStream_t s);
+
+cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int32_t* vis_len, const int32_t* k,
+                               int32_t batch, int32_t max_vis_len, int32_t* idx_out, int32_t k_stride,
+                               cudaStream_t s);
+
+cudaError_t configure_kernels();   // one-time cudaFuncSetAttribute calls (current device)
+
+void count_launches(int n);
+
+}  // namespace fastocr
