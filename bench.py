@@ -1,0 +1,470 @@
+#!/usr/bin/env python
+"""Benchmark of the FastOCR decode-step attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one post-warm-up decode step of Algorithm 1 over all layers of the workload: focal
+layers run dense attention with fused scoring plus top-k, every other layer runs pruned attention
+over text + the current fixation set, the set of the deepest focal layer is carried to the next
+step. The default workload is the roofline-sweep point the target is stated on (7B-shaped heads,
+batch 64, N = 8192 image tokens, 256 text tokens, tau = 0.05) with 28 distinct layer caches
+(31 GB, far beyond L2) scheduled with rho = 0.1 as in the 7B-shaped decode configuration.
+
+Prints ONE JSON line (rank 0). Roofline figures use algorithmic bytes: the K and V rows the
+method must read (2 x H_kv x 128 x 2 bytes per attended token) plus the index list.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import fixation_track, get_config, make_kv, make_queries, make_page_table, scatter_to_pages  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--N", type=int, default=8192, help="image tokens (cfg4 only)")
+    ap.add_argument("--batch", type=int, default=64, help="sequences (cfg4 only)")
+    ap.add_argument("--tau", type=float, default=None)
+    ap.add_argument("--layers", type=int, default=None, help="override the number of layer caches")
+    ap.add_argument("--distinct-steps", type=int, default=16, help="length of the replayed fixation track")
+    ap.add_argument("--focal", default=None, help="comma-separated focal layers (skips Focal Layer Selection)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def workload_config(args):
+    if args.workload == "cfg4":
+        cfg = get_config("cfg4", N=args.N, batch=args.batch, layers=args.layers or 28)
+        cfg.name = f"cfg4[N={args.N},B={args.batch}]x{cfg.layers}layers"
+    else:
+        cfg = get_config(args.workload)
+        if args.layers:
+            cfg.layers = args.layers
+    if args.tau is not None:
+        cfg.tau = args.tau
+    return cfg
+
+
+class Workload:
+    """Device-resident synthetic decode state: per-layer caches, a cyclic track of `n_distinct`
+    decode steps (queries + sequence lengths), kept counts."""
+
+    def __init__(self, cfg, n_distinct, device, rank=0, seq_slice=None, device_api=True):
+        from workloads import kept_count_hint
+        fo = None
+        if device_api:
+            import paper_2605_17447_b200 as fo
+        self.cfg, self.dev, self.nd = cfg, device, n_distinct
+        B_all = cfg.batch
+        lo, hi = seq_slice or (0, B_all)
+        self.seqs = list(range(lo, hi))
+        B = self.B = hi - lo
+        self.seq_offset = rank * B_all + lo            # distinct data per rank (weak scaling)
+        self.H, self.Hkv, self.L = cfg.num_q_heads, cfg.num_kv_heads, cfg.layers
+        self.vis_start = [cfg.vis_start[b] for b in self.seqs]
+        self.vis_len = [cfg.vis_len[b] for b in self.seqs]
+        self.S0 = [cfg.seq_len(0)[b] for b in self.seqs]
+        self.text0 = [s - n for s, n in zip(self.S0, self.vis_len)]
+        self.k = [(fo.kept_count if fo else kept_count_hint)(n, cfg.tau) for n in self.vis_len]
+        self.S_stride = max(self.S0) + n_distinct
+        self.max_kept = max(k + t for k, t in zip(self.k, self.text0)) + n_distinct
+        self.sm_scale = 1.0 / math.sqrt(cfg.head_dim)
+        i32 = lambda x: torch.tensor(x, dtype=torch.int32, device=device)
+        self.vis_start_d, self.vis_len_d, self.k_d = i32(self.vis_start), i32(self.vis_len), i32(self.k)
+        # step s of the track attends S0 + s + 1 tokens (the current token included)
+        self.seq_len_table = torch.stack([i32([s0 + s + 1 for s0 in self.S0]) for s in range(n_distinct)])
+        self.seq_len_d = self.seq_len_table[0].clone()
+        gh = torch.tensor([cfg.grid_h[b] for b in self.seqs], device=device)
+        gw = torch.tensor([cfg.grid_w[b] for b in self.seqs], device=device)
+        tracks = np.stack([fixation_track(cfg.seed, self.seq_offset + i, n_distinct, cfg.grid_h[b], cfg.grid_w[b], cfg.advance)
+                           for i, b in enumerate(self.seqs)])                                 # [B][nd][2]
+        self.views, self.K, self.V = [], [], []
+        self.q_all = torch.empty(n_distinct, self.L, B, self.H, cfg.head_dim, dtype=torch.bfloat16, device=device)
+        self.block_table = None
+        if cfg.page_size:
+            table, self.num_pages = make_page_table(cfg.seed + rank, [self.S_stride] * B, cfg.page_size)
+            self.block_table = table.to(device)
+        for l in range(self.L):
+            K, V = make_kv(cfg.seed, l, B, self.S_stride, self.Hkv, cfg.head_dim, device, seq_offset=self.seq_offset)
+            for s in range(n_distinct):
+                centres = torch.tensor(tracks[:, s, :], device=device)
+                self.q_all[s, l] = make_queries(cfg.seed, l, s, lambda b, pos: K[b, pos], self.vis_start_d.long(), centres,
+                                                gh, gw, self.H, seq_offset=self.seq_offset)
+            if cfg.page_size:
+                K = scatter_to_pages(K, [self.S_stride] * B, self.block_table.cpu(), self.num_pages, cfg.page_size)
+                V = scatter_to_pages(V, [self.S_stride] * B, self.block_table.cpu(), self.num_pages, cfg.page_size)
+            self.K.append(K)
+            self.V.append(V)
+            if fo:
+                self.views.append(fo.KVView(K, V, self.seq_len_d, self.vis_start_d, self.vis_len_d, self.H, self.S_stride,
+                                            self.sm_scale, block_table=self.block_table))
+        self.fo = fo
+        if fo:
+            self.ctx = fo.Context(B, self.H, self.Hkv, self.S_stride, max(self.vis_len))
+            self.fix = torch.zeros(B, max(max(self.k), 1), dtype=torch.int32, device=device)
+
+    def flat_row(self, s):
+        """Row index (into the cache viewed as [rows][Hkv][d]) of the token appended at track step s."""
+        pos = torch.tensor([s0 + s for s0 in self.S0], device=self.dev)
+        b = torch.arange(self.B, device=self.dev)
+        if self.cfg.page_size:
+            ps = self.cfg.page_size
+            return self.block_table[b, pos // ps].long() * ps + pos % ps
+        return b * self.S_stride + pos
+
+    # ---- byte model: rows of K and V the method must read, bf16 ----
+    def row_bytes(self):
+        return self.Hkv * self.cfg.head_dim * 2
+
+    def dense_bytes(self, s):
+        return 2 * self.row_bytes() * sum(s0 + s + 1 for s0 in self.S0)
+
+    def sparse_bytes(self, s):
+        return 2 * self.row_bytes() * sum(k + t + s + 1 for k, t in zip(self.k, self.text0)) + 4 * sum(self.k)
+
+    def set_step(self, s):
+        self.seq_len_d.copy_(self.seq_len_table[s % self.nd])
+
+    def logical_rows(self, l, b, S):
+        """K, V rows [S][Hkv][d] of local sequence b, layer l, as CPU tensors (for the oracle)."""
+        if self.cfg.page_size:
+            ps = self.cfg.page_size
+            pages = self.block_table[b, :(S + ps - 1) // ps].long()
+            K = self.K[l][pages].reshape(-1, self.Hkv, self.cfg.head_dim)[:S]
+            V = self.V[l][pages].reshape(-1, self.Hkv, self.cfg.head_dim)[:S]
+        else:
+            K, V = self.K[l][b, :S], self.V[l][b, :S]
+        return K.cpu().contiguous(), V.cpu().contiguous()
+
+
+def choose_focal_layers(w: Workload):
+    """Focal Layer Selection (Section 3.1.1): w warm-up steps of full attention, record Eq. 1's
+    image-attention ratio per layer (batch mean), then rank + greedy gap. Untimed set-up."""
+    cfg, fo = w.cfg, w.fo
+    steps = max(1, min(cfg.warmup, w.nd))
+    scores = torch.zeros(w.B, max(w.vis_len), dtype=torch.float32, device=w.dev)
+    mass = torch.zeros(w.B, dtype=torch.float32, device=w.dev)
+    ratio = np.zeros((steps, w.L))
+    for s in range(steps):
+        w.set_step(s)
+        for l in range(w.L):
+            fo.fastocr_focal_scores(w.ctx, w.views[l], w.q_all[s, l], scores, image_mass_out=mass)
+            ratio[s, l] = float(mass.mean())
+    return fo.focal_layers(ratio.mean(axis=0), cfg.rho, cfg.gap), ratio.mean(axis=0)
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.strip().split(", ") for r in open(self.f.name) if r.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons, power = [], [], set(), []
+        for r in rows:
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2])); power.append(float(r[3]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if val.strip().lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [c for c, p in zip(sm, power) if p >= 0.5 * max(power)] or sm
+        return {"sm_mhz": float(np.median(busy)), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm),
+                "power_w_max": max(power)}
+
+
+def timed(fn, steps, dist_barrier):
+    dist_barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(steps):
+        fn(t)
+    e1.record()
+    torch.cuda.synchronize()
+    dist_barrier()
+    return e0.elapsed_time(e1)
+
+
+def oracle_step_sample(w: Workload, focal, seq_ids, s):
+    """The oracle's Algorithm-1 step for some sequences of track step s. Returns seconds of oracle
+    compute (input copies excluded) and the traces."""
+    import oracle
+    cfg = w.cfg
+    total, traces = 0.0, []
+    deepest = max(focal) if focal else 0
+    for b in seq_ids:
+        S = w.S0[b] + s + 1
+        layers = []
+        for l in range(w.L):
+            K, V = w.logical_rows(l, b, S)
+            layers.append((w.q_all[s % w.nd, l, b].cpu(), K, V))
+        # last step's fixation set, from the oracle's own scoring of the previous step
+        sp = (s - 1) % w.nd
+        Kp, _ = w.logical_rows(deepest, b, w.S0[b] + sp + 1)
+        sc, _ = oracle.scores(w.q_all[sp, deepest, b].cpu(), Kp, w.sm_scale, w.vis_start[b], w.vis_len[b])
+        f_last = oracle.topk(sc, w.k[b])
+        t0 = time.perf_counter()
+        tr = oracle.decode_step(layers, focal, f_last, w.vis_start[b], w.vis_len[b], cfg.tau, w.sm_scale)
+        total += time.perf_counter() - t0
+        traces.append(tr)
+    return total, traces
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload.
+    Each timed step is one sequence's Algorithm-1 step over a subset of the layers, sized so that
+    the whole run ends within a few minutes; the value is scaled to the full batch and depth."""
+    import oracle
+    cfg = workload_config(args)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"      # holds inputs only; the oracle runs on host cores
+    budget = 120.0 / max(1, args.steps + args.warmup)         # seconds of oracle time per step
+    threads = max(1, min(oracle.num_threads(), cfg.num_q_heads))
+    S = cfg.seq_len(0)[0]
+    per_layer = 4e-9 * cfg.num_q_heads * cfg.head_dim * S * (3 * cfg.rho + 0.15) / threads   # rough
+    n_layers = cfg.layers
+    while n_layers > 4 and per_layer * n_layers > budget:
+        n_layers = max(4, n_layers // 2)
+    sub = workload_config(args)
+    sub.layers = n_layers
+    w = Workload(sub, 2, dev, seq_slice=(0, 1), device_api=False)
+    ratios = []
+    for l in range(n_layers):                                  # one warm-up step of Eq. 1 per layer
+        K, _ = w.logical_rows(l, 0, w.S0[0] + 1)
+        ratios.append(oracle.scores(w.q_all[0, l, 0].cpu(), K, w.sm_scale, w.vis_start[0], w.vis_len[0])[1])
+    focal = oracle.profile_focal_layers([ratios], max(cfg.rho, 1.0 / n_layers), cfg.gap)
+    for _ in range(args.warmup):
+        oracle_step_sample(w, focal, [0], 1)
+    t = 0.0
+    for _ in range(args.steps):
+        dt, _ = oracle_step_sample(w, focal, [0], 1)
+        t += dt
+    per_step_full = t / max(1, args.steps) * cfg.batch * (cfg.layers / n_layers) * 1e6
+    sample = (f"1 of {cfg.batch} sequences, {n_layers} of {cfg.layers} layers ({len(focal)} focal), "
+              f"scaled to the full batch and depth")
+    line = {"impl": "reference", "metric": "fastocr decode-attention step time", "value": per_step_full, "unit": "us/step",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step_full / 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "tau": cfg.tau, "rho": cfg.rho},
+            "cpu_baseline": {"value": per_step_full, "unit": "us/step", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": per_step_full, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+    barrier = (lambda: dist.barrier()) if dist else (lambda: None)
+
+    import paper_2605_17447_b200 as fo
+    cfg = workload_config(args)
+    peak, peak_kind = measured_peaks()
+    # sequences are independent: every rank holds its own full batch (weak scaling), no data-path collective
+    w = Workload(cfg, args.distinct_steps, dev, rank=rank)
+    if args.focal is not None:
+        focal = sorted(int(x) for x in args.focal.split(",") if x != "")
+    else:
+        focal, _ = choose_focal_layers(w)
+    is_focal = [l in focal for l in range(w.L)]
+    out = torch.empty(w.L, w.B, w.H, cfg.head_dim, dtype=torch.bfloat16, device=dev)
+    plan = fo.StepPlan(w.ctx, w.views, is_focal, w.k_d, w.fix, max(w.vis_len), w.max_kept)
+    state = {"have": False}
+
+    def fastocr_step(t):
+        w.set_step(t)
+        state["have"] = plan.run(w.q_all[t % w.nd], out, state["have"])
+
+    def dense_step(t):
+        w.set_step(t)
+        for l in range(w.L):
+            fo.fastocr_dense_decode_attn(w.ctx, w.views[l], w.q_all[t % w.nd, l], out[l])
+
+    for t in range(max(3, args.warmup)):
+        fastocr_step(t)
+    launches0 = fo.launch_count()
+    clocks = ClockSampler(local)
+    ms = timed(fastocr_step, args.steps, barrier)
+    clock_info = clocks.stop()
+    launches = fo.launch_count() - launches0
+    dense_steps = max(3, min(args.steps, 20))
+    for t in range(3):
+        dense_step(t)
+    ms_dense = timed(dense_step, dense_steps, barrier) / dense_steps
+
+    # per-kernel average durations over the same steps (events around every launch)
+    prof_steps = min(args.steps, 50)
+    w.ctx.profile_begin(prof_steps * (w.L * 4 + 8))
+    for t in range(prof_steps):
+        fastocr_step(t)
+    prof = w.ctx.profile_end()
+
+    if dist:
+        tt = torch.tensor([ms, ms_dense], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms, ms_dense = float(tt[0]), float(tt[1])
+    us_step = ms / args.steps * 1e3
+
+    n_focal = len(focal)
+    mean_s = (w.nd - 1) / 2.0
+    sparse_b = w.sparse_bytes(mean_s)
+    dense_b = w.dense_bytes(mean_s)
+    step_bytes = n_focal * dense_b + (w.L - n_focal) * sparse_b
+    kern = {}
+    for name, bytes_per in (("attn_sparse", sparse_b), ("attn_dense", dense_b)):
+        tot, n = prof[name]
+        if n:
+            us = tot / n * 1e3
+            kern[name] = {"us_per_launch": us, "launches_per_step": n / prof_steps, "algorithmic_bytes": bytes_per,
+                          "gbs": bytes_per / us / 1e3, "frac_of_measured": bytes_per / us / 1e3 / peak,
+                          "frac_of_8tbs": bytes_per / us / 1e3 / NOMINAL_HBM_GBS}
+    for name in ("combine", "scores_finalize", "select_topk"):
+        tot, n = prof[name]
+        if n:
+            kern[name] = {"us_per_launch": tot / n * 1e3, "launches_per_step": n / prof_steps}
+    share = {name: prof[name][0] for name in prof if prof[name][1]}
+    dominant = max(("attn_sparse", "attn_dense"), key=lambda n: share.get(n, 0.0))
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(tpath):
+        traffic = json.load(open(tpath)).get(dominant, {}).get("traffic_bytes_per_launch")
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": kern[dominant]["gbs"], "peak": peak, "unit": "GB/s",
+                "frac": kern[dominant]["frac_of_measured"], "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                "frac_of_8tbs": kern[dominant]["frac_of_8tbs"]}
+
+    # ---- end to end: per step, pinned-host queries + the new token's K/V rows in, outputs back ----
+    e2e = None
+    if not args.no_e2e:
+        q_host = w.q_all.cpu().pin_memory()                                         # [nd][L][B][H][d]
+        rows = [w.flat_row(s) for s in range(w.nd)]                                 # step s appends position S0+s
+        flatK = [k.view(-1, w.Hkv, cfg.head_dim) for k in w.K]
+        flatV = [v.view(-1, w.Hkv, cfg.head_dim) for v in w.V]
+        newkv_host = torch.stack([torch.stack([torch.stack([flatK[l][rows[s]], flatV[l][rows[s]]]) for l in range(w.L)])
+                                  for s in range(w.nd)]).cpu().pin_memory()         # [nd][L][2][B][Hkv][d]
+        out_host = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        q_dev = torch.empty_like(w.q_all[0])
+        newkv_dev = torch.empty(newkv_host.shape[1:], dtype=newkv_host.dtype, device=dev)
+
+        def e2e_step(t):
+            s = t % w.nd
+            w.set_step(t)
+            q_dev.copy_(q_host[s], non_blocking=True)
+            newkv_dev.copy_(newkv_host[s], non_blocking=True)
+            for l in range(w.L):                        # append the current token's K/V rows to every layer's cache
+                flatK[l].index_copy_(0, rows[s], newkv_dev[l, 0])
+                flatV[l].index_copy_(0, rows[s], newkv_dev[l, 1])
+            state["have"] = plan.run(q_dev, out, state["have"])
+            out_host.copy_(out, non_blocking=True)
+
+        for t in range(3):
+            e2e_step(t)
+        e2e_steps = min(args.steps, 50)
+        ms_e2e = timed(e2e_step, e2e_steps, barrier) / e2e_steps
+        if dist:
+            tt = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms_e2e = float(tt[0])
+        e2e = {"value": ms_e2e * 1e3, "unit": "us/step",
+               "h2d_bytes_per_step": int(q_host[0].numel() * 2 + newkv_host[0].numel() * 2),
+               "d2h_bytes_per_step": int(out_host.numel() * out_host.element_size()),
+               "note": "per step: pinned-host queries and the new token's K/V rows in (appended to every layer's cache), "
+                       "all layer outputs back to pinned host memory; the KV cache itself is resident by definition"}
+
+    cpu_base = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        dt1, _ = oracle_step_sample(w, focal, [0], 1)
+        n_s = int(max(1, min(w.B, args.cpu_seconds / max(dt1, 1e-3))))
+        dt, _ = oracle_step_sample(w, focal, list(range(n_s)), 1)
+        cpu_base = {"value": dt / n_s * w.B * 1e6, "unit": "us/step", "cores": oracle.num_threads(), "kind": "oracle",
+                    "sample": f"{n_s} of {w.B} sequences, all {w.L} layers, one step ({dt:.2f} s of oracle time), scaled to the batch"}
+
+    if rank == 0:
+        line = {
+            "metric": "fastocr decode-attention step time", "value": us_step, "unit": "us/step", "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": us_step / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "layers": w.L, "focal_layers": focal, "batch_per_gpu": w.B, "global_batch": w.B * world,
+                       "num_q_heads": w.H, "num_kv_heads": w.Hkv, "head_dim": cfg.head_dim, "vis_tokens": [min(w.vis_len), max(w.vis_len)],
+                       "text_tokens": [min(w.text0), max(w.text0)], "tau": cfg.tau, "rho": cfg.rho, "gap": cfg.gap, "kept": [min(w.k), max(w.k)],
+                       "kv_dtype": "bf16", "paged": bool(cfg.page_size), "cache_bytes": int(sum(k.numel() * 4 for k in w.K)),
+                       "l2": "inputs larger than L2: every layer has its own cache and the step cycles through all of them",
+                       "parallelism": f"dp{world} (sequences sharded, no collective)"},
+            "dense_us_per_step": ms_dense * 1e3, "speedup_vs_dense": ms_dense * 1e3 / us_step,
+            "step_algorithmic_bytes": step_bytes, "step_gbs": step_bytes / us_step / 1e3,
+            "step_frac_of_8tbs": step_bytes / us_step / 1e3 / NOMINAL_HBM_GBS, "step_frac_of_measured": step_bytes / us_step / 1e3 / peak,
+            "dense_step_gbs": w.L * dense_b / (ms_dense * 1e3) / 1e3,
+            "kernels": kern, "roofline": roofline, "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clock_info,
+        }
+        print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

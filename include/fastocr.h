@@ -180,6 +180,27 @@ int32_t fastocr_focal_layers(const double* mean_ratio, int32_t num_layers, doubl
 /* Appendix B: self-attention FLOPs of one decode step, b*l*(8h^2 + 4hs). Host-only. */
 double fastocr_attn_flops(double batch, double layers, double hidden, double seq_len);
 
+/*
+ * Optional per-kernel timing (the paper has no counterpart; measurement aid). Between
+ * fastocr_profile_begin and fastocr_profile_end every launch of this context is bracketed by CUDA
+ * events on its stream. fastocr_profile_begin creates `max_launches` event pairs (not a hot-path
+ * call; launches beyond that are not timed); fastocr_profile_end synchronises, adds up elapsed
+ * milliseconds and launch counts per kernel class into the two host arrays of length
+ * FASTOCR_PROF_CLASSES, and destroys the events. Do not use while a stream is being captured.
+ */
+enum {
+  FASTOCR_PROF_ATTN_DENSE = 0,  /* split-KV attention kernel, full cache, K and V          */
+  FASTOCR_PROF_ATTN_KEYS = 1,   /* same kernel, keys only (stand-alone scoring)             */
+  FASTOCR_PROF_ATTN_SPARSE = 2, /* same kernel over the kept set                            */
+  FASTOCR_PROF_COMBINE = 3,     /* split merge                                              */
+  FASTOCR_PROF_FINALIZE = 4,    /* logits -> head-averaged scores                           */
+  FASTOCR_PROF_TOPK = 5,        /* selection                                                */
+  FASTOCR_PROF_MASS = 6,        /* image-mass reduction                                     */
+  FASTOCR_PROF_CLASSES = 7
+};
+fastocr_status fastocr_profile_begin(fastocr_ctx* ctx, int32_t max_launches);
+fastocr_status fastocr_profile_end(fastocr_ctx* ctx, double* ms_per_class, int64_t* launches_per_class);
+
 /* Number of kernels this library has launched on any context since load (for bench accounting). */
 int64_t fastocr_launch_count(void);
 

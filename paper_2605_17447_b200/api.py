@@ -18,6 +18,9 @@ from . import _lib
 _STATUS = {1: "invalid argument", 2: "unsupported", 3: "workspace limits exceeded", 4: "CUDA error"}
 
 
+PROF_CLASSES = ("attn_dense", "attn_keys", "attn_sparse", "combine", "scores_finalize", "select_topk", "image_mass")
+
+
 class FastOCRError(RuntimeError):
     def __init__(self, code: int, msg: str):
         super().__init__(f"fastocr: {_STATUS.get(code, code)}: {msg}")
@@ -118,6 +121,16 @@ class Context:
     def device_faults(self) -> int:
         return int(self._lib.fastocr_device_faults(self._h))
 
+    def profile_begin(self, max_launches: int) -> None:
+        self.check(self._lib.fastocr_profile_begin(self._h, int(max_launches)))
+
+    def profile_end(self):
+        """-> {class name: (total ms, launches)} for the launches since profile_begin."""
+        ms = (C.c_double * len(PROF_CLASSES))()
+        n = (C.c_int64 * len(PROF_CLASSES))()
+        self.check(self._lib.fastocr_profile_end(self._h, ms, n))
+        return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(PROF_CLASSES)}
+
 
 def kept_count(n_vis: int, tau: float) -> int:
     return int(_lib.load().fastocr_kept_count(int(n_vis), float(tau)))
@@ -198,3 +211,29 @@ def fastocr_decode_step(ctx: Context, layers: Sequence[KVView], q: torch.Tensor,
                                            int(bool(has_fixation)), int(max_vis_len), int(max_kept), C.byref(have),
                                            _stream(stream)))
     return bool(have.value)
+
+
+class StepPlan:
+    """fastocr_decode_step with everything that does not change between steps marshalled once
+    (the per-step Python cost is then a single foreign call)."""
+
+    def __init__(self, ctx: Context, layers: Sequence[KVView], is_focal: Sequence[bool], k: torch.Tensor,
+                 fixation: torch.Tensor, max_vis_len: int, max_kept: int = 0):
+        self.ctx = ctx
+        self.L = len(layers)
+        self._keep = (list(layers), k, fixation)
+        self._arr = (_lib.KVViewStruct * self.L)(*[kv.struct() for kv in layers])
+        self._focal = np.ascontiguousarray(np.asarray(is_focal, dtype=np.uint8))
+        self._k = _ptr(_dev(k, torch.int32, "k"))
+        self._fix = _ptr(_dev(fixation, torch.int32, "fixation"))
+        self._k_stride = int(fixation.shape[-1])
+        self._max_vis, self._max_kept = int(max_vis_len), int(max_kept)
+        self._have = C.c_int(0)
+
+    def run(self, q: torch.Tensor, out: torch.Tensor, has_fixation: bool, stream=None) -> bool:
+        c = self.ctx
+        c.check(c._lib.fastocr_decode_step(c._h, self.L, self._arr, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()),
+                                           int(out.dtype == torch.float32), self._focal.ctypes.data, self._k, self._fix,
+                                           self._k_stride, int(bool(has_fixation)), self._max_vis, self._max_kept,
+                                           C.byref(self._have), _stream(stream)))
+        return bool(self._have.value)

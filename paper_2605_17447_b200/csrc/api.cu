@@ -35,6 +35,11 @@ struct fastocr_ctx {
   int target_items = 0;         // tuning: desired number of CTAs per attention launch
   int min_chunk = 0;            // tuning: smallest split, tokens
   char err[512] = {0};
+  // optional per-launch timing
+  std::vector<cudaEvent_t> prof_ev;   // 2 per timed launch
+  std::vector<int> prof_class;
+  size_t prof_used = 0;
+  bool prof_on = false;
 };
 
 namespace {
@@ -137,6 +142,26 @@ fastocr_status cuda_fail(fastocr_ctx* ctx, cudaError_t e, const char* what) {
   return fail(ctx, FASTOCR_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
+// Brackets one launch with events when profiling is on.
+struct ProfScope {
+  fastocr_ctx* ctx;
+  cudaStream_t s;
+  bool armed = false;
+  ProfScope(fastocr_ctx* c, int cls, cudaStream_t st) : ctx(c), s(st) {
+    if (c->prof_on && c->prof_used + 2 <= c->prof_ev.size()) {
+      armed = true;
+      c->prof_class.push_back(cls);
+      cudaEventRecord(c->prof_ev[c->prof_used], st);
+    }
+  }
+  ~ProfScope() {
+    if (armed) {
+      cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s);
+      ctx->prof_used += 2;
+    }
+  }
+};
+
 #define FASTOCR_TRY_CUDA(expr, what)                         \
   do {                                                       \
     cudaError_t e_ = (expr);                                 \
@@ -152,12 +177,20 @@ fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
     a.logits = ctx->logits;
     a.n_stride = ctx->lim.max_vis_len;
   }
-  FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
-  FASTOCR_TRY_CUDA(fastocr::launch_attn_combine(a, out, out_is_fp32, want_scores ? ctx->stats : nullptr, s), "combine launch");
-  if (want_scores)
+  {
+    ProfScope p(ctx, out != nullptr ? FASTOCR_PROF_ATTN_DENSE : FASTOCR_PROF_ATTN_KEYS, s);
+    FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
+  }
+  {
+    ProfScope p(ctx, FASTOCR_PROF_COMBINE, s);
+    FASTOCR_TRY_CUDA(fastocr::launch_attn_combine(a, out, out_is_fp32, want_scores ? ctx->stats : nullptr, s), "combine launch");
+  }
+  if (want_scores) {
+    ProfScope p(ctx, FASTOCR_PROF_FINALIZE, s);
     FASTOCR_TRY_CUDA(fastocr::launch_scores_finalize(ctx->logits, ctx->stats, kv->vis_len, kv->batch, kv->num_q_heads,
                                                      ctx->lim.max_vis_len, max_vis, scores_out, n_stride, s),
                      "score finalisation launch");
+  }
   return FASTOCR_OK;
 }
 
@@ -169,8 +202,14 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
   a.idx = idx;
   a.kcount = k;
   a.k_stride = k_stride;
-  FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
-  FASTOCR_TRY_CUDA(fastocr::launch_attn_combine(a, out, out_is_fp32, nullptr, s), "combine launch");
+  {
+    ProfScope p(ctx, FASTOCR_PROF_ATTN_SPARSE, s);
+    FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
+  }
+  {
+    ProfScope p(ctx, FASTOCR_PROF_COMBINE, s);
+    FASTOCR_TRY_CUDA(fastocr::launch_attn_combine(a, out, out_is_fp32, nullptr, s), "combine launch");
+  }
   return FASTOCR_OK;
 }
 
@@ -286,8 +325,10 @@ fastocr_status fastocr_focal_scores(fastocr_ctx* ctx, const fastocr_kv_view* kv,
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   st = dense_impl(ctx, kv, q, nullptr, 0, scores_out, n_stride, max_vis, s);
   if (st != FASTOCR_OK) return st;
-  if (image_mass_out != nullptr)
+  if (image_mass_out != nullptr) {
+    ProfScope p(ctx, FASTOCR_PROF_MASS, s);
     FASTOCR_TRY_CUDA(fastocr::launch_image_mass(scores_out, n_stride, kv->vis_len, kv->batch, image_mass_out, s), "image mass launch");
+  }
   return FASTOCR_OK;
 }
 
@@ -301,6 +342,7 @@ fastocr_status fastocr_select_topk(fastocr_ctx* ctx, const float* scores, int32_
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "need batch, n_stride, k_stride > 0 and 0 < max_vis_len <= n_stride");
   if (max_vis_len > fastocr::kTopkMaxN)
     return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "max_vis_len %d exceeds %d", max_vis_len, fastocr::kTopkMaxN);
+  ProfScope p(ctx, FASTOCR_PROF_TOPK, static_cast<cudaStream_t>(stream));
   FASTOCR_TRY_CUDA(fastocr::launch_select_topk(scores, n_stride, vis_len, k, batch, max_vis_len, idx_out, k_stride,
                                                static_cast<cudaStream_t>(stream)),
                    "top-k launch");
@@ -347,9 +389,12 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
       // full attention + scoring + selection; the refreshed set replaces the current one
       st = dense_impl(ctx, &layers[l], ql, ol, out_is_fp32, ctx->scores, ctx->lim.max_vis_len, max_vis_len, s);
       if (st != FASTOCR_OK) return st;
-      FASTOCR_TRY_CUDA(fastocr::launch_select_topk(ctx->scores, ctx->lim.max_vis_len, layers[l].vis_len, k, layers[l].batch,
-                                                   max_vis_len, fixation, k_stride, s),
-                       "top-k launch");
+      {
+        ProfScope p(ctx, FASTOCR_PROF_TOPK, s);
+        FASTOCR_TRY_CUDA(fastocr::launch_select_topk(ctx->scores, ctx->lim.max_vis_len, layers[l].vis_len, k, layers[l].batch,
+                                                     max_vis_len, fixation, k_stride, s),
+                         "top-k launch");
+      }
       have = true;
     } else {
       st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, s);
@@ -387,6 +432,43 @@ int32_t fastocr_focal_layers(const double* mean_ratio, int32_t num_layers, doubl
 
 double fastocr_attn_flops(double batch, double layers, double hidden, double seq_len) {
   return batch * layers * (8.0 * hidden * hidden + 4.0 * hidden * seq_len);
+}
+
+fastocr_status fastocr_profile_begin(fastocr_ctx* ctx, int32_t max_launches) {
+  if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
+  if (max_launches <= 0 || ctx->prof_on) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "profile_begin: bad size or already profiling");
+  cudaSetDevice(ctx->device);
+  ctx->prof_ev.assign(static_cast<size_t>(max_launches) * 2, nullptr);
+  for (auto& ev : ctx->prof_ev) FASTOCR_TRY_CUDA(cudaEventCreate(&ev), "cudaEventCreate");
+  ctx->prof_class.clear();
+  ctx->prof_class.reserve(max_launches);
+  ctx->prof_used = 0;
+  ctx->prof_on = true;
+  return FASTOCR_OK;
+}
+
+fastocr_status fastocr_profile_end(fastocr_ctx* ctx, double* ms_per_class, int64_t* launches_per_class) {
+  if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
+  if (!ctx->prof_on || ms_per_class == nullptr || launches_per_class == nullptr)
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "profile_end: not profiling or NULL output");
+  ctx->prof_on = false;
+  for (int c = 0; c < FASTOCR_PROF_CLASSES; ++c) {
+    ms_per_class[c] = 0.0;
+    launches_per_class[c] = 0;
+  }
+  cudaError_t e = cudaDeviceSynchronize();
+  for (size_t i = 0; e == cudaSuccess && i + 2 <= ctx->prof_used && i / 2 < ctx->prof_class.size(); i += 2) {
+    float ms = 0.f;
+    e = cudaEventElapsedTime(&ms, ctx->prof_ev[i], ctx->prof_ev[i + 1]);
+    ms_per_class[ctx->prof_class[i / 2]] += ms;
+    launches_per_class[ctx->prof_class[i / 2]] += 1;
+  }
+  for (auto ev : ctx->prof_ev) cudaEventDestroy(ev);
+  ctx->prof_ev.clear();
+  ctx->prof_class.clear();
+  ctx->prof_used = 0;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "profile_end");
+  return FASTOCR_OK;
 }
 
 int64_t fastocr_launch_count(void) { return fastocr::g_launches.load(std::memory_order_relaxed); }

@@ -277,11 +277,11 @@ def test_argument_errors_are_reported_not_launched(fo, ctx):
     q = case.q.cuda()
     out = torch.empty(1, 28, 128, dtype=torch.float32, device="cuda")
     before = fo.launch_count()
-    bad = case.device_view()
-    bad.max_seq_len = 10 ** 6                                   # beyond the context limits
-    with pytest.raises(fo.FastOCRError) as e:
-        fo.fastocr_dense_decode_attn(ctx, bad, q, out)
+    small = fo.Context(max_batch=1, num_q_heads=28, num_kv_heads=4, max_seq_len=32, max_vis_len=64)
+    with pytest.raises(fo.FastOCRError) as e:                   # 72 cached tokens > the context's 32
+        fo.fastocr_dense_decode_attn(small, kv, q, out)
     assert e.value.code == 3
+    small.close()
     bad = case.device_view()
     bad.num_q_heads = 12                                        # group of 3: unsupported
     with pytest.raises(fo.FastOCRError) as e:

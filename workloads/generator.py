@@ -89,10 +89,13 @@ def make_kv(seed: int, layer: int, batch: int, tokens: int, num_kv_heads: int, h
     outs = []
     for tensor_id in (0, 1):
         key = stream_key(seed, 101, layer, tensor_id)
-        t = torch.empty(batch, tokens, num_kv_heads, head_dim, dtype=torch.bfloat16, device=device)
-        for b in range(batch):
-            t[b] = normal_bf16(key, (tokens, num_kv_heads, head_dim), device,
-                               offset=(b + seq_offset) * stride * row)
+        if stride == tokens:      # the whole tensor is one contiguous counter range
+            t = normal_bf16(key, (batch, tokens, num_kv_heads, head_dim), device, offset=seq_offset * stride * row)
+        else:
+            t = torch.empty(batch, tokens, num_kv_heads, head_dim, dtype=torch.bfloat16, device=device)
+            for b in range(batch):
+                t[b] = normal_bf16(key, (tokens, num_kv_heads, head_dim), device,
+                                   offset=(b + seq_offset) * stride * row)
         outs.append(t)
     return outs[0], outs[1]
 
