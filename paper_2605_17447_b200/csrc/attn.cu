@@ -4,19 +4,25 @@
 //
 // Work decomposition: CTA = (split c, KV head g, sequence b). The CTA first builds, in shared
 // memory, the table of physical cache rows of the tokens it attends (this is the only place where
-// dense / pruned / paged differ), then its warps stream those rows.
+// dense / pruned / paged differ), then each of its warps streams 16-token blocks of those rows.
 //
-// Data path: each lane owns 16 bytes (8 bf16) of a 256-byte K or V row; 16 lanes cover a row, so a
-// warp handles two tokens side by side and four tokens per pipeline stage. Rows travel
-// HBM -> shared memory with 16-byte cp.async into a per-lane ring (kStages deep, no cross-thread
-// hand-off, hence no barrier in the main loop) and are consumed with ld.shared.v4.
-// Arithmetic: fp32 throughout, issued as packed fma.rn.f32x2 so that the FMA pipe, not the issue
-// port, is the limit; one K row is dotted with all G query heads of the group while in registers.
-// Partial dot products are combined across the 16 lanes with a reduce-scatter (15 shuffles per 16
-// values) that leaves each (token, head) logit in exactly one lane, which applies the online
-// softmax; probabilities are handed back to all lanes through a 128-byte shared-memory slot.
-// The running maximum is only raised when a logit exceeds it by more than 2^8 (the accumulators
-// stay in range and the rescale branch is rare).
+// Data path: every lane copies, with 16-byte cp.async, exactly the K and V bytes it will later
+// need as tensor-core fragments into its own slots of a shared-memory ring (kStages deep; no
+// cross-thread hand-off, hence no barrier in the main loop) and reads them back with ld.shared.v4.
+//
+// Arithmetic: with a GQA group of 7 or 8 query heads per KV head, q.K^T and P.V are skinny matrix
+// products ([16 tokens x 128] x [128 x 8 heads]); on the fp32 CUDA cores they need more issue slots
+// than the HBM stream leaves time for, so both run on the tensor cores as warp-level
+// mma.sync.m16n8k16 (bf16 inputs, fp32 accumulation):
+//   S^T[head][token] = Q[head][d] . K^T[d][token]   (heads on M, padded to 16; 8 tokens per tile)
+//   O^T[d][head]    += V^T[d][token] . P[token][head] (16 dims per tile; 16 tokens on K)
+// The accumulator layout of S^T is exactly the B-operand layout P needs, so probabilities never
+// leave registers. bf16 products are exact in fp32; P is split into a bf16 high part and a bf16
+// remainder (two MMAs) so that the weighted sum keeps about 16 bits of P. The contraction index
+// order inside an MMA is free, which lets every fragment be a plain 16-byte row segment: K needs
+// no transposition at all, V^T is formed from pairs of rows with two byte-permutes per register.
+// The online softmax keeps a per-head running maximum that is raised only when a logit exceeds
+// it by more than 2^8, so the rescale branch is rare.
 #include "kernels.h"
 
 #include <cuda_bf16.h>
@@ -24,34 +30,11 @@
 namespace fastocr {
 namespace {
 
-constexpr int kStages = 6;
+constexpr int kStages = 3;
 constexpr int kThreads = kAttnWarps * 32;
+constexpr int kBlockTokens = 16;        // tokens per warp per pipeline stage
 constexpr float kRescaleSlack = 8.0f;   // log2 units
 
-typedef unsigned long long u64;
-
-__device__ __forceinline__ u64 pack2(float lo, float hi) {
-  u64 r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ u64 ffma2(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ u64 fmul2(u64 a, u64 b) {
-  u64 d;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-// two bf16 packed in a 32-bit word -> (low element, high element) widened exactly to fp32
-__device__ __forceinline__ u64 widen2(uint32_t w) {
-  return pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-}
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -69,6 +52,18 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 r;
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr) : "memory");
   return r;
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 struct SeqGeom {
@@ -90,24 +85,25 @@ __device__ __forceinline__ SeqGeom load_geom(const AttnLaunch& a, int b) {
   return s;
 }
 
-// shared-memory carve-up (bytes)
+// shared-memory carve-up (bytes). A stage holds, per lane, 8 K slots (+ 8 V slots) of 16 bytes.
 template <bool HAS_V>
 struct Smem {
-  static constexpr int kSlots = HAS_V ? 4 : 2;
-  static constexpr int kRingBytes = kAttnWarps * kStages * kSlots * 32 * 16;
-  static constexpr int kProbBytes = kAttnWarps * 2 * 32 * 4;
+  static constexpr int kSlots = HAS_V ? 16 : 8;
+  static constexpr int kStageBytes = kSlots * 32 * 16;             // per warp
+  static constexpr int kRingBytes = kAttnWarps * kStages * kStageBytes;
+  static constexpr int kMergeBytes = (kAttnWarps * 16 + kAttnWarps * kMaxGroup * kHeadDim) * 4;
   static constexpr int ring = 0;
-  static constexpr int prob = kRingBytes;
-  static constexpr int rows = kRingBytes + kProbBytes;       // int32 [chunk_tokens]
+  static constexpr int rows = kRingBytes > kMergeBytes ? kRingBytes : kMergeBytes;   // int32 [chunk_tokens]
   static int total(int chunk_tokens) { return rows + chunk_tokens * 4; }
 };
 
 template <int G, bool HAS_V>
-__global__ void __launch_bounds__(kThreads, 3) attn_partial_kernel(const AttnLaunch a) {
+__global__ void __launch_bounds__(kThreads, 2) attn_partial_kernel(const AttnLaunch a) {
   extern __shared__ __align__(16) unsigned char smem[];
   using L = Smem<HAS_V>;
   const int c = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, l16 = lane & 15, half = lane >> 4;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g8 = lane >> 2, t4 = lane & 3;             // MMA fragment coordinates: group, thread-in-group
 
   const SeqGeom sg = load_geom(a, b);
   const int start = c * a.chunk_tokens;
@@ -139,48 +135,54 @@ __global__ void __launch_bounds__(kThreads, 3) attn_partial_kernel(const AttnLau
     rows_s[i] = row;
   }
 
-  // ---- queries of this KV group, pre-scaled to the log2 domain, as f32x2 pairs ----------------
-  u64 q2[G][4];
+  // ---- A fragments of Q: lane (g8, t4) holds head g8, dims 32j + 8 t4 .. + 8 (j = 0..3) -------
+  uint32_t qw[4][4];
   {
-    const float qs = a.sm_scale * 1.4426950408889634f;
     const uint4* qp = reinterpret_cast<const uint4*>(a.q) +
-                      (static_cast<int64_t>(b) * a.num_q_heads + static_cast<int64_t>(g) * G) * (kHeadDim / 8) + l16;
+                      (static_cast<int64_t>(b) * a.num_q_heads + static_cast<int64_t>(g) * G + g8) * (kHeadDim / 8) + t4;
 #pragma unroll
-    for (int h = 0; h < G; ++h) {
-      const uint4 w = __ldg(qp + h * (kHeadDim / 8));
-      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        q2[h][i] = pack2(__uint_as_float(ww[i] << 16) * qs, __uint_as_float(ww[i] & 0xffff0000u) * qs);
-      }
+    for (int j = 0; j < 4; ++j) {
+      uint4 w = make_uint4(0u, 0u, 0u, 0u);
+      if (g8 < G) w = __ldg(qp + 4 * j);
+      qw[j][0] = w.x; qw[j][1] = w.y; qw[j][2] = w.z; qw[j][3] = w.w;
     }
   }
   __syncthreads();
 
+  const float scale_log2 = a.sm_scale * 1.4426950408889634f;
   const int64_t row_elems = static_cast<int64_t>(a.num_kv_heads) * kHeadDim;
   const int64_t seq_base = a.page_size > 0 ? 0 : static_cast<int64_t>(b) * a.seq_stride_tokens * row_elems;
-  const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(a.k) + seq_base + g * kHeadDim + l16 * 8;
+  const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(a.k) + seq_base + g * kHeadDim + 8 * t4;
   const __nv_bfloat16* vbase =
-      HAS_V ? reinterpret_cast<const __nv_bfloat16*>(a.v) + seq_base + g * kHeadDim + l16 * 8 : nullptr;
+      HAS_V ? reinterpret_cast<const __nv_bfloat16*>(a.v) + seq_base + g * kHeadDim + 8 * g8 : nullptr;
 
-  const int n_quads = (cnt + kQuad - 1) / kQuad;
-  const int n_iter = n_quads > warp ? (n_quads - warp + kAttnWarps - 1) / kAttnWarps : 0;
+  const int n_blocks = (cnt + kBlockTokens - 1) / kBlockTokens;
+  const int n_iter = n_blocks > warp ? (n_blocks - warp + kAttnWarps - 1) / kAttnWarps : 0;
 
   const uint32_t smem_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
-  const uint32_t ring_lane = smem_u32 + L::ring + (warp * kStages * L::kSlots * 32 + lane) * 16;
-  float* prob_s = reinterpret_cast<float*>(smem + L::prob) + warp * 64;
+  const uint32_t ring_lane = smem_u32 + L::ring + warp * kStages * L::kStageBytes + lane * 16;
 
+  // Slots of a stage: 0..3 K of token g8 (dims 32j + 8 t4), 4..7 K of token 8 + g8,
+  // 8 + 2u + piece: V of token {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4}[u], dims 64 piece + 8 g8 .. + 8.
   auto issue = [&](int it) {
     if (it < n_iter) {
-      const int t0 = (warp + it * kAttnWarps) * kQuad + half * 2;
-      const int r0 = rows_s[min(t0, cnt - 1)];
-      const int r1 = rows_s[min(t0 + 1, cnt - 1)];
-      const uint32_t dst = ring_lane + (it % kStages) * (L::kSlots * 32 * 16);
-      cp_async16(dst, kbase + r0 * row_elems);
-      cp_async16(dst + 512, kbase + r1 * row_elems);
+      const int tok0 = (warp + it * kAttnWarps) * kBlockTokens;
+      const uint32_t dst = ring_lane + (it % kStages) * L::kStageBytes;
+      const __nv_bfloat16* ka = kbase + rows_s[min(tok0 + g8, cnt - 1)] * row_elems;
+      const __nv_bfloat16* kb = kbase + rows_s[min(tok0 + 8 + g8, cnt - 1)] * row_elems;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        cp_async16(dst + j * 512, ka + 32 * j);
+        cp_async16(dst + (4 + j) * 512, kb + 32 * j);
+      }
       if (HAS_V) {
-        cp_async16(dst + 1024, vbase + r0 * row_elems);
-        cp_async16(dst + 1536, vbase + r1 * row_elems);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int tk = tok0 + 2 * t4 + (u & 1) + 8 * (u >> 1);
+          const __nv_bfloat16* vr = vbase + rows_s[min(tk, cnt - 1)] * row_elems;
+          cp_async16(dst + (8 + 2 * u) * 512, vr);
+          cp_async16(dst + (9 + 2 * u) * 512, vr + 64);
+        }
       }
     }
     cp_async_commit();
@@ -189,172 +191,126 @@ __global__ void __launch_bounds__(kThreads, 3) attn_partial_kernel(const AttnLau
 #pragma unroll
   for (int s = 0; s < kStages - 1; ++s) issue(s);
 
-  // online-softmax state. Owner lanes (one per (token-in-pair, head)) keep m_ref / l_part.
-  u64 acc2[G][4];
+  // O^T accumulators: o[j] is the 16 x 8 tile of dims {64 (j >> 2) + 8 g8 + 2 (j & 3) + (0|1)} x heads;
+  // o[j][0..1] = even dim, heads 2 t4, 2 t4 + 1; o[j][2..3] = odd dim, same heads.
+  float o[8][4];
 #pragma unroll
-  for (int h = 0; h < G; ++h)
+  for (int j = 0; j < 8; ++j)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) acc2[h][i] = 0ULL;
-  float m_ref = -INFINITY, l_part = 0.f;
-  const int own_h = l16 & 7, own_tt = l16 >> 3;
-  const bool own_head_ok = own_h < G;
+    for (int i = 0; i < 4; ++i) o[j][i] = 0.f;
+  float m_ref = -INFINITY, l_part = 0.f;               // for head g8 (identical in the 4 lanes of a group)
+  const bool head_ok = g8 < G;
   const int vis_lo = sg.vs, vis_hi = sg.vs + sg.N;
-  float* logit_row = (a.logits != nullptr && own_head_ok)
-                         ? a.logits + (static_cast<int64_t>(b) * a.num_q_heads + g * G + own_h) * a.n_stride
+  float* logit_row = (a.logits != nullptr && head_ok)
+                         ? a.logits + (static_cast<int64_t>(b) * a.num_q_heads + g * G + g8) * a.n_stride
                          : nullptr;
 
   for (int it = 0; it < n_iter; ++it) {
     cp_async_wait<kStages - 2>();
-    const uint32_t src = ring_lane + (it % kStages) * (L::kSlots * 32 * 16);
-    const uint4 k0 = lds128(src), k1 = lds128(src + 512);
-    uint4 v0, v1;
+    const uint32_t src = ring_lane + (it % kStages) * L::kStageBytes;
+    // ---- S^T = Q K^T for the two 8-token tiles ------------------------------------------------
+    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint4 ka = lds128(src + j * 512), kb = lds128(src + (4 + j) * 512);
+      mma_bf16(sa, qw[j][0], 0u, qw[j][1], 0u, ka.x, ka.y);
+      mma_bf16(sa, qw[j][2], 0u, qw[j][3], 0u, ka.z, ka.w);
+      mma_bf16(sb, qw[j][0], 0u, qw[j][1], 0u, kb.x, kb.y);
+      mma_bf16(sb, qw[j][2], 0u, qw[j][3], 0u, kb.z, kb.w);
+    }
+    uint4 vw[4][2];
     if (HAS_V) {
-      v0 = lds128(src + 1024);
-      v1 = lds128(src + 1536);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        vw[u][0] = lds128(src + (8 + 2 * u) * 512);
+        vw[u][1] = lds128(src + (9 + 2 * u) * 512);
+      }
     }
     issue(it + kStages - 1);
 
-    // ---- partial dot products: 2 tokens x G heads over this lane's 8 dims ---------------------
-    float vals[16];
-    {
-      const uint32_t kw[2][4] = {{k0.x, k0.y, k0.z, k0.w}, {k1.x, k1.y, k1.z, k1.w}};
+    // ---- online softmax for head g8, tokens tok0 + {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4} ------
+    const int tok0 = (warp + it * kAttnWarps) * kBlockTokens;
+    float x[4] = {sa[0] * scale_log2, sa[1] * scale_log2, sb[0] * scale_log2, sb[1] * scale_log2};
 #pragma unroll
-      for (int t = 0; t < 2; ++t) {
-        u64 kp[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) kp[i] = widen2(kw[t][i]);
-#pragma unroll
-        for (int h = 0; h < 8; ++h) {
-          if (h < G) {
-            u64 s2 = fmul2(kp[0], q2[h][0]);
-#pragma unroll
-            for (int i = 1; i < 4; ++i) s2 = ffma2(kp[i], q2[h][i], s2);
-            float lo, hi;
-            unpack2(s2, lo, hi);
-            vals[t * 8 + h] = lo + hi;
-          } else {
-            vals[t * 8 + h] = 0.f;
-          }
-        }
+    for (int i = 0; i < 4; ++i) {
+      const int tok = tok0 + 2 * t4 + (i & 1) + 8 * (i >> 1);
+      const bool valid = head_ok && tok < cnt;
+      x[i] = valid ? x[i] : -INFINITY;
+      if (logit_row != nullptr && valid) {
+        const int pos = start + tok;                   // dense / scoring mode: position == list index
+        if (pos >= vis_lo && pos < vis_hi && pos - vis_lo < a.n_stride) logit_row[pos - vis_lo] = x[i];
       }
     }
-    // ---- reduce-scatter over the 16 lanes of a row: lane l16 ends with value index l16 --------
-    float x;
-    {
-      const bool b3 = l16 & 8, b2 = l16 & 4, b1 = l16 & 2, b0 = l16 & 1;
-      float v8[8], v4[4], v2[2];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float send = b3 ? vals[i] : vals[i + 8];
-        const float keep = b3 ? vals[i + 8] : vals[i];
-        v8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float send = b2 ? v8[i] : v8[i + 4];
-        const float keep = b2 ? v8[i + 4] : v8[i];
-        v4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-      }
-#pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        const float send = b1 ? v4[i] : v4[i + 2];
-        const float keep = b1 ? v4[i + 2] : v4[i];
-        v2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-      }
-      const float send = b0 ? v2[0] : v2[1];
-      const float keep = b0 ? v2[1] : v2[0];
-      x = keep + __shfl_xor_sync(0xffffffffu, send, 1);
-    }
-    // ---- owner lane: online softmax for (token, head) ----------------------------------------
-    const int tok = (warp + it * kAttnWarps) * kQuad + half * 2 + own_tt;   // index inside the chunk
-    const bool valid = own_head_ok && tok < cnt;
-    x = valid ? x : -INFINITY;
-    if (logit_row != nullptr && valid) {
-      const int pos = start + tok;                     // dense / scoring mode: position == list index
-      if (pos >= vis_lo && pos < vis_hi && pos - vis_lo < a.n_stride) logit_row[pos - vis_lo] = x;
-    }
-    float mx = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 8));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-    const bool raise = mx > m_ref + kRescaleSlack;
-    if (__any_sync(0xffffffffu, raise)) {
+    float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+    if (__any_sync(0xffffffffu, mx > m_ref + kRescaleSlack)) {
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const bool raise = mx > m_ref + kRescaleSlack;
       const float alpha = raise ? fast_exp2(m_ref - mx) : 1.f;     // m_ref = -inf gives 0
       if (raise) m_ref = mx;
       l_part *= alpha;
+      if (HAS_V) {
+        const float a0 = __shfl_sync(0xffffffffu, alpha, 8 * t4);       // head 2 t4 lives in group 2 t4
+        const float a1 = __shfl_sync(0xffffffffu, alpha, 8 * t4 + 4);   // head 2 t4 + 1
 #pragma unroll
-      for (int h = 0; h < G; ++h) {
-        const float ah = __shfl_sync(0xffffffffu, alpha, h);
-        const u64 a2 = pack2(ah, ah);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc2[h][i] = fmul2(acc2[h][i], a2);
+        for (int j = 0; j < 8; ++j) {
+          o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1;
+        }
       }
     }
-    const float p = valid ? fast_exp2(x - m_ref) : 0.f;
-    l_part += p;
+    float p[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      p[i] = (x[i] == -INFINITY) ? 0.f : fast_exp2(x[i] - m_ref);
+      l_part += p[i];
+    }
 
     if (HAS_V) {
-      float* slot = prob_s + (it & 1) * 32;
-      slot[lane] = p;
-      __syncwarp();
-      const float4* pv = reinterpret_cast<const float4*>(slot + half * 16);
-      const float4 pa = pv[0], pb = pv[1], pc = pv[2], pd = pv[3];
-      const float pp[2][8] = {{pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w},
-                              {pc.x, pc.y, pc.z, pc.w, pd.x, pd.y, pd.z, pd.w}};
-      const uint32_t vw[2][4] = {{v0.x, v0.y, v0.z, v0.w}, {v1.x, v1.y, v1.z, v1.w}};
+      // B fragments of P (tokens on K, head g8 on N): high bf16 part and remainder
+      const uint32_t ph0 = pack_bf16(p[0], p[1]), ph1 = pack_bf16(p[2], p[3]);
+      const uint32_t pl0 = pack_bf16(p[0] - __uint_as_float(ph0 << 16), p[1] - __uint_as_float(ph0 & 0xffff0000u));
+      const uint32_t pl1 = pack_bf16(p[2] - __uint_as_float(ph1 << 16), p[3] - __uint_as_float(ph1 & 0xffff0000u));
 #pragma unroll
-      for (int t = 0; t < 2; ++t) {
-        u64 vp[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) vp[i] = widen2(vw[t][i]);
-#pragma unroll
-        for (int h = 0; h < G; ++h) {
-          const u64 p2 = pack2(pp[t][h], pp[t][h]);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) acc2[h][i] = ffma2(vp[i], p2, acc2[h][i]);
-        }
+      for (int j = 0; j < 8; ++j) {
+        const int piece = j >> 2, i = j & 3;
+        const uint32_t w0 = (&vw[0][piece].x)[i], w1 = (&vw[1][piece].x)[i];
+        const uint32_t w2 = (&vw[2][piece].x)[i], w3 = (&vw[3][piece].x)[i];
+        // A fragment of V^T: rows = (even dim, odd dim), columns = token pairs
+        const uint32_t a0 = __byte_perm(w0, w1, 0x5410), a1 = __byte_perm(w0, w1, 0x7632);
+        const uint32_t a2 = __byte_perm(w2, w3, 0x5410), a3 = __byte_perm(w2, w3, 0x7632);
+        mma_bf16(o[j], a0, a1, a2, a3, ph0, ph1);
+        mma_bf16(o[j], a0, a1, a2, a3, pl0, pl1);
       }
     }
   }
   cp_async_wait<0>();
 
-  // ---- merge inside the warp -----------------------------------------------------------------
-  l_part += __shfl_xor_sync(0xffffffffu, l_part, 8);
-  l_part += __shfl_xor_sync(0xffffffffu, l_part, 16);
-  float acc[G][8];
-  if (HAS_V) {
-#pragma unroll
-    for (int h = 0; h < G; ++h)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float lo, hi;
-        unpack2(acc2[h][i], lo, hi);
-        lo += __shfl_xor_sync(0xffffffffu, lo, 16);
-        hi += __shfl_xor_sync(0xffffffffu, hi, 16);
-        acc[h][2 * i] = lo;
-        acc[h][2 * i + 1] = hi;
-      }
-  }
+  // ---- merge inside the warp: the sum of probabilities of head g8 ----------------------------
+  l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
+  l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
   __syncthreads();                                     // every warp is done with its ring
 
   // ---- merge across warps (re-using the ring space) and emit the split's partial --------------
   float* m_s = reinterpret_cast<float*>(smem + L::ring);            // [warps][8]
   float* l_s = m_s + kAttnWarps * 8;                                 // [warps][8]
-  float* acc_s = l_s + kAttnWarps * 8;                               // [warps][G][128]
-  if (lane < 8) {
-    m_s[warp * 8 + lane] = (lane < G) ? m_ref : -INFINITY;
-    l_s[warp * 8 + lane] = (lane < G) ? l_part : 0.f;
+  float* acc_s = l_s + kAttnWarps * 8;                               // [warps][8][128]
+  if (t4 == 0) {
+    m_s[warp * 8 + g8] = head_ok ? m_ref : -INFINITY;
+    l_s[warp * 8 + g8] = head_ok ? l_part : 0.f;
   }
-  if (HAS_V && half == 0) {
+  if (HAS_V) {
 #pragma unroll
-    for (int h = 0; h < G; ++h) {
-      float4* dst = reinterpret_cast<float4*>(acc_s + (warp * G + h) * kHeadDim + l16 * 8);
-      dst[0] = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
-      dst[1] = make_float4(acc[h][4], acc[h][5], acc[h][6], acc[h][7]);
+    for (int j = 0; j < 8; ++j) {
+      const int d0 = 64 * (j >> 2) + 8 * g8 + 2 * (j & 3);
+      float* base = acc_s + (warp * 8 + 2 * t4) * kHeadDim + d0;
+      *reinterpret_cast<float2*>(base) = make_float2(o[j][0], o[j][2]);
+      *reinterpret_cast<float2*>(base + kHeadDim) = make_float2(o[j][1], o[j][3]);
     }
   }
   __syncthreads();
   const int64_t item = (static_cast<int64_t>(b) * a.num_kv_heads + g) * a.max_chunks + c;
-  for (int o = tid; o < G * kHeadDim; o += kThreads) {
-    const int h = o / kHeadDim, dd = o % kHeadDim;
+  for (int e = tid; e < G * kHeadDim; e += kThreads) {
+    const int h = e / kHeadDim, dd = e % kHeadDim;
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, m_s[w * 8 + h]);
@@ -364,7 +320,7 @@ __global__ void __launch_bounds__(kThreads, 3) attn_partial_kernel(const AttnLau
       const float mw = m_s[w * 8 + h];
       const float sc = (mw == -INFINITY) ? 0.f : exp2f(mw - M);
       den += l_s[w * 8 + h] * sc;
-      if (HAS_V) num += acc_s[(w * G + h) * kHeadDim + dd] * sc;
+      if (HAS_V) num += acc_s[(w * 8 + h) * kHeadDim + dd] * sc;
     }
     if (HAS_V) a.part_acc[(item * G + h) * kHeadDim + dd] = num;
     if (dd == 0) {

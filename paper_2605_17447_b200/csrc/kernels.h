@@ -8,9 +8,8 @@ namespace fastocr {
 constexpr int kHeadDim = 128;
 constexpr int kMaxGroup = 8;          // query heads per KV head handled by one CTA
 constexpr int kAttnWarps = 4;         // warps per attention CTA
-constexpr int kQuad = 4;              // tokens one warp consumes per pipeline stage
-constexpr int kTokensPerCtaIter = kAttnWarps * kQuad;
-constexpr int kMaxChunk = 4096;       // tokens per split (row table lives in shared memory)
+constexpr int kTokensPerCtaIter = kAttnWarps * 16;   // each warp consumes 16 tokens per pipeline stage
+constexpr int kMaxChunk = 2048;       // tokens per split (row table lives in shared memory)
 constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
 
 struct AttnLaunch {
