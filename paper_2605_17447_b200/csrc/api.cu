@@ -6,7 +6,6 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -25,15 +24,15 @@ struct fastocr_ctx {
   int device = 0;
   int sm_count = 148;
   fastocr_limits lim{};
-  int64_t cap_items = 0;        // (sequence, KV head, split) partial slots
+  int64_t cap_items = 0;        // partial slots: one per (team, sequence) pair and KV head
   float* part_acc = nullptr;    // [cap_items][8][128]
   float* part_ml = nullptr;     // [cap_items][8][2]
+  int32_t* plan = nullptr;      // [2 + kMaxUnits + 1] decomposition written by the attention kernel
   float* logits = nullptr;      // [max_batch][H][max_vis_len]
   float* stats = nullptr;       // [max_batch][H][2]
   float* scores = nullptr;      // [max_batch][max_vis_len] (decode_step scratch)
   unsigned long long* faults = nullptr;
-  int target_items = 0;         // tuning: desired number of CTAs per attention launch
-  int min_chunk = 0;            // tuning: smallest split, tokens
+  int ctas_per_sm = 1;          // persistent attention CTAs per SM
   char err[512] = {0};
   // optional per-launch timing
   std::vector<cudaEvent_t> prof_ev;   // 2 per timed launch
@@ -55,34 +54,6 @@ fastocr_status fail(fastocr_ctx* ctx, fastocr_status code, const char* fmt, ...)
 }
 
 bool group_supported(int G) { return G == 1 || G == 2 || G == 4 || G == 7 || G == 8; }
-
-int env_int(const char* name, int dflt) {
-  const char* v = std::getenv(name);
-  return (v != nullptr && *v != 0) ? std::atoi(v) : dflt;
-}
-
-int round_up(int x, int m) { return (x + m - 1) / m * m; }
-
-// Split planning: how many tokens one CTA streams. Enough CTAs to keep every SM busy with a few
-// resident CTAs and to even out the tail, but no smaller than min_chunk tokens so that the
-// prologue (query load, row table, pipeline fill) is amortised.
-void plan_split(const fastocr_ctx* ctx, int batch, int num_kv_heads, int max_len, int* chunk_tokens,
-                int* max_chunks) {
-  const int64_t units = static_cast<int64_t>(batch) * num_kv_heads;
-  int64_t nch = (ctx->target_items + units - 1) / units;
-  const int min_chunk = units >= 64 ? ctx->min_chunk : 32;
-  const int64_t by_min = max_len / min_chunk > 0 ? max_len / min_chunk : 1;
-  if (nch > by_min) nch = by_min;
-  const int64_t by_cap = ctx->cap_items / units > 0 ? ctx->cap_items / units : 1;
-  if (nch > by_cap) nch = by_cap;
-  if (nch < 1) nch = 1;
-  int chunk = round_up(static_cast<int>((max_len + nch - 1) / nch), fastocr::kTokensPerCtaIter);
-  if (chunk > fastocr::kMaxChunk) chunk = fastocr::kMaxChunk;
-  if (chunk < fastocr::kTokensPerCtaIter) chunk = fastocr::kTokensPerCtaIter;
-  *chunk_tokens = chunk;
-  *max_chunks = (max_len + chunk - 1) / chunk;
-  if (*max_chunks < 1) *max_chunks = 1;
-}
 
 fastocr_status check_view(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, bool need_v) {
   if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
@@ -107,6 +78,11 @@ fastocr_status check_view(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "seq_stride_tokens < max_seq_len");
   }
   if (!(kv->sm_scale > 0.f) || !std::isfinite(kv->sm_scale)) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "sm_scale must be positive");
+  {
+    const int ts = fastocr::team_size_for(kv->num_kv_heads);
+    if (static_cast<int64_t>(kv->batch) * (kv->num_kv_heads / ts) > fastocr::kMaxUnits)
+      return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "batch x KV-head slices exceeds %d", fastocr::kMaxUnits);
+  }
   if (kv->batch > ctx->lim.max_batch || kv->num_q_heads > ctx->lim.num_q_heads ||
       kv->num_kv_heads > ctx->lim.num_kv_heads || kv->max_seq_len > ctx->lim.max_seq_len)
     return fail(ctx, FASTOCR_ERR_WORKSPACE, "view (B=%d H=%d Hkv=%d S<=%d) exceeds the context limits (B=%d H=%d Hkv=%d S<=%d)",
@@ -134,7 +110,11 @@ AttnLaunch make_launch(const fastocr_ctx* ctx, const fastocr_kv_view* kv, const 
   a.part_acc = ctx->part_acc;
   a.part_ml = ctx->part_ml;
   a.fault_counter = ctx->faults;
-  plan_split(ctx, kv->batch, kv->num_kv_heads, max_len, &a.chunk_tokens, &a.max_chunks);
+  a.plan_out = ctx->plan;
+  a.team_size = fastocr::team_size_for(kv->num_kv_heads);
+  a.units_per_seq = kv->num_kv_heads / a.team_size;
+  a.grid_ctas = ctx->sm_count * ctx->ctas_per_sm;
+  (void)max_len;
   return a;
 }
 
@@ -245,13 +225,9 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
     return FASTOCR_ERR_CUDA;
   }
   ctx->sm_count = sm > 0 ? sm : 148;
-  ctx->target_items = env_int("FASTOCR_TARGET_ITEMS", ctx->sm_count * 3 * 8);
-  ctx->min_chunk = env_int("FASTOCR_MIN_CHUNK", 128);
-  if (ctx->min_chunk < fastocr::kTokensPerCtaIter) ctx->min_chunk = fastocr::kTokensPerCtaIter;
-  const int64_t units = static_cast<int64_t>(lim->max_batch) * lim->num_kv_heads;
-  const int64_t min_chunks = (lim->max_seq_len + fastocr::kMaxChunk - 1) / fastocr::kMaxChunk;
-  ctx->cap_items = units * min_chunks;
-  if (ctx->cap_items < 2 * ctx->target_items) ctx->cap_items = 2 * ctx->target_items;
+  // one partial slot per (team, unit) pair that can occur: teams + units, times the team size
+  ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * ctx->ctas_per_sm * fastocr::kAttnWarps +
+                   static_cast<int64_t>(lim->max_batch) * lim->num_kv_heads + 64;
   const int64_t nvis = lim->max_vis_len > 0 ? lim->max_vis_len : 1;
   const size_t bytes_acc = static_cast<size_t>(ctx->cap_items) * fastocr::kMaxGroup * fastocr::kHeadDim * sizeof(float);
   const size_t bytes_ml = static_cast<size_t>(ctx->cap_items) * fastocr::kMaxGroup * 2 * sizeof(float);
@@ -261,6 +237,7 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   if ((e = cudaMalloc(&ctx->part_acc, bytes_acc)) != cudaSuccess || (e = cudaMalloc(&ctx->part_ml, bytes_ml)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->logits, bytes_logits)) != cudaSuccess || (e = cudaMalloc(&ctx->stats, bytes_stats)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->scores, bytes_scores)) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->plan, (2 + fastocr::kMaxUnits + 1) * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->faults, sizeof(unsigned long long))) != cudaSuccess ||
       (e = cudaMemset(ctx->faults, 0, sizeof(unsigned long long))) != cudaSuccess) {
     fastocr_destroy(ctx);
@@ -278,6 +255,7 @@ void fastocr_destroy(fastocr_ctx* ctx) {
   cudaFree(ctx->logits);
   cudaFree(ctx->stats);
   cudaFree(ctx->scores);
+  cudaFree(ctx->plan);
   cudaFree(ctx->faults);
   delete ctx;
 }

@@ -1,14 +1,26 @@
-// Decode attention kernels for sm_100a: one templated split-KV flash-decode core serves dense
+// Decode attention kernels for sm_100a: one templated persistent flash-decode core serves dense
 // attention (Eq. 2, focal case), the keys-only scoring pass, and pruned attention over the kept
 // set K = T u F (Eq. 2, non-focal case), on contiguous or paged caches.
 //
-// Work decomposition: CTA = (split c, KV head g, sequence b). The CTA first builds, in shared
-// memory, the table of physical cache rows of the tokens it attends (this is the only place where
-// dense / pruned / paged differ), then each of its warps streams 16-token blocks of those rows.
+// Work decomposition (stream-K over tokens). All attended tokens of the launch are laid end to end
+// in one index space, sequence after sequence, each sequence padded to a multiple of 16 tokens.
+// That space is cut into equal ranges, one per "team"; a team is one warp per KV head (so the
+// whole 1-2 KB token row is fetched by neighbouring warps at about the same time), and the grid is
+// one persistent CTA of eight autonomous warps per SM. Every warp therefore streams the same
+// number of 16-token blocks, pays one pipeline prologue per launch, and never meets a CTA barrier
+// after set-up. A range may cross sequence boundaries: the warp then writes the partial result
+// (running max, sum, unnormalised output) of the sequence it leaves and starts a new one; a small
+// merge kernel combines the partials of every (sequence, head).
 //
-// Data path: every lane copies, with 16-byte cp.async, exactly the K and V bytes it will later
-// need as tensor-core fragments into its own slots of a shared-memory ring (kStages deep; no
-// cross-thread hand-off, hence no barrier in the main loop) and reads them back with ld.shared.v4.
+// Data path: a block's 16 K rows and 16 V rows (256 bytes each) travel HBM -> shared memory with
+// 16-byte cp.async, one full row per half-warp per instruction (so every request covers whole
+// 128-byte lines), into a per-warp ring (kStages deep; hand-off inside the warp only: one
+// __syncwarp per block). Rows are stored with their 16-byte chunks XOR-swizzled so that the
+// tensor-core fragment reads (ld.shared.v4, each lane its own chunks) are bank-conflict free.
+// Cache rows are located two blocks
+// ahead of the copies by lanes 0-15 (one token each): first the logical position (a load from the
+// index list for selected image tokens), one block later the physical row (a block-table load for
+// paged caches), so neither lookup sits on the critical path.
 //
 // Arithmetic: with a GQA group of 7 or 8 query heads per KV head, q.K^T and P.V are skinny matrix
 // products ([16 tokens x 128] x [128 x 8 heads]); on the fp32 CUDA cores they need more issue slots
@@ -66,153 +78,275 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// number of attended tokens of sequence b and the pieces needed to enumerate them
 struct SeqGeom {
-  int S, vs, N, kept_vis, n_tok;   // n_tok = number of attended tokens
+  int vs, N, kept_vis, n_tok;
 };
-
 __device__ __forceinline__ SeqGeom load_geom(const AttnLaunch& a, int b) {
   SeqGeom s;
-  s.S = a.seq_len[b];
+  const int S = a.seq_len[b];
   s.vs = a.vis_start[b];
   s.N = a.vis_len[b];
   if (a.idx != nullptr) {
-    int kk = a.kcount[b];
+    const int kk = a.kcount[b];
     s.kept_vis = kk < 0 ? 0 : (kk > s.N ? s.N : kk);
   } else {
     s.kept_vis = s.N;
   }
-  s.n_tok = s.S - s.N + s.kept_vis;
+  s.n_tok = max(S - s.N + s.kept_vis, 0);
   return s;
 }
 
-// shared-memory carve-up (bytes). A stage holds, per lane, 8 K slots (+ 8 V slots) of 16 bytes.
+// chunk swizzles of a staged row (16 chunks of 16 bytes): K fragments are read by (token g8,
+// chunk 4j + t4), V fragments by (token pair index t4, chunk g8); see the bank analysis in the reads
+__device__ __forceinline__ int k_swz(int tok) { return (tok & 1) << 2; }
+__device__ __forceinline__ int v_swz(int tok) { return ((tok >> 1) & 3) << 1; }
+
+// shared-memory carve-up (bytes). A stage holds a 16 x 256 B K tile (+ the same for V) per warp.
 template <bool HAS_V>
 struct Smem {
-  static constexpr int kSlots = HAS_V ? 16 : 8;
-  static constexpr int kStageBytes = kSlots * 32 * 16;             // per warp
+  static constexpr int kTileBytes = kBlockTokens * kHeadDim * 2;
+  static constexpr int kStageBytes = (HAS_V ? 2 : 1) * kTileBytes;   // per warp
   static constexpr int kRingBytes = kAttnWarps * kStages * kStageBytes;
-  static constexpr int kMergeBytes = (kAttnWarps * 16 + kAttnWarps * kMaxGroup * kHeadDim) * 4;
   static constexpr int ring = 0;
-  static constexpr int rows = kRingBytes > kMergeBytes ? kRingBytes : kMergeBytes;   // int32 [chunk_tokens]
-  static int total(int chunk_tokens) { return rows + chunk_tokens * 4; }
+  static constexpr int prefix = kRingBytes;                          // int32 [kMaxUnits + 1]
+  static constexpr int total = prefix + (kMaxUnits + 1) * 4;
 };
 
+// Unit u (a sequence, or a sequence x team-sized slice of its KV heads) -> sequence and first KV head.
+__device__ __forceinline__ void unit_to_seq(const AttnLaunch& a, int u, int& b, int& g_base) {
+  if (a.units_per_seq == 1) {
+    b = u;
+    g_base = 0;
+  } else {
+    b = u / a.units_per_seq;
+    g_base = (u - b * a.units_per_seq) * a.team_size;
+  }
+}
+
 template <int G, bool HAS_V>
-__global__ void __launch_bounds__(kThreads, 2) attn_partial_kernel(const AttnLaunch a) {
+__global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaunch a) {
   extern __shared__ __align__(16) unsigned char smem[];
   using L = Smem<HAS_V>;
-  const int c = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g8 = lane >> 2, t4 = lane & 3;             // MMA fragment coordinates: group, thread-in-group
+  const int units = a.batch * a.units_per_seq;
 
-  const SeqGeom sg = load_geom(a, b);
-  const int start = c * a.chunk_tokens;
-  if (start >= sg.n_tok) return;                       // whole CTA leaves together
-  const int cnt = min(a.chunk_tokens, sg.n_tok - start);
-
-  // ---- table of physical rows for the attended tokens [start, start + cnt) -------------------
-  int32_t* rows_s = reinterpret_cast<int32_t*>(smem + L::rows);
-  for (int i = tid; i < cnt; i += kThreads) {
-    const int j = start + i;
-    int pos = j;
-    if (a.idx != nullptr) {                            // kept set: text before | selected image | text after
-      if (j >= sg.vs + sg.kept_vis) {
-        pos = j - sg.kept_vis + sg.N;
-      } else if (j >= sg.vs) {
-        int r = a.idx[static_cast<int64_t>(b) * a.k_stride + (j - sg.vs)];
-        if (r < 0 || r >= sg.N) {                      // never read outside the image span
-          atomicAdd(a.fault_counter, 1ULL);
-          r = r < 0 ? 0 : sg.N - 1;
-        }
-        pos = sg.vs + r;
+  // ---- set-up: padded token prefix over units (warp 0), the only CTA barrier of the kernel -----
+  int* prefix_s = reinterpret_cast<int*>(smem + L::prefix);
+  if (warp == 0) {
+    int carry = 0;
+    for (int u0 = 0; u0 < units; u0 += 32) {
+      const int u = u0 + lane;
+      int n = 0;
+      if (u < units) {
+        int b, gb;
+        unit_to_seq(a, u, b, gb);
+        n = (load_geom(a, b).n_tok + kBlockTokens - 1) & ~(kBlockTokens - 1);
       }
-    }
-    int row = pos;
-    if (a.page_size > 0) {
-      const int page = a.block_table[static_cast<int64_t>(b) * a.max_pages + pos / a.page_size];
-      row = page * a.page_size + pos % a.page_size;
-    }
-    rows_s[i] = row;
-  }
-
-  // ---- A fragments of Q: lane (g8, t4) holds head g8, dims 32j + 8 t4 .. + 8 (j = 0..3) -------
-  uint32_t qw[4][4];
-  {
-    const uint4* qp = reinterpret_cast<const uint4*>(a.q) +
-                      (static_cast<int64_t>(b) * a.num_q_heads + static_cast<int64_t>(g) * G + g8) * (kHeadDim / 8) + t4;
+      int incl = n;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint4 w = make_uint4(0u, 0u, 0u, 0u);
-      if (g8 < G) w = __ldg(qp + 4 * j);
-      qw[j][0] = w.x; qw[j][1] = w.y; qw[j][2] = w.z; qw[j][3] = w.w;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      if (u < units) prefix_s[u] = carry + incl - n;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
     }
+    if (lane == 0) prefix_s[units] = carry;
   }
   __syncthreads();
+  const int total_tok = prefix_s[units];
+  const int teams = (gridDim.x * kAttnWarps) / a.team_size;
+  const int per_team = (((total_tok + teams - 1) / teams) + kBlockTokens - 1) & ~(kBlockTokens - 1);
+  if (blockIdx.x == 0 && a.plan_out != nullptr) {      // the merge kernel re-uses the plan
+    for (int i = tid; i <= units; i += kThreads) a.plan_out[2 + i] = prefix_s[i];
+    if (tid == 0) {
+      a.plan_out[0] = per_team;
+      a.plan_out[1] = teams;
+    }
+  }
+  const int wglobal = blockIdx.x * kAttnWarps + warp;
+  const int team = wglobal / a.team_size, team_lane = wglobal - team * a.team_size;
+  const int r0 = team * per_team;
+  const int r1 = min(total_tok, r0 + per_team);
+  if (per_team == 0 || r0 >= r1) return;               // nothing for this warp (no barrier follows)
+  const int n_blocks = (r1 - r0) / kBlockTokens;
 
   const float scale_log2 = a.sm_scale * 1.4426950408889634f;
   const int64_t row_elems = static_cast<int64_t>(a.num_kv_heads) * kHeadDim;
-  const int64_t seq_base = a.page_size > 0 ? 0 : static_cast<int64_t>(b) * a.seq_stride_tokens * row_elems;
-  const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(a.k) + seq_base + g * kHeadDim + 8 * t4;
-  const __nv_bfloat16* vbase =
-      HAS_V ? reinterpret_cast<const __nv_bfloat16*>(a.v) + seq_base + g * kHeadDim + 8 * g8 : nullptr;
-
-  const int n_blocks = (cnt + kBlockTokens - 1) / kBlockTokens;
-  const int n_iter = n_blocks > warp ? (n_blocks - warp + kAttnWarps - 1) / kAttnWarps : 0;
-
+  const int64_t seq_elems = a.page_size > 0 ? 0 : a.seq_stride_tokens * row_elems;
+  const int c16 = lane & 15, half = lane >> 4;          // copy role: chunk of a row, which row of a pair
+  const __nv_bfloat16* kptr = reinterpret_cast<const __nv_bfloat16*>(a.k) + 8 * c16;
+  const __nv_bfloat16* vptr = HAS_V ? reinterpret_cast<const __nv_bfloat16*>(a.v) + 8 * c16 : nullptr;
   const uint32_t smem_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
-  const uint32_t ring_lane = smem_u32 + L::ring + warp * kStages * L::kStageBytes + lane * 16;
+  const uint32_t ring_warp = smem_u32 + L::ring + warp * kStages * L::kStageBytes;
 
-  // Slots of a stage: 0..3 K of token g8 (dims 32j + 8 t4), 4..7 K of token 8 + g8,
-  // 8 + 2u + piece: V of token {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4}[u], dims 64 piece + 8 g8 .. + 8.
-  auto issue = [&](int it) {
-    if (it < n_iter) {
-      const int tok0 = (warp + it * kAttnWarps) * kBlockTokens;
-      const uint32_t dst = ring_lane + (it % kStages) * L::kStageBytes;
-      const __nv_bfloat16* ka = kbase + rows_s[min(tok0 + g8, cnt - 1)] * row_elems;
-      const __nv_bfloat16* kb = kbase + rows_s[min(tok0 + 8 + g8, cnt - 1)] * row_elems;
+  // ---- block descriptors: a cursor walks the range; a 5-deep register FIFO feeds the stages ----
+  // stage P (block n+4): logical position of token `lane` (< 16) of the block
+  // stage R (block n+3): physical row of that token
+  // stage I (block n+2): cp.async of the block's K/V fragments
+  // stage C (block n):   MMAs, softmax, partial flush
+  int cur_u = 0, cur_end = 0;                          // cursor: unit containing the next offset
+  {
+    int lo = 0, hi = units;                            // largest u with prefix[u] <= r0
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (prefix_s[mid] <= r0) lo = mid; else hi = mid;
+    }
+    cur_u = lo;
+    while (prefix_s[cur_u + 1] <= r0) ++cur_u;         // skip empty units
+    cur_end = prefix_s[cur_u + 1];
+  }
+  int cur_b, cur_gb;
+  unit_to_seq(a, cur_u, cur_b, cur_gb);
+  SeqGeom cur_geom = load_geom(a, cur_b);
+
+  int fu[5], fj[5], fb[5];                             // unit, first token within unit, sequence
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        cp_async16(dst + j * 512, ka + 32 * j);
-        cp_async16(dst + (4 + j) * 512, kb + 32 * j);
+  for (int i = 0; i < 5; ++i) { fu[i] = -1; fj[i] = 0; fb[i] = 0; }
+  int pos_p = 0, row_p = 0;                            // lanes 0..15: position (block n+4 -> n+3), row (n+3 -> n+2)
+
+  // describe block n (if it exists) into FIFO slot `slot` and start its position lookup
+  auto stage_pos = [&](int n, int& du, int& dj, int& db) -> int {
+    if (n >= n_blocks) { du = -1; return 0; }
+    const int off = r0 + n * kBlockTokens;
+    while (off >= cur_end) {
+      ++cur_u;
+      cur_end = prefix_s[cur_u + 1];
+      if (off < cur_end) {
+        unit_to_seq(a, cur_u, cur_b, cur_gb);
+        cur_geom = load_geom(a, cur_b);
       }
-      if (HAS_V) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int tk = tok0 + 2 * t4 + (u & 1) + 8 * (u >> 1);
-          const __nv_bfloat16* vr = vbase + rows_s[min(tk, cnt - 1)] * row_elems;
-          cp_async16(dst + (8 + 2 * u) * 512, vr);
-          cp_async16(dst + (9 + 2 * u) * 512, vr + 64);
+    }
+    du = cur_u;
+    dj = off - prefix_s[cur_u];
+    db = cur_b;
+    int pos = 0;
+    if (lane < kBlockTokens) {
+      const int j = min(dj + lane, cur_geom.n_tok - 1);
+      pos = j;
+      if (a.idx != nullptr) {                          // kept set: text before | selected image | text after
+        if (j >= cur_geom.vs + cur_geom.kept_vis) {
+          pos = j - cur_geom.kept_vis + cur_geom.N;
+        } else if (j >= cur_geom.vs) {
+          int r = __ldg(a.idx + static_cast<int64_t>(cur_b) * a.k_stride + (j - cur_geom.vs));
+          if (r < 0 || r >= cur_geom.N) {              // never read outside the image span
+            atomicAdd(a.fault_counter, 1ULL);
+            r = r < 0 ? 0 : cur_geom.N - 1;
+          }
+          pos = cur_geom.vs + r;
         }
+      }
+    }
+    return pos;
+  };
+  auto stage_row = [&](int du, int db, int pos) -> int {
+    if (du < 0 || a.page_size == 0 || lane >= kBlockTokens) return pos;
+    const int page = __ldg(a.block_table + static_cast<int64_t>(db) * a.max_pages + pos / a.page_size);
+    return page * a.page_size + pos % a.page_size;
+  };
+  auto stage_issue = [&](int n, int du, int db, int row) {
+    if (du >= 0) {
+      int b_unused, gb;
+      unit_to_seq(a, du, b_unused, gb);
+      const int64_t base = db * seq_elems + static_cast<int64_t>(gb + team_lane) * kHeadDim;
+      const uint32_t dst = ring_warp + (n % kStages) * L::kStageBytes;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {                    // rows 2i (lanes 0-15) and 2i + 1 (lanes 16-31)
+        const int tok = 2 * i + half;
+        const int64_t roff = base + __shfl_sync(0xffffffffu, row, tok) * row_elems;
+        cp_async16(dst + tok * 256 + ((c16 ^ k_swz(tok)) << 4), kptr + roff);
+        if (HAS_V) cp_async16(dst + L::kTileBytes + tok * 256 + ((c16 ^ v_swz(tok)) << 4), vptr + roff);
       }
     }
     cp_async_commit();
   };
 
-#pragma unroll
-  for (int s = 0; s < kStages - 1; ++s) issue(s);
+  // ---- prologue: positions of blocks 0..3, rows of 0..2, copies of 0..1 -------------------------
+  int pos0 = stage_pos(0, fu[0], fj[0], fb[0]);
+  int pos1 = stage_pos(1, fu[1], fj[1], fb[1]);
+  int pos2 = stage_pos(2, fu[2], fj[2], fb[2]);
+  pos_p = stage_pos(3, fu[3], fj[3], fb[3]);
+  {
+    const int row0 = stage_row(fu[0], fb[0], pos0);
+    const int row1 = stage_row(fu[1], fb[1], pos1);
+    row_p = stage_row(fu[2], fb[2], pos2);
+    stage_issue(0, fu[0], fb[0], row0);
+    stage_issue(1, fu[1], fb[1], row1);
+  }
 
-  // O^T accumulators: o[j] is the 16 x 8 tile of dims {64 (j >> 2) + 8 g8 + 2 (j & 3) + (0|1)} x heads;
-  // o[j][0..1] = even dim, heads 2 t4, 2 t4 + 1; o[j][2..3] = odd dim, same heads.
-  float o[8][4];
-#pragma unroll
-  for (int j = 0; j < 8; ++j)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) o[j][i] = 0.f;
-  float m_ref = -INFINITY, l_part = 0.f;               // for head g8 (identical in the 4 lanes of a group)
+  // ---- per-unit state ----------------------------------------------------------------------------
+  uint32_t qw[4][4];                                   // A fragments of Q: head g8, dims 32j + 8 t4 .. + 8
+  float o[8][4];                                       // O^T tiles: dims {64 (j>>2) + 8 g8 + 2 (j&3) + (0|1)} x heads {2 t4, 2 t4 + 1}
+  float m_ref = -INFINITY, l_part = 0.f;               // head g8 (identical in the 4 lanes of a group)
   const bool head_ok = g8 < G;
-  const int vis_lo = sg.vs, vis_hi = sg.vs + sg.N;
-  float* logit_row = (a.logits != nullptr && head_ok)
-                         ? a.logits + (static_cast<int64_t>(b) * a.num_q_heads + g * G + g8) * a.n_stride
-                         : nullptr;
+  int act_u = -1, act_g = 0, act_ntok = 0, act_vs = 0, act_N = 0;
+  float* logit_row = nullptr;
 
-  for (int it = 0; it < n_iter; ++it) {
-    cp_async_wait<kStages - 2>();
-    const uint32_t src = ring_lane + (it % kStages) * L::kStageBytes;
-    // ---- S^T = Q K^T for the two 8-token tiles ------------------------------------------------
-    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+  auto begin_unit = [&](int u, int b) {
+    int b2, gb;
+    unit_to_seq(a, u, b2, gb);
+    act_u = u;
+    act_g = gb + team_lane;
+    const SeqGeom sg = load_geom(a, b);
+    act_ntok = sg.n_tok; act_vs = sg.vs; act_N = sg.N;
+    const uint4* qp = reinterpret_cast<const uint4*>(a.q) +
+                      (static_cast<int64_t>(b) * a.num_q_heads + static_cast<int64_t>(act_g) * G + g8) * (kHeadDim / 8) + t4;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const uint4 ka = lds128(src + j * 512), kb = lds128(src + (4 + j) * 512);
+      uint4 w = make_uint4(0u, 0u, 0u, 0u);
+      if (head_ok) w = __ldg(qp + 4 * j);
+      qw[j][0] = w.x; qw[j][1] = w.y; qw[j][2] = w.z; qw[j][3] = w.w;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) o[j][i] = 0.f;
+    m_ref = -INFINITY;
+    l_part = 0.f;
+    logit_row = (a.logits != nullptr && head_ok)
+                    ? a.logits + (static_cast<int64_t>(b) * a.num_q_heads + act_g * G + g8) * a.n_stride
+                    : nullptr;
+  };
+  // partial of (team, unit) for this warp's KV head: slot (team + unit) * team_size + team_lane
+  auto end_unit = [&]() {
+    float l = l_part;
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    const int64_t slot = (static_cast<int64_t>(team) + act_u) * a.team_size + team_lane;
+    if (t4 == 0 && head_ok) {
+      a.part_ml[(slot * kMaxGroup + g8) * 2 + 0] = m_ref;
+      a.part_ml[(slot * kMaxGroup + g8) * 2 + 1] = l;
+    }
+    if (HAS_V) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int d0 = 64 * (j >> 2) + 8 * g8 + 2 * (j & 3);
+        float* base = a.part_acc + (slot * kMaxGroup + 2 * t4) * kHeadDim + d0;
+        if (2 * t4 < G) *reinterpret_cast<float2*>(base) = make_float2(o[j][0], o[j][2]);
+        if (2 * t4 + 1 < G) *reinterpret_cast<float2*>(base + kHeadDim) = make_float2(o[j][1], o[j][3]);
+      }
+    }
+  };
+
+  for (int n = 0; n < n_blocks; ++n) {
+    if (fu[0] != act_u) {                              // the range enters a new sequence
+      if (act_u >= 0) end_unit();
+      begin_unit(fu[0], fb[0]);
+    }
+    cp_async_wait<kStages - 2>();
+    __syncwarp();                                      // every lane's copies of this block have landed
+    const uint32_t src = ring_warp + (n % kStages) * L::kStageBytes;
+    // ---- S^T = Q K^T for the two 8-token tiles ------------------------------------------------
+    // lane (g8, t4) reads chunk 4j + t4 of rows g8 and 8 + g8: per 8-lane phase two rows whose
+    // swizzles differ in bit 2, i.e. eight distinct 16-byte bank groups
+    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+    const uint32_t krow = src + g8 * 256;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t coff = ((4 * j + t4) ^ k_swz(g8)) << 4;        // k_swz(8 + g8) == k_swz(g8)
+      const uint4 ka = lds128(krow + coff), kb = lds128(krow + 8 * 256 + coff);
       mma_bf16(sa, qw[j][0], 0u, qw[j][1], 0u, ka.x, ka.y);
       mma_bf16(sa, qw[j][2], 0u, qw[j][3], 0u, ka.z, ka.w);
       mma_bf16(sb, qw[j][0], 0u, qw[j][1], 0u, kb.x, kb.y);
@@ -221,24 +355,29 @@ __global__ void __launch_bounds__(kThreads, 2) attn_partial_kernel(const AttnLau
     uint4 vw[4][2];
     if (HAS_V) {
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        vw[u][0] = lds128(src + (8 + 2 * u) * 512);
-        vw[u][1] = lds128(src + (9 + 2 * u) * 512);
+      for (int u = 0; u < 4; ++u) {                    // rows {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4}, chunks g8 and 8 + g8
+        const int tk = 2 * t4 + (u & 1) + 8 * (u >> 1);
+        const uint32_t vrow = src + L::kTileBytes + tk * 256;
+        vw[u][0] = lds128(vrow + ((g8 ^ v_swz(tk)) << 4));
+        vw[u][1] = lds128(vrow + (((8 + g8) ^ v_swz(tk)) << 4));
       }
     }
-    issue(it + kStages - 1);
+    // ---- keep the look-ahead stages moving ----------------------------------------------------
+    stage_issue(n + 2, fu[2], fb[2], row_p);
+    row_p = stage_row(fu[3], fb[3], pos_p);
+    pos_p = stage_pos(n + 4, fu[4], fj[4], fb[4]);
 
-    // ---- online softmax for head g8, tokens tok0 + {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4} ------
-    const int tok0 = (warp + it * kAttnWarps) * kBlockTokens;
+    // ---- online softmax for head g8, tokens j0 + {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4} ---------
+    const int j0 = fj[0];
     float x[4] = {sa[0] * scale_log2, sa[1] * scale_log2, sb[0] * scale_log2, sb[1] * scale_log2};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const int tok = tok0 + 2 * t4 + (i & 1) + 8 * (i >> 1);
-      const bool valid = head_ok && tok < cnt;
+      const int tok = j0 + 2 * t4 + (i & 1) + 8 * (i >> 1);         // index in the sequence's attended list
+      const bool valid = head_ok && tok < act_ntok;
       x[i] = valid ? x[i] : -INFINITY;
-      if (logit_row != nullptr && valid) {
-        const int pos = start + tok;                   // dense / scoring mode: position == list index
-        if (pos >= vis_lo && pos < vis_hi && pos - vis_lo < a.n_stride) logit_row[pos - vis_lo] = x[i];
+      if (logit_row != nullptr && valid) {             // dense / scoring mode: position == list index
+        const int rel = tok - act_vs;
+        if (rel >= 0 && rel < act_N && rel < a.n_stride) logit_row[rel] = x[i];
       }
     }
     float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
@@ -282,77 +421,43 @@ __global__ void __launch_bounds__(kThreads, 2) attn_partial_kernel(const AttnLau
         mma_bf16(o[j], a0, a1, a2, a3, pl0, pl1);
       }
     }
+    // ---- advance the descriptor FIFO ----------------------------------------------------------
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { fu[i] = fu[i + 1]; fj[i] = fj[i + 1]; fb[i] = fb[i + 1]; }
   }
   cp_async_wait<0>();
-
-  // ---- merge inside the warp: the sum of probabilities of head g8 ----------------------------
-  l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
-  l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
-  __syncthreads();                                     // every warp is done with its ring
-
-  // ---- merge across warps (re-using the ring space) and emit the split's partial --------------
-  float* m_s = reinterpret_cast<float*>(smem + L::ring);            // [warps][8]
-  float* l_s = m_s + kAttnWarps * 8;                                 // [warps][8]
-  float* acc_s = l_s + kAttnWarps * 8;                               // [warps][8][128]
-  if (t4 == 0) {
-    m_s[warp * 8 + g8] = head_ok ? m_ref : -INFINITY;
-    l_s[warp * 8 + g8] = head_ok ? l_part : 0.f;
-  }
-  if (HAS_V) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int d0 = 64 * (j >> 2) + 8 * g8 + 2 * (j & 3);
-      float* base = acc_s + (warp * 8 + 2 * t4) * kHeadDim + d0;
-      *reinterpret_cast<float2*>(base) = make_float2(o[j][0], o[j][2]);
-      *reinterpret_cast<float2*>(base + kHeadDim) = make_float2(o[j][1], o[j][3]);
-    }
-  }
-  __syncthreads();
-  const int64_t item = (static_cast<int64_t>(b) * a.num_kv_heads + g) * a.max_chunks + c;
-  for (int e = tid; e < G * kHeadDim; e += kThreads) {
-    const int h = e / kHeadDim, dd = e % kHeadDim;
-    float M = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, m_s[w * 8 + h]);
-    float num = 0.f, den = 0.f;
-#pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) {
-      const float mw = m_s[w * 8 + h];
-      const float sc = (mw == -INFINITY) ? 0.f : exp2f(mw - M);
-      den += l_s[w * 8 + h] * sc;
-      if (HAS_V) num += acc_s[(w * 8 + h) * kHeadDim + dd] * sc;
-    }
-    if (HAS_V) a.part_acc[(item * G + h) * kHeadDim + dd] = num;
-    if (dd == 0) {
-      a.part_ml[(item * G + h) * 2 + 0] = M;
-      a.part_ml[(item * G + h) * 2 + 1] = den;
-    }
-  }
+  if (act_u >= 0) end_unit();
 }
 
-// One CTA per (sequence, query head): merge the splits.
+// One CTA per (sequence, query head): merge the partials of the teams whose ranges touch it.
 __global__ void __launch_bounds__(kHeadDim) attn_combine_kernel(const AttnLaunch a, void* out, int out_is_fp32,
                                                                 float* stats) {
   const int h = blockIdx.x, b = blockIdx.y, dd = threadIdx.x;
   const int G = a.num_q_heads / a.num_kv_heads;
-  const int g = h / G, hh = h % G;
-  const SeqGeom sg = load_geom(a, b);
-  const int n_chunks = sg.n_tok > 0 ? (sg.n_tok + a.chunk_tokens - 1) / a.chunk_tokens : 0;
-  const int64_t item0 = (static_cast<int64_t>(b) * a.num_kv_heads + g) * a.max_chunks;
-  float M = -INFINITY;
-  for (int c = 0; c < n_chunks; ++c) M = fmaxf(M, a.part_ml[((item0 + c) * G + hh) * 2]);
-  float num = 0.f, den = 0.f;
-  for (int c = 0; c < n_chunks; ++c) {
-    const float mc = a.part_ml[((item0 + c) * G + hh) * 2];
-    const float sc = (mc == -INFINITY) ? 0.f : exp2f(mc - M);
-    den += a.part_ml[((item0 + c) * G + hh) * 2 + 1] * sc;
-    if (out != nullptr) num += a.part_acc[((item0 + c) * G + hh) * kHeadDim + dd] * sc;
+  const int g = h / G, hh = h - g * G;
+  const int u = b * a.units_per_seq + g / a.team_size, team_lane = g % a.team_size;
+  const int per_team = a.plan_out[0];
+  const int begin = a.plan_out[2 + u], end = a.plan_out[3 + u];
+  float M = -INFINITY, num = 0.f, den = 0.f;
+  if (end > begin && per_team > 0) {
+    const int t_lo = begin / per_team, t_hi = (end - 1) / per_team;
+    for (int t = t_lo; t <= t_hi; ++t) {
+      const int64_t slot = (static_cast<int64_t>(t) + u) * a.team_size + team_lane;
+      const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (slot * kMaxGroup + hh) * 2);
+      const float acc = out != nullptr ? a.part_acc[(slot * kMaxGroup + hh) * kHeadDim + dd] : 0.f;
+      if (ml.x == -INFINITY) continue;
+      const float Mn = fmaxf(M, ml.x);
+      const float s_old = (M == -INFINITY) ? 0.f : exp2f(M - Mn), s_new = exp2f(ml.x - Mn);
+      num = num * s_old + acc * s_new;
+      den = den * s_old + ml.y * s_new;
+      M = Mn;
+    }
   }
   if (out != nullptr) {
-    const float o = den > 0.f ? num / den : 0.f;
+    const float r = den > 0.f ? num / den : 0.f;
     const int64_t oi = (static_cast<int64_t>(b) * a.num_q_heads + h) * kHeadDim + dd;
-    if (out_is_fp32) reinterpret_cast<float*>(out)[oi] = o;
-    else reinterpret_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(o);
+    if (out_is_fp32) reinterpret_cast<float*>(out)[oi] = r;
+    else reinterpret_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(r);
   }
   if (stats != nullptr && dd == 0) {
     stats[(static_cast<int64_t>(b) * a.num_q_heads + h) * 2 + 0] = M;
@@ -401,17 +506,15 @@ __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restric
 
 template <int G, bool HAS_V>
 cudaError_t launch_partial_t(const AttnLaunch& a, cudaStream_t s) {
-  const int smem = Smem<HAS_V>::total(a.chunk_tokens);
-  dim3 grid(a.max_chunks, a.num_kv_heads, a.batch);
-  attn_partial_kernel<G, HAS_V><<<grid, kThreads, smem, s>>>(a);
+  attn_stream_kernel<G, HAS_V><<<a.grid_ctas, kThreads, Smem<HAS_V>::total, s>>>(a);
   count_launches(1);
   return cudaGetLastError();
 }
 
 template <int G, bool HAS_V>
 cudaError_t configure_t() {
-  return cudaFuncSetAttribute(attn_partial_kernel<G, HAS_V>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Smem<HAS_V>::total(kMaxChunk));
+  return cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Smem<HAS_V>::total);
 }
 
 }  // namespace
@@ -434,6 +537,11 @@ cudaError_t launch_attn_partial(const AttnLaunch& a, cudaStream_t s) {
 
 cudaError_t configure_kernels() {
   cudaError_t e;
+  // keep the SMs' shared-memory carve-out where the attention kernel needs it, so that the small
+  // kernels in between do not trigger a reconfiguration
+  if ((e = cudaFuncSetAttribute(attn_combine_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(scores_finalize_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(image_mass_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
 #define X(g)                                                \
   if ((e = configure_t<g, true>()) != cudaSuccess) return e; \
   if ((e = configure_t<g, false>()) != cudaSuccess) return e;

@@ -7,10 +7,14 @@ namespace fastocr {
 
 constexpr int kHeadDim = 128;
 constexpr int kMaxGroup = 8;          // query heads per KV head handled by one CTA
-constexpr int kAttnWarps = 4;         // warps per attention CTA
-constexpr int kTokensPerCtaIter = kAttnWarps * 16;   // each warp consumes 16 tokens per pipeline stage
-constexpr int kMaxChunk = 2048;       // tokens per split (row table lives in shared memory)
+constexpr int kAttnWarps = 8;         // autonomous warps per persistent attention CTA
+constexpr int kMaxUnits = 2048;       // sequences x KV-head slices per launch (prefix lives in shared memory)
 constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
+
+// Warps per team: one per KV head when that divides the CTA's warp count, else one.
+inline int team_size_for(int num_kv_heads) {
+  return (num_kv_heads == 1 || num_kv_heads == 2 || num_kv_heads == 4 || num_kv_heads == 8) ? num_kv_heads : 1;
+}
 
 struct AttnLaunch {
   // cache view
@@ -30,12 +34,15 @@ struct AttnLaunch {
   const int32_t* idx;
   const int32_t* kcount;
   int32_t k_stride;
-  // split geometry
-  int32_t chunk_tokens;       // multiple of kTokensPerCtaIter, <= kMaxChunk
-  int32_t max_chunks;         // grid.x
+  // decomposition: a team is team_size warps (one per KV head of a unit); a unit is one sequence x
+  // team_size consecutive KV heads; units_per_seq = num_kv_heads / team_size
+  int32_t team_size;
+  int32_t units_per_seq;
+  int32_t grid_ctas;          // persistent CTAs (kAttnWarps warps each)
   // workspace
-  float* part_acc;            // [B][Hkv][max_chunks][G][128]
-  float* part_ml;             // [B][Hkv][max_chunks][G][2]  (max, sum) in the log2 domain
+  float* part_acc;            // [slots][8][128], slot = (team + unit) * team_size + lane-in-team
+  float* part_ml;             // [slots][8][2]  (max, sum) in the log2 domain
+  int32_t* plan_out;          // [2 + units + 1]: tokens per team, teams, padded token prefix per unit
   float* logits;              // nullptr or [B][H][n_stride], log2-domain logits of image tokens
   int32_t n_stride;
   unsigned long long* fault_counter;
