@@ -358,7 +358,7 @@ def main():
 
     # per-kernel average durations over the same steps (events around every launch)
     prof_steps = min(args.steps, 50)
-    w.ctx.profile_begin(prof_steps * (w.L * 4 + 8))
+    w.ctx.profile_begin(prof_steps * (w.L * 2 + 8))
     for t in range(prof_steps):
         fastocr_step(t)
     prof = w.ctx.profile_end()
@@ -382,7 +382,7 @@ def main():
             kern[name] = {"us_per_launch": us, "launches_per_step": n / prof_steps, "algorithmic_bytes": bytes_per,
                           "gbs": bytes_per / us / 1e3, "frac_of_measured": bytes_per / us / 1e3 / peak,
                           "frac_of_8tbs": bytes_per / us / 1e3 / NOMINAL_HBM_GBS}
-    for name in ("combine", "scores_finalize", "select_topk"):
+    for name in ("scores_finalize", "select_topk"):
         tot, n = prof[name]
         if n:
             kern[name] = {"us_per_launch": tot / n * 1e3, "launches_per_step": n / prof_steps}

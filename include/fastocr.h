@@ -193,11 +193,10 @@ enum {
   FASTOCR_PROF_ATTN_DENSE = 0,  /* split-KV attention kernel, full cache, K and V          */
   FASTOCR_PROF_ATTN_KEYS = 1,   /* same kernel, keys only (stand-alone scoring)             */
   FASTOCR_PROF_ATTN_SPARSE = 2, /* same kernel over the kept set                            */
-  FASTOCR_PROF_COMBINE = 3,     /* split merge                                              */
-  FASTOCR_PROF_FINALIZE = 4,    /* logits -> head-averaged scores                           */
-  FASTOCR_PROF_TOPK = 5,        /* selection                                                */
-  FASTOCR_PROF_MASS = 6,        /* image-mass reduction                                     */
-  FASTOCR_PROF_CLASSES = 7
+  FASTOCR_PROF_FINALIZE = 3,    /* logits -> head-averaged scores                           */
+  FASTOCR_PROF_TOPK = 4,        /* selection                                                */
+  FASTOCR_PROF_MASS = 5,        /* image-mass reduction                                     */
+  FASTOCR_PROF_CLASSES = 6
 };
 fastocr_status fastocr_profile_begin(fastocr_ctx* ctx, int32_t max_launches);
 fastocr_status fastocr_profile_end(fastocr_ctx* ctx, double* ms_per_class, int64_t* launches_per_class);

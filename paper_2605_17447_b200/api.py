@@ -18,7 +18,7 @@ from . import _lib
 _STATUS = {1: "invalid argument", 2: "unsupported", 3: "workspace limits exceeded", 4: "CUDA error"}
 
 
-PROF_CLASSES = ("attn_dense", "attn_keys", "attn_sparse", "combine", "scores_finalize", "select_topk", "image_mass")
+PROF_CLASSES = ("attn_dense", "attn_keys", "attn_sparse", "scores_finalize", "select_topk", "image_mass")
 
 
 class FastOCRError(RuntimeError):

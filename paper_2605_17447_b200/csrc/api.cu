@@ -27,7 +27,7 @@ struct fastocr_ctx {
   int64_t cap_items = 0;        // partial slots: one per (team, sequence) pair and KV head
   float* part_acc = nullptr;    // [cap_items][8][128]
   float* part_ml = nullptr;     // [cap_items][8][2]
-  int32_t* plan = nullptr;      // [2 + kMaxUnits + 1] decomposition written by the attention kernel
+  int32_t* counters = nullptr;  // [kMaxUnits * 8] arrival counters of the split merge (zero between launches)
   float* logits = nullptr;      // [max_batch][H][max_vis_len]
   float* stats = nullptr;       // [max_batch][H][2]
   float* scores = nullptr;      // [max_batch][max_vis_len] (decode_step scratch)
@@ -110,7 +110,7 @@ AttnLaunch make_launch(const fastocr_ctx* ctx, const fastocr_kv_view* kv, const 
   a.part_acc = ctx->part_acc;
   a.part_ml = ctx->part_ml;
   a.fault_counter = ctx->faults;
-  a.plan_out = ctx->plan;
+  a.counters = ctx->counters;
   a.team_size = fastocr::team_size_for(kv->num_kv_heads);
   a.units_per_seq = kv->num_kv_heads / a.team_size;
   a.grid_ctas = ctx->sm_count * ctx->ctas_per_sm;
@@ -157,13 +157,12 @@ fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
     a.logits = ctx->logits;
     a.n_stride = ctx->lim.max_vis_len;
   }
+  a.out = out;
+  a.out_is_fp32 = out_is_fp32;
+  a.stats = want_scores ? ctx->stats : nullptr;
   {
     ProfScope p(ctx, out != nullptr ? FASTOCR_PROF_ATTN_DENSE : FASTOCR_PROF_ATTN_KEYS, s);
     FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
-  }
-  {
-    ProfScope p(ctx, FASTOCR_PROF_COMBINE, s);
-    FASTOCR_TRY_CUDA(fastocr::launch_attn_combine(a, out, out_is_fp32, want_scores ? ctx->stats : nullptr, s), "combine launch");
   }
   if (want_scores) {
     ProfScope p(ctx, FASTOCR_PROF_FINALIZE, s);
@@ -182,13 +181,11 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
   a.idx = idx;
   a.kcount = k;
   a.k_stride = k_stride;
+  a.out = out;
+  a.out_is_fp32 = out_is_fp32;
   {
     ProfScope p(ctx, FASTOCR_PROF_ATTN_SPARSE, s);
     FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
-  }
-  {
-    ProfScope p(ctx, FASTOCR_PROF_COMBINE, s);
-    FASTOCR_TRY_CUDA(fastocr::launch_attn_combine(a, out, out_is_fp32, nullptr, s), "combine launch");
   }
   return FASTOCR_OK;
 }
@@ -237,7 +234,8 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   if ((e = cudaMalloc(&ctx->part_acc, bytes_acc)) != cudaSuccess || (e = cudaMalloc(&ctx->part_ml, bytes_ml)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->logits, bytes_logits)) != cudaSuccess || (e = cudaMalloc(&ctx->stats, bytes_stats)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->scores, bytes_scores)) != cudaSuccess ||
-      (e = cudaMalloc(&ctx->plan, (2 + fastocr::kMaxUnits + 1) * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->counters, fastocr::kMaxUnits * 8 * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMemset(ctx->counters, 0, fastocr::kMaxUnits * 8 * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->faults, sizeof(unsigned long long))) != cudaSuccess ||
       (e = cudaMemset(ctx->faults, 0, sizeof(unsigned long long))) != cudaSuccess) {
     fastocr_destroy(ctx);
@@ -255,7 +253,7 @@ void fastocr_destroy(fastocr_ctx* ctx) {
   cudaFree(ctx->logits);
   cudaFree(ctx->stats);
   cudaFree(ctx->scores);
-  cudaFree(ctx->plan);
+  cudaFree(ctx->counters);
   cudaFree(ctx->faults);
   delete ctx;
 }

@@ -8,9 +8,10 @@
 // whole 1-2 KB token row is fetched by neighbouring warps at about the same time), and the grid is
 // one persistent CTA of eight autonomous warps per SM. Every warp therefore streams the same
 // number of 16-token blocks, pays one pipeline prologue per launch, and never meets a CTA barrier
-// after set-up. A range may cross sequence boundaries: the warp then writes the partial result
-// (running max, sum, unnormalised output) of the sequence it leaves and starts a new one; a small
-// merge kernel combines the partials of every (sequence, head).
+// after set-up. A range may cross sequence boundaries: the warp then finishes the sequence it leaves
+// and starts a new one. A sequence covered by one team is normalised and written by that team;
+// one shared by several teams is merged by whichever of them arrives last (partials in global
+// memory, one atomic arrival counter per sequence and KV head, nobody waits).
 //
 // Data path: a block's 16 K rows and 16 V rows (256 bytes each) travel HBM -> shared memory with
 // 16-byte cp.async, one full row per half-warp per instruction (so every request covers whole
@@ -76,6 +77,12 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// two adjacent outputs (even index), bf16 or fp32
+__device__ __forceinline__ void store_pair(void* out, int is_fp32, int64_t index, float x, float y) {
+  if (is_fp32) *reinterpret_cast<float2*>(reinterpret_cast<float*>(out) + index) = make_float2(x, y);
+  else *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(out) + index) = __floats2bfloat162_rn(x, y);
 }
 
 // number of attended tokens of sequence b and the pieces needed to enumerate them
@@ -159,11 +166,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
   const int total_tok = prefix_s[units];
   const int teams = (gridDim.x * kAttnWarps) / a.team_size;
   const int per_team = (((total_tok + teams - 1) / teams) + kBlockTokens - 1) & ~(kBlockTokens - 1);
-  if (blockIdx.x == 0 && a.plan_out != nullptr) {      // the merge kernel re-uses the plan
-    for (int i = tid; i <= units; i += kThreads) a.plan_out[2 + i] = prefix_s[i];
-    if (tid == 0) {
-      a.plan_out[0] = per_team;
-      a.plan_out[1] = teams;
+  if (blockIdx.x == 0) {                               // sequences with nothing to attend: zeros
+    for (int u = 0; u < units; ++u) {
+      if (prefix_s[u + 1] != prefix_s[u]) continue;
+      int b, gb;
+      unit_to_seq(a, u, b, gb);
+      const int64_t head0 = static_cast<int64_t>(b) * a.num_q_heads + static_cast<int64_t>(gb) * G;
+      for (int e = tid; e < a.team_size * G * kHeadDim / 2; e += kThreads)
+        if (HAS_V) store_pair(a.out, a.out_is_fp32, head0 * kHeadDim + 2 * e, 0.f, 0.f);
+      for (int e = tid; e < a.team_size * G; e += kThreads)
+        if (a.stats != nullptr) {
+          a.stats[(head0 + e) * 2 + 0] = -INFINITY;
+          a.stats[(head0 + e) * 2 + 1] = 0.f;
+        }
     }
   }
   const int wglobal = blockIdx.x * kAttnWarps + warp;
@@ -281,13 +296,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
   float o[8][4];                                       // O^T tiles: dims {64 (j>>2) + 8 g8 + 2 (j&3) + (0|1)} x heads {2 t4, 2 t4 + 1}
   float m_ref = -INFINITY, l_part = 0.f;               // head g8 (identical in the 4 lanes of a group)
   const bool head_ok = g8 < G;
-  int act_u = -1, act_g = 0, act_ntok = 0, act_vs = 0, act_N = 0;
+  int act_u = -1, act_b = 0, act_g = 0, act_ntok = 0, act_vs = 0, act_N = 0;
   float* logit_row = nullptr;
 
   auto begin_unit = [&](int u, int b) {
     int b2, gb;
     unit_to_seq(a, u, b2, gb);
     act_u = u;
+    act_b = b;
     act_g = gb + team_lane;
     const SeqGeom sg = load_geom(a, b);
     act_ntok = sg.n_tok; act_vs = sg.vs; act_N = sg.N;
@@ -309,11 +325,35 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
                     ? a.logits + (static_cast<int64_t>(b) * a.num_q_heads + act_g * G + g8) * a.n_stride
                     : nullptr;
   };
-  // partial of (team, unit) for this warp's KV head: slot (team + unit) * team_size + team_lane
+  // Leaving a sequence. If its whole (padded) token range lies inside this team's range the warp
+  // normalises and writes the result itself. Otherwise it stores its partial (slot (team + unit) *
+  // team_size + lane-in-team), bumps the (unit, KV head) arrival counter, and the warp that arrives
+  // last merges all partials of that (unit, KV head): no waiting anywhere.
   auto end_unit = [&]() {
     float l = l_part;
     l += __shfl_xor_sync(0xffffffffu, l, 1);
     l += __shfl_xor_sync(0xffffffffu, l, 2);
+    const int ubeg = prefix_s[act_u], uend = prefix_s[act_u + 1];
+    const int t_lo = ubeg / per_team, t_hi = (uend - 1) / per_team;
+    const int64_t head0 = static_cast<int64_t>(act_b) * a.num_q_heads + static_cast<int64_t>(act_g) * G;
+    if (t_lo == t_hi) {
+      if (t4 == 0 && head_ok && a.stats != nullptr) {
+        a.stats[(head0 + g8) * 2 + 0] = m_ref;
+        a.stats[(head0 + g8) * 2 + 1] = l;
+      }
+      if (HAS_V) {
+        const float l0 = __shfl_sync(0xffffffffu, l, 8 * t4), l1 = __shfl_sync(0xffffffffu, l, 8 * t4 + 4);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int d0 = 64 * (j >> 2) + 8 * g8 + 2 * (j & 3);
+          if (2 * t4 < G) store_pair(a.out, a.out_is_fp32, (head0 + 2 * t4) * kHeadDim + d0,
+                                     l0 > 0.f ? o[j][0] / l0 : 0.f, l0 > 0.f ? o[j][2] / l0 : 0.f);
+          if (2 * t4 + 1 < G) store_pair(a.out, a.out_is_fp32, (head0 + 2 * t4 + 1) * kHeadDim + d0,
+                                         l1 > 0.f ? o[j][1] / l1 : 0.f, l1 > 0.f ? o[j][3] / l1 : 0.f);
+        }
+      }
+      return;
+    }
     const int64_t slot = (static_cast<int64_t>(team) + act_u) * a.team_size + team_lane;
     if (t4 == 0 && head_ok) {
       a.part_ml[(slot * kMaxGroup + g8) * 2 + 0] = m_ref;
@@ -326,6 +366,67 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
         float* base = a.part_acc + (slot * kMaxGroup + 2 * t4) * kHeadDim + d0;
         if (2 * t4 < G) *reinterpret_cast<float2*>(base) = make_float2(o[j][0], o[j][2]);
         if (2 * t4 + 1 < G) *reinterpret_cast<float2*>(base + kHeadDim) = make_float2(o[j][1], o[j][3]);
+      }
+    }
+    __threadfence();                                   // partial visible before the arrival is counted
+    __syncwarp();
+    int* counter = a.counters + act_u * a.team_size + team_lane;
+    int prev = 0;
+    if (lane == 0) prev = atomicAdd(counter, 1);
+    prev = __shfl_sync(0xffffffffu, prev, 0);
+    if (prev != t_hi - t_lo) return;                   // someone else arrives later and merges
+    if (lane == 0) *counter = 0;                       // ready for the next launch
+    __threadfence();
+    // lane owns dims 4 lane .. 4 lane + 3 of every head; two partials per round, all loads of a
+    // round issued before any is used (the merge costs one memory latency per round)
+    float M[G], den[G];
+    float4 num[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      M[h] = -INFINITY;
+      den[h] = 0.f;
+      num[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    for (int t0 = t_lo; t0 <= t_hi; t0 += 2) {
+      float2 ml[2][G];
+      float4 acc[2][G];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int t = min(t0 + r, t_hi);               // an odd tail re-reads the last partial (ignored below)
+        const int64_t sl = (static_cast<int64_t>(t) + act_u) * a.team_size + team_lane;
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          ml[r][h] = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (sl * kMaxGroup + h) * 2));
+          acc[r][h] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (HAS_V) acc[r][h] = __ldcg(reinterpret_cast<const float4*>(a.part_acc + (sl * kMaxGroup + h) * kHeadDim) + lane);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        if (t0 + r > t_hi) continue;
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          if (ml[r][h].x == -INFINITY) continue;
+          const float Mn = fmaxf(M[h], ml[r][h].x);
+          const float so = (M[h] == -INFINITY) ? 0.f : exp2f(M[h] - Mn), sn = exp2f(ml[r][h].x - Mn);
+          num[h].x = num[h].x * so + acc[r][h].x * sn; num[h].y = num[h].y * so + acc[r][h].y * sn;
+          num[h].z = num[h].z * so + acc[r][h].z * sn; num[h].w = num[h].w * so + acc[r][h].w * sn;
+          den[h] = den[h] * so + ml[r][h].y * sn;
+          M[h] = Mn;
+        }
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      if (HAS_V) {
+        const int64_t oi = (head0 + h) * kHeadDim + 4 * lane;
+        const float inv = den[h] > 0.f ? 1.f / den[h] : 0.f;
+        store_pair(a.out, a.out_is_fp32, oi, num[h].x * inv, num[h].y * inv);
+        store_pair(a.out, a.out_is_fp32, oi + 2, num[h].z * inv, num[h].w * inv);
+      }
+      if (lane == 0 && a.stats != nullptr) {
+        a.stats[(head0 + h) * 2 + 0] = M[h];
+        a.stats[(head0 + h) * 2 + 1] = den[h];
       }
     }
   };
@@ -429,42 +530,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
   if (act_u >= 0) end_unit();
 }
 
-// One CTA per (sequence, query head): merge the partials of the teams whose ranges touch it.
-__global__ void __launch_bounds__(kHeadDim) attn_combine_kernel(const AttnLaunch a, void* out, int out_is_fp32,
-                                                                float* stats) {
-  const int h = blockIdx.x, b = blockIdx.y, dd = threadIdx.x;
-  const int G = a.num_q_heads / a.num_kv_heads;
-  const int g = h / G, hh = h - g * G;
-  const int u = b * a.units_per_seq + g / a.team_size, team_lane = g % a.team_size;
-  const int per_team = a.plan_out[0];
-  const int begin = a.plan_out[2 + u], end = a.plan_out[3 + u];
-  float M = -INFINITY, num = 0.f, den = 0.f;
-  if (end > begin && per_team > 0) {
-    const int t_lo = begin / per_team, t_hi = (end - 1) / per_team;
-    for (int t = t_lo; t <= t_hi; ++t) {
-      const int64_t slot = (static_cast<int64_t>(t) + u) * a.team_size + team_lane;
-      const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (slot * kMaxGroup + hh) * 2);
-      const float acc = out != nullptr ? a.part_acc[(slot * kMaxGroup + hh) * kHeadDim + dd] : 0.f;
-      if (ml.x == -INFINITY) continue;
-      const float Mn = fmaxf(M, ml.x);
-      const float s_old = (M == -INFINITY) ? 0.f : exp2f(M - Mn), s_new = exp2f(ml.x - Mn);
-      num = num * s_old + acc * s_new;
-      den = den * s_old + ml.y * s_new;
-      M = Mn;
-    }
-  }
-  if (out != nullptr) {
-    const float r = den > 0.f ? num / den : 0.f;
-    const int64_t oi = (static_cast<int64_t>(b) * a.num_q_heads + h) * kHeadDim + dd;
-    if (out_is_fp32) reinterpret_cast<float*>(out)[oi] = r;
-    else reinterpret_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(r);
-  }
-  if (stats != nullptr && dd == 0) {
-    stats[(static_cast<int64_t>(b) * a.num_q_heads + h) * 2 + 0] = M;
-    stats[(static_cast<int64_t>(b) * a.num_q_heads + h) * 2 + 1] = den;
-  }
-}
-
 constexpr int kFinalizeThreads = 256;
 
 __global__ void __launch_bounds__(kFinalizeThreads) scores_finalize_kernel(
@@ -539,7 +604,6 @@ cudaError_t configure_kernels() {
   cudaError_t e;
   // keep the SMs' shared-memory carve-out where the attention kernel needs it, so that the small
   // kernels in between do not trigger a reconfiguration
-  if ((e = cudaFuncSetAttribute(attn_combine_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(scores_finalize_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(image_mass_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
 #define X(g)                                                \
@@ -548,13 +612,6 @@ cudaError_t configure_kernels() {
   FASTOCR_FOR_EACH_GROUP(X)
 #undef X
   return cudaSuccess;
-}
-
-cudaError_t launch_attn_combine(const AttnLaunch& a, void* out, int out_is_fp32, float* stats, cudaStream_t s) {
-  dim3 grid(a.num_q_heads, a.batch);
-  attn_combine_kernel<<<grid, kHeadDim, 0, s>>>(a, out, out_is_fp32, stats);
-  count_launches(1);
-  return cudaGetLastError();
 }
 
 cudaError_t launch_scores_finalize(const float* logits, const float* stats, const int32_t* vis_len, int32_t batch,

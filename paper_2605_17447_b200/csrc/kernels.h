@@ -42,17 +42,17 @@ struct AttnLaunch {
   // workspace
   float* part_acc;            // [slots][8][128], slot = (team + unit) * team_size + lane-in-team
   float* part_ml;             // [slots][8][2]  (max, sum) in the log2 domain
-  int32_t* plan_out;          // [2 + units + 1]: tokens per team, teams, padded token prefix per unit
+  int32_t* counters;          // [units * team_size] arrival counters, zero between launches
+  // results
+  void* out;                  // [B][H][128] bf16 or fp32 (unused when v == nullptr)
+  int32_t out_is_fp32;
+  float* stats;               // nullptr or [B][H][2]: per-head softmax (max, sum) over the whole attended set
   float* logits;              // nullptr or [B][H][n_stride], log2-domain logits of image tokens
   int32_t n_stride;
   unsigned long long* fault_counter;
 };
 
 cudaError_t launch_attn_partial(const AttnLaunch& a, cudaStream_t s);
-
-// Merges the per-split partials of every (sequence, head): writes out (bf16 / fp32) unless out is
-// nullptr, and the global (max, sum) per head to stats [B][H][2] unless stats is nullptr.
-cudaError_t launch_attn_combine(const AttnLaunch& a, void* out, int out_is_fp32, float* stats, cudaStream_t s);
 
 // scores[b][i] = (1/H) sum_h 2^(logit[b][h][i] - max_h) / sum_h  for i < vis_len[b].
 cudaError_t launch_scores_finalize(const float* logits, const float* stats, const int32_t* vis_len, int32_t batch,
