@@ -21,20 +21,23 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
+def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str | None = None) -> str:
+    """Compile the library. extra_flags / out build a variant (e.g. -DFASTOCR_TRACE) elsewhere."""
+    if out is None and not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
+    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")] + list(extra_flags)
+    lib = out or LIB
+    tag = "" if out is None else "." + os.path.basename(out).replace(".so", "")
     if verbose:
         flags += ["-Xptxas", "-v"]
     objs = []
     for src in SOURCES:
-        obj = os.path.join(CSRC, src.replace(".cu", ".o"))
+        obj = os.path.join(CSRC, src.replace(".cu", tag + ".o"))
         subprocess.check_call([nvcc, *flags, "-c", os.path.join(CSRC, src), "-o", obj])
         objs.append(obj)
-    subprocess.check_call([nvcc, "-shared", "-o", LIB, *objs, "-lcudart"])
-    return LIB
+    subprocess.check_call([nvcc, "-shared", "-o", lib, *objs, "-lcudart"])
+    return lib
 
 
 if __name__ == "__main__":

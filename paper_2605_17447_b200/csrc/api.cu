@@ -27,12 +27,13 @@ struct fastocr_ctx {
   int64_t cap_items = 0;        // partial slots: one per (team, sequence) pair and KV head
   float* part_acc = nullptr;    // [cap_items][8][128]
   float* part_ml = nullptr;     // [cap_items][8][2]
-  int32_t* counters = nullptr;  // [kMaxUnits * 8] arrival counters of the split merge (zero between launches)
+  int32_t* counters = nullptr;  // [kMaxUnits * kAttnWarps] arrival counters of the split merge (zero between launches)
   float* logits = nullptr;      // [max_batch][H][max_vis_len]
   float* stats = nullptr;       // [max_batch][H][2]
   float* scores = nullptr;      // [max_batch][max_vis_len] (decode_step scratch)
   unsigned long long* faults = nullptr;
-  int ctas_per_sm = 1;          // persistent attention CTAs per SM
+  int ctas_per_sm = 2;          // persistent attention CTAs per SM
+  unsigned long long* trace = nullptr;   // set only by debug builds
   char err[512] = {0};
   // optional per-launch timing
   std::vector<cudaEvent_t> prof_ev;   // 2 per timed launch
@@ -111,6 +112,7 @@ AttnLaunch make_launch(const fastocr_ctx* ctx, const fastocr_kv_view* kv, const 
   a.part_ml = ctx->part_ml;
   a.fault_counter = ctx->faults;
   a.counters = ctx->counters;
+  a.trace = ctx->trace;
   a.team_size = fastocr::team_size_for(kv->num_kv_heads);
   a.units_per_seq = kv->num_kv_heads / a.team_size;
   a.grid_ctas = ctx->sm_count * ctx->ctas_per_sm;
@@ -234,8 +236,8 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   if ((e = cudaMalloc(&ctx->part_acc, bytes_acc)) != cudaSuccess || (e = cudaMalloc(&ctx->part_ml, bytes_ml)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->logits, bytes_logits)) != cudaSuccess || (e = cudaMalloc(&ctx->stats, bytes_stats)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->scores, bytes_scores)) != cudaSuccess ||
-      (e = cudaMalloc(&ctx->counters, fastocr::kMaxUnits * 8 * sizeof(int32_t))) != cudaSuccess ||
-      (e = cudaMemset(ctx->counters, 0, fastocr::kMaxUnits * 8 * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->counters, fastocr::kMaxUnits * fastocr::kAttnWarps * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMemset(ctx->counters, 0, fastocr::kMaxUnits * fastocr::kAttnWarps * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->faults, sizeof(unsigned long long))) != cudaSuccess ||
       (e = cudaMemset(ctx->faults, 0, sizeof(unsigned long long))) != cudaSuccess) {
     fastocr_destroy(ctx);
@@ -446,6 +448,11 @@ fastocr_status fastocr_profile_end(fastocr_ctx* ctx, double* ms_per_class, int64
   if (e != cudaSuccess) return cuda_fail(ctx, e, "profile_end");
   return FASTOCR_OK;
 }
+
+#ifdef FASTOCR_TRACE
+// debug builds: device buffer of 8 timestamps per attention warp (not part of the public interface)
+void fastocr_debug_set_trace(fastocr_ctx* ctx, unsigned long long* buf) { ctx->trace = buf; }
+#endif
 
 int64_t fastocr_launch_count(void) { return fastocr::g_launches.load(std::memory_order_relaxed); }
 

@@ -6,7 +6,7 @@
 // in one index space, sequence after sequence, each sequence padded to a multiple of 16 tokens.
 // That space is cut into equal ranges, one per "team"; a team is one warp per KV head (so the
 // whole 1-2 KB token row is fetched by neighbouring warps at about the same time), and the grid is
-// one persistent CTA of eight autonomous warps per SM. Every warp therefore streams the same
+// two persistent CTAs of four autonomous warps per SM. Every warp therefore streams the same
 // number of 16-token blocks, pays one pipeline prologue per launch, and never meets a CTA barrier
 // after set-up. A range may cross sequence boundaries: the warp then finishes the sequence it leaves
 // and starts a new one. A sequence covered by one team is normalised and written by that team;
@@ -47,6 +47,7 @@ constexpr int kStages = 3;
 constexpr int kThreads = kAttnWarps * 32;
 constexpr int kBlockTokens = 16;        // tokens per warp per pipeline stage
 constexpr float kRescaleSlack = 8.0f;   // log2 units
+constexpr int kMergeRound = 3;          // partials fetched together by the merging warp
 
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -131,14 +132,29 @@ __device__ __forceinline__ void unit_to_seq(const AttnLaunch& a, int u, int& b, 
   }
 }
 
+#ifdef FASTOCR_TRACE
+__device__ __forceinline__ unsigned long long trace_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define FASTOCR_TRACE_MARK(slot)                                                                            \
+  do {                                                                                                      \
+    if (a.trace != nullptr && lane == 0) a.trace[(blockIdx.x * kAttnWarps + warp) * 8 + (slot)] = trace_now(); \
+  } while (0)
+#else
+#define FASTOCR_TRACE_MARK(slot) do { } while (0)
+#endif
+
 template <int G, bool HAS_V>
-__global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaunch a) {
+__global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaunch a) {
   extern __shared__ __align__(16) unsigned char smem[];
   using L = Smem<HAS_V>;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g8 = lane >> 2, t4 = lane & 3;             // MMA fragment coordinates: group, thread-in-group
   const int units = a.batch * a.units_per_seq;
 
+  FASTOCR_TRACE_MARK(0);
   // ---- set-up: padded token prefix over units (warp 0), the only CTA barrier of the kernel -----
   int* prefix_s = reinterpret_cast<int*>(smem + L::prefix);
   if (warp == 0) {
@@ -163,6 +179,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
     if (lane == 0) prefix_s[units] = carry;
   }
   __syncthreads();
+  FASTOCR_TRACE_MARK(1);
   const int total_tok = prefix_s[units];
   const int teams = (gridDim.x * kAttnWarps) / a.team_size;
   const int per_team = (((total_tok + teams - 1) / teams) + kBlockTokens - 1) & ~(kBlockTokens - 1);
@@ -217,13 +234,17 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
   unit_to_seq(a, cur_u, cur_b, cur_gb);
   SeqGeom cur_geom = load_geom(a, cur_b);
 
-  int fu[5], fj[5], fb[5];                             // unit, first token within unit, sequence
+  int fu[5], fj[5], fb[5], fvs[5], fN[5];              // unit, first token within unit, sequence, image span
 #pragma unroll
-  for (int i = 0; i < 5; ++i) { fu[i] = -1; fj[i] = 0; fb[i] = 0; }
+  for (int i = 0; i < 5; ++i) { fu[i] = -1; fj[i] = 0; fb[i] = 0; fvs[i] = 0; fN[i] = 0; }
   int pos_p = 0, row_p = 0;                            // lanes 0..15: position (block n+4 -> n+3), row (n+3 -> n+2)
+  bool idx_p = false;                                  // pos_p is a raw index-list entry
 
-  // describe block n (if it exists) into FIFO slot `slot` and start its position lookup
-  auto stage_pos = [&](int n, int& du, int& dj, int& db) -> int {
+  // Describe block n (if it exists) and start its position lookup. For a selected image token the
+  // value returned is the raw entry of the index list and `from_idx` is set: nothing may depend on
+  // the loaded value here, it is checked and turned into a position one block later (stage_row).
+  auto stage_pos = [&](int n, int& du, int& dj, int& db, int& dvs, int& dN, bool& from_idx) -> int {
+    from_idx = false;
     if (n >= n_blocks) { du = -1; return 0; }
     const int off = r0 + n * kBlockTokens;
     while (off >= cur_end) {
@@ -237,6 +258,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
     du = cur_u;
     dj = off - prefix_s[cur_u];
     db = cur_b;
+    dvs = cur_geom.vs;
+    dN = cur_geom.N;
     int pos = 0;
     if (lane < kBlockTokens) {
       const int j = min(dj + lane, cur_geom.n_tok - 1);
@@ -245,19 +268,23 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
         if (j >= cur_geom.vs + cur_geom.kept_vis) {
           pos = j - cur_geom.kept_vis + cur_geom.N;
         } else if (j >= cur_geom.vs) {
-          int r = __ldg(a.idx + static_cast<int64_t>(cur_b) * a.k_stride + (j - cur_geom.vs));
-          if (r < 0 || r >= cur_geom.N) {              // never read outside the image span
-            atomicAdd(a.fault_counter, 1ULL);
-            r = r < 0 ? 0 : cur_geom.N - 1;
-          }
-          pos = cur_geom.vs + r;
+          pos = __ldg(a.idx + static_cast<int64_t>(cur_b) * a.k_stride + (j - cur_geom.vs));
+          from_idx = true;
         }
       }
     }
     return pos;
   };
-  auto stage_row = [&](int du, int db, int pos) -> int {
-    if (du < 0 || a.page_size == 0 || lane >= kBlockTokens) return pos;
+  auto stage_row = [&](int du, int db, int dvs, int dN, bool from_idx, int pos) -> int {
+    if (du < 0 || lane >= kBlockTokens) return pos;
+    if (from_idx) {
+      if (pos < 0 || pos >= dN) {                      // never read outside the image span
+        atomicAdd(a.fault_counter, 1ULL);
+        pos = pos < 0 ? 0 : dN - 1;
+      }
+      pos += dvs;
+    }
+    if (a.page_size == 0) return pos;
     const int page = __ldg(a.block_table + static_cast<int64_t>(db) * a.max_pages + pos / a.page_size);
     return page * a.page_size + pos % a.page_size;
   };
@@ -279,17 +306,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
   };
 
   // ---- prologue: positions of blocks 0..3, rows of 0..2, copies of 0..1 -------------------------
-  int pos0 = stage_pos(0, fu[0], fj[0], fb[0]);
-  int pos1 = stage_pos(1, fu[1], fj[1], fb[1]);
-  int pos2 = stage_pos(2, fu[2], fj[2], fb[2]);
-  pos_p = stage_pos(3, fu[3], fj[3], fb[3]);
+  bool idx0, idx1, idx2;
+  int pos0 = stage_pos(0, fu[0], fj[0], fb[0], fvs[0], fN[0], idx0);
+  int pos1 = stage_pos(1, fu[1], fj[1], fb[1], fvs[1], fN[1], idx1);
+  int pos2 = stage_pos(2, fu[2], fj[2], fb[2], fvs[2], fN[2], idx2);
+  pos_p = stage_pos(3, fu[3], fj[3], fb[3], fvs[3], fN[3], idx_p);
   {
-    const int row0 = stage_row(fu[0], fb[0], pos0);
-    const int row1 = stage_row(fu[1], fb[1], pos1);
-    row_p = stage_row(fu[2], fb[2], pos2);
+    const int row0 = stage_row(fu[0], fb[0], fvs[0], fN[0], idx0, pos0);
+    const int row1 = stage_row(fu[1], fb[1], fvs[1], fN[1], idx1, pos1);
+    row_p = stage_row(fu[2], fb[2], fvs[2], fN[2], idx2, pos2);
     stage_issue(0, fu[0], fb[0], row0);
     stage_issue(1, fu[1], fb[1], row1);
   }
+  FASTOCR_TRACE_MARK(2);
 
   // ---- per-unit state ----------------------------------------------------------------------------
   uint32_t qw[4][4];                                   // A fragments of Q: head g8, dims 32j + 8 t4 .. + 8
@@ -377,7 +406,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
     if (prev != t_hi - t_lo) return;                   // someone else arrives later and merges
     if (lane == 0) *counter = 0;                       // ready for the next launch
     __threadfence();
-    // lane owns dims 4 lane .. 4 lane + 3 of every head; two partials per round, all loads of a
+    // lane owns dims 4 lane .. 4 lane + 3 of every head; kMergeRound partials per round, all loads of a
     // round issued before any is used (the merge costs one memory latency per round)
     float M[G], den[G];
     float4 num[G];
@@ -387,11 +416,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
       den[h] = 0.f;
       num[h] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    for (int t0 = t_lo; t0 <= t_hi; t0 += 2) {
-      float2 ml[2][G];
-      float4 acc[2][G];
+    for (int t0 = t_lo; t0 <= t_hi; t0 += kMergeRound) {
+      float2 ml[kMergeRound][G];
+      float4 acc[kMergeRound][G];
 #pragma unroll
-      for (int r = 0; r < 2; ++r) {
+      for (int r = 0; r < kMergeRound; ++r) {
         const int t = min(t0 + r, t_hi);               // an odd tail re-reads the last partial (ignored below)
         const int64_t sl = (static_cast<int64_t>(t) + act_u) * a.team_size + team_lane;
 #pragma unroll
@@ -402,7 +431,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
         }
       }
 #pragma unroll
-      for (int r = 0; r < 2; ++r) {
+      for (int r = 0; r < kMergeRound; ++r) {
         if (t0 + r > t_hi) continue;
 #pragma unroll
         for (int h = 0; h < G; ++h) {
@@ -438,6 +467,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
     }
     cp_async_wait<kStages - 2>();
     __syncwarp();                                      // every lane's copies of this block have landed
+    if (n == 0) FASTOCR_TRACE_MARK(3);
     const uint32_t src = ring_warp + (n % kStages) * L::kStageBytes;
     // ---- S^T = Q K^T for the two 8-token tiles ------------------------------------------------
     // lane (g8, t4) reads chunk 4j + t4 of rows g8 and 8 + g8: per 8-lane phase two rows whose
@@ -465,8 +495,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
     }
     // ---- keep the look-ahead stages moving ----------------------------------------------------
     stage_issue(n + 2, fu[2], fb[2], row_p);
-    row_p = stage_row(fu[3], fb[3], pos_p);
-    pos_p = stage_pos(n + 4, fu[4], fj[4], fb[4]);
+    row_p = stage_row(fu[3], fb[3], fvs[3], fN[3], idx_p, pos_p);
+    pos_p = stage_pos(n + 4, fu[4], fj[4], fb[4], fvs[4], fN[4], idx_p);
 
     // ---- online softmax for head g8, tokens j0 + {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4} ---------
     const int j0 = fj[0];
@@ -524,10 +554,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_stream_kernel(const AttnLaun
     }
     // ---- advance the descriptor FIFO ----------------------------------------------------------
 #pragma unroll
-    for (int i = 0; i < 4; ++i) { fu[i] = fu[i + 1]; fj[i] = fj[i + 1]; fb[i] = fb[i + 1]; }
+    for (int i = 0; i < 4; ++i) {
+      fu[i] = fu[i + 1]; fj[i] = fj[i + 1]; fb[i] = fb[i + 1]; fvs[i] = fvs[i + 1]; fN[i] = fN[i + 1];
+    }
   }
   cp_async_wait<0>();
+  FASTOCR_TRACE_MARK(4);
   if (act_u >= 0) end_unit();
+  FASTOCR_TRACE_MARK(5);
 }
 
 constexpr int kFinalizeThreads = 256;

@@ -7,13 +7,15 @@ namespace fastocr {
 
 constexpr int kHeadDim = 128;
 constexpr int kMaxGroup = 8;          // query heads per KV head handled by one CTA
-constexpr int kAttnWarps = 8;         // autonomous warps per persistent attention CTA
+constexpr int kAttnWarps = 4;         // autonomous warps per persistent attention CTA (two CTAs per SM)
 constexpr int kMaxUnits = 2048;       // sequences x KV-head slices per launch (prefix lives in shared memory)
 constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
 
 // Warps per team: one per KV head when that divides the CTA's warp count, else one.
 inline int team_size_for(int num_kv_heads) {
-  return (num_kv_heads == 1 || num_kv_heads == 2 || num_kv_heads == 4 || num_kv_heads == 8) ? num_kv_heads : 1;
+  for (int ts = kAttnWarps; ts > 1; ts >>= 1)
+    if (num_kv_heads % ts == 0) return ts;
+  return 1;
 }
 
 struct AttnLaunch {
@@ -50,6 +52,7 @@ struct AttnLaunch {
   float* logits;              // nullptr or [B][H][n_stride], log2-domain logits of image tokens
   int32_t n_stride;
   unsigned long long* fault_counter;
+  unsigned long long* trace;  // debug builds only (FASTOCR_TRACE): per-warp timestamps
 };
 
 cudaError_t launch_attn_partial(const AttnLaunch& a, cudaStream_t s);
