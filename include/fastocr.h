@@ -157,7 +157,8 @@ fastocr_status fastocr_sparse_decode_attn(fastocr_ctx* ctx, const fastocr_kv_vie
  *   refreshes the set; every other layer attends text + the current set. On return (in stream
  *   order) `fixation` holds the set of the deepest focal layer: the F_last of the next step.
  *   layers   host array [L] of views (all with the same batch / heads / spans)
- *   q, out   device [L][B][H][128]; out bf16 or fp32
+ *   q, out   device [L][B][H][128]; out bf16 or fp32; q and out must not overlap (consecutive
+ *            pruned layers are launched so that one may start while the previous one drains)
  *   is_focal host uint8 [L]: membership in the focal layer set C
  *   k        device int32 [B]; fixation device int32 [B][k_stride] (in/out)
  *   max_vis_len, max_kept: host bounds as above

@@ -113,6 +113,7 @@ AttnLaunch make_launch(const fastocr_ctx* ctx, const fastocr_kv_view* kv, const 
   a.fault_counter = ctx->faults;
   a.counters = ctx->counters;
   a.trace = ctx->trace;
+  a.wait_at_start = 1;
   a.team_size = fastocr::team_size_for(kv->num_kv_heads);
   a.units_per_seq = kv->num_kv_heads / a.team_size;
   a.grid_ctas = ctx->sm_count * ctx->ctas_per_sm;
@@ -175,14 +176,17 @@ fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
   return FASTOCR_OK;
 }
 
+// inputs_settled: nothing this launch reads (lengths, index list, queries, cache) was written by
+// the launch issued just before it on the stream, so it may start while that one drains.
 fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, const int32_t* idx,
                            const int32_t* k, int32_t k_stride, int32_t max_kept, void* out, int out_is_fp32,
-                           cudaStream_t s) {
+                           bool inputs_settled, cudaStream_t s) {
   const int max_len = (max_kept > 0 && max_kept < kv->max_seq_len) ? max_kept : kv->max_seq_len;
   AttnLaunch a = make_launch(ctx, kv, q, true, max_len);
   a.idx = idx;
   a.kcount = k;
   a.k_stride = k_stride;
+  a.wait_at_start = inputs_settled ? 0 : 1;
   a.out = out;
   a.out_is_fp32 = out_is_fp32;
   {
@@ -334,7 +338,7 @@ fastocr_status fastocr_sparse_decode_attn(fastocr_ctx* ctx, const fastocr_kv_vie
   if (st != FASTOCR_OK) return st;
   if (idx == nullptr || k == nullptr || out == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL idx, k or out");
   if (k_stride <= 0 || max_kept < 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "k_stride must be positive, max_kept non-negative");
-  return sparse_impl(ctx, kv, q, idx, k, k_stride, max_kept, out, out_is_fp32, static_cast<cudaStream_t>(stream));
+  return sparse_impl(ctx, kv, q, idx, k, k_stride, max_kept, out, out_is_fp32, false, static_cast<cudaStream_t>(stream));
 }
 
 fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
@@ -358,6 +362,7 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
   const int64_t per_layer = static_cast<int64_t>(layers[0].batch) * layers[0].num_q_heads * fastocr::kHeadDim;
   const size_t q_bytes = per_layer * 2, o_bytes = per_layer * (out_is_fp32 ? 4 : 2);
   bool have = has_fixation != 0;
+  bool prev_was_pruned = false;   // the launch just before was a pruned-attention kernel of this step
   for (int l = 0; l < num_layers; ++l) {
     const void* ql = static_cast<const char*>(q) + l * q_bytes;
     void* ol = static_cast<char*>(out) + l * o_bytes;
@@ -374,9 +379,13 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
                          "top-k launch");
       }
       have = true;
+      prev_was_pruned = false;
     } else {
-      st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, s);
+      // a pruned layer that follows another pruned layer reads nothing the latter wrote (its
+      // queries, index set and cache were all complete before), so the two may overlap
+      st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, prev_was_pruned, s);
       if (st != FASTOCR_OK) return st;
+      prev_was_pruned = !ctx->prof_on;
     }
   }
   if (has_fixation_out != nullptr) *has_fixation_out = have ? 1 : 0;

@@ -80,6 +80,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// Programmatic dependent launch: a launch of this kernel may begin while the previous kernel in the
+// stream is still draining. dependents_may_launch() lets the next kernel's CTAs be scheduled as
+// soon as resources free up; wait_for_prior_grids() blocks until every earlier kernel has finished
+// and its writes are visible (a no-op when the launch carried no such attribute).
+__device__ __forceinline__ void dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void wait_for_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // two adjacent outputs (even index), bf16 or fp32
 __device__ __forceinline__ void store_pair(void* out, int is_fp32, int64_t index, float x, float y) {
   if (is_fp32) *reinterpret_cast<float2*>(reinterpret_cast<float*>(out) + index) = make_float2(x, y);
@@ -155,6 +162,10 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
   const int units = a.batch * a.units_per_seq;
 
   FASTOCR_TRACE_MARK(0);
+  // Everything read before the first wait_for_prior_grids() (lengths, index list, queries, cache)
+  // must not have been produced by the kernel launched just before this one; the host says so.
+  if (a.wait_at_start) wait_for_prior_grids();
+  dependents_may_launch();
   // ---- set-up: padded token prefix over units (warp 0), the only CTA barrier of the kernel -----
   int* prefix_s = reinterpret_cast<int*>(smem + L::prefix);
   if (warp == 0) {
@@ -186,6 +197,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
   if (blockIdx.x == 0) {                               // sequences with nothing to attend: zeros
     for (int u = 0; u < units; ++u) {
       if (prefix_s[u + 1] != prefix_s[u]) continue;
+      wait_for_prior_grids();
       int b, gb;
       unit_to_seq(a, u, b, gb);
       const int64_t head0 = static_cast<int64_t>(b) * a.num_q_heads + static_cast<int64_t>(gb) * G;
@@ -359,6 +371,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
   // team_size + lane-in-team), bumps the (unit, KV head) arrival counter, and the warp that arrives
   // last merges all partials of that (unit, KV head): no waiting anywhere.
   auto end_unit = [&]() {
+    wait_for_prior_grids();                            // results and the shared workspace are written from here on
     float l = l_part;
     l += __shfl_xor_sync(0xffffffffu, l, 1);
     l += __shfl_xor_sync(0xffffffffu, l, 2);
@@ -605,9 +618,19 @@ __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restric
 
 template <int G, bool HAS_V>
 cudaError_t launch_partial_t(const AttnLaunch& a, cudaStream_t s) {
-  attn_stream_kernel<G, HAS_V><<<a.grid_ctas, kThreads, Smem<HAS_V>::total, s>>>(a);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.grid_ctas);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = Smem<HAS_V>::total;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, attn_stream_kernel<G, HAS_V>, a);
   count_launches(1);
-  return cudaGetLastError();
+  return e;
 }
 
 template <int G, bool HAS_V>

@@ -41,6 +41,7 @@ struct AttnLaunch {
   int32_t team_size;
   int32_t units_per_seq;
   int32_t grid_ctas;          // persistent CTAs (kAttnWarps warps each)
+  int32_t wait_at_start;      // 0: no input of this launch was written by the launch just before it
   // workspace
   float* part_acc;            // [slots][8][128], slot = (team + unit) * team_size + lane-in-team
   float* part_ml;             // [slots][8][2]  (max, sum) in the log2 domain
