@@ -27,13 +27,14 @@ struct fastocr_ctx {
   int64_t cap_items = 0;        // partial slots: one per (team, sequence) pair and KV head
   float* part_acc = nullptr;    // [cap_items][8][128]
   float* part_ml = nullptr;     // [cap_items][8][2]
-  int32_t* counters = nullptr;  // [kMaxUnits * kAttnWarps] arrival counters of the split merge (zero between launches)
+  int32_t* counters = nullptr;  // [kMaxUnits] arrival counters of the split merge (zero between launches)
   float* logits = nullptr;      // [max_batch][H][max_vis_len]
   float* stats = nullptr;       // [max_batch][H][2]
   float* scores = nullptr;      // [max_batch][max_vis_len] (decode_step scratch)
   unsigned long long* faults = nullptr;
   int ctas_per_sm = 2;          // persistent attention CTAs per SM
   unsigned long long* trace = nullptr;   // set only by debug builds
+  unsigned trace_seq = 0;
   char err[512] = {0};
   // optional per-launch timing
   std::vector<cudaEvent_t> prof_ev;   // 2 per timed launch
@@ -79,11 +80,8 @@ fastocr_status check_view(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "seq_stride_tokens < max_seq_len");
   }
   if (!(kv->sm_scale > 0.f) || !std::isfinite(kv->sm_scale)) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "sm_scale must be positive");
-  {
-    const int ts = fastocr::team_size_for(kv->num_kv_heads);
-    if (static_cast<int64_t>(kv->batch) * (kv->num_kv_heads / ts) > fastocr::kMaxUnits)
-      return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "batch x KV-head slices exceeds %d", fastocr::kMaxUnits);
-  }
+  if (static_cast<int64_t>(kv->batch) * kv->num_kv_heads > fastocr::kMaxUnits)
+    return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "batch x num_kv_heads exceeds %d", fastocr::kMaxUnits);
   if (kv->batch > ctx->lim.max_batch || kv->num_q_heads > ctx->lim.num_q_heads ||
       kv->num_kv_heads > ctx->lim.num_kv_heads || kv->max_seq_len > ctx->lim.max_seq_len)
     return fail(ctx, FASTOCR_ERR_WORKSPACE, "view (B=%d H=%d Hkv=%d S<=%d) exceeds the context limits (B=%d H=%d Hkv=%d S<=%d)",
@@ -92,7 +90,7 @@ fastocr_status check_view(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
   return FASTOCR_OK;
 }
 
-AttnLaunch make_launch(const fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, bool with_v, int max_len) {
+AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, bool with_v, int max_len) {
   AttnLaunch a{};
   a.k = kv->k;
   a.v = with_v ? kv->v : nullptr;
@@ -112,10 +110,13 @@ AttnLaunch make_launch(const fastocr_ctx* ctx, const fastocr_kv_view* kv, const 
   a.part_ml = ctx->part_ml;
   a.fault_counter = ctx->faults;
   a.counters = ctx->counters;
-  a.trace = ctx->trace;
+#ifdef FASTOCR_TRACE
+  // debug builds: eight rotating trace regions, one per launch
+  a.trace = ctx->trace != nullptr ? ctx->trace + (ctx->trace_seq++ % 8) * 16384 : nullptr;
+#else
+  a.trace = nullptr;
+#endif
   a.wait_at_start = 1;
-  a.team_size = fastocr::team_size_for(kv->num_kv_heads);
-  a.units_per_seq = kv->num_kv_heads / a.team_size;
   a.grid_ctas = ctx->sm_count * ctx->ctas_per_sm;
   (void)max_len;
   return a;
@@ -228,8 +229,8 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
     return FASTOCR_ERR_CUDA;
   }
   ctx->sm_count = sm > 0 ? sm : 148;
-  // one partial slot per (team, unit) pair that can occur: teams + units, times the team size
-  ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * ctx->ctas_per_sm * fastocr::kAttnWarps +
+  // one partial slot per (CTA, unit) pair that can occur: CTAs + units
+  ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * ctx->ctas_per_sm +
                    static_cast<int64_t>(lim->max_batch) * lim->num_kv_heads + 64;
   const int64_t nvis = lim->max_vis_len > 0 ? lim->max_vis_len : 1;
   const size_t bytes_acc = static_cast<size_t>(ctx->cap_items) * fastocr::kMaxGroup * fastocr::kHeadDim * sizeof(float);
@@ -240,8 +241,8 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   if ((e = cudaMalloc(&ctx->part_acc, bytes_acc)) != cudaSuccess || (e = cudaMalloc(&ctx->part_ml, bytes_ml)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->logits, bytes_logits)) != cudaSuccess || (e = cudaMalloc(&ctx->stats, bytes_stats)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->scores, bytes_scores)) != cudaSuccess ||
-      (e = cudaMalloc(&ctx->counters, fastocr::kMaxUnits * fastocr::kAttnWarps * sizeof(int32_t))) != cudaSuccess ||
-      (e = cudaMemset(ctx->counters, 0, fastocr::kMaxUnits * fastocr::kAttnWarps * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->counters, fastocr::kMaxUnits * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMemset(ctx->counters, 0, fastocr::kMaxUnits * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->faults, sizeof(unsigned long long))) != cudaSuccess ||
       (e = cudaMemset(ctx->faults, 0, sizeof(unsigned long long))) != cudaSuccess) {
     fastocr_destroy(ctx);

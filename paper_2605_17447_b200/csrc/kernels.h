@@ -8,15 +8,8 @@ namespace fastocr {
 constexpr int kHeadDim = 128;
 constexpr int kMaxGroup = 8;          // query heads per KV head handled by one CTA
 constexpr int kAttnWarps = 4;         // autonomous warps per persistent attention CTA (two CTAs per SM)
-constexpr int kMaxUnits = 2048;       // sequences x KV-head slices per launch (prefix lives in shared memory)
+constexpr int kMaxUnits = 1024;       // sequences x KV heads per launch (their row prefix lives in shared memory)
 constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
-
-// Warps per team: one per KV head when that divides the CTA's warp count, else one.
-inline int team_size_for(int num_kv_heads) {
-  for (int ts = kAttnWarps; ts > 1; ts >>= 1)
-    if (num_kv_heads % ts == 0) return ts;
-  return 1;
-}
 
 struct AttnLaunch {
   // cache view
@@ -36,16 +29,12 @@ struct AttnLaunch {
   const int32_t* idx;
   const int32_t* kcount;
   int32_t k_stride;
-  // decomposition: a team is team_size warps (one per KV head of a unit); a unit is one sequence x
-  // team_size consecutive KV heads; units_per_seq = num_kv_heads / team_size
-  int32_t team_size;
-  int32_t units_per_seq;
   int32_t grid_ctas;          // persistent CTAs (kAttnWarps warps each)
   int32_t wait_at_start;      // 0: no input of this launch was written by the launch just before it
   // workspace
-  float* part_acc;            // [slots][8][128], slot = (team + unit) * team_size + lane-in-team
+  float* part_acc;            // [slots][8][128], slot = CTA index + unit index (unit = sequence * Hkv + KV head)
   float* part_ml;             // [slots][8][2]  (max, sum) in the log2 domain
-  int32_t* counters;          // [units * team_size] arrival counters, zero between launches
+  int32_t* counters;          // [units] arrival counters, zero between launches
   // results
   void* out;                  // [B][H][128] bf16 or fp32 (unused when v == nullptr)
   int32_t out_is_fp32;
