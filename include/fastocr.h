@@ -183,6 +183,29 @@ int32_t fastocr_focal_layers(const double* mean_ratio, int32_t num_layers, doubl
 double fastocr_attn_flops(double batch, double layers, double hidden, double seq_len);
 
 /*
+ * Pruned decode attention without a context and without any allocation (the paper has no
+ * counterpart; this exists for callers that cannot call cudaMalloc: engines that give all of HBM
+ * to their own pool at start-up, allocator-tracked frameworks, decode loops that must stay out of
+ * the driver's allocator). Same computation and arguments as fastocr_sparse_decode_attn, but the
+ * scratch of the split merge is a fixed array inside the library (about 2.7 MB of device memory
+ * on every GPU that loads it, held until the process exits) instead of a context's workspace.
+ *   - Limit: batch * num_kv_heads <= FASTOCR_NOALLOC_MAX_UNITS, else FASTOCR_ERR_WORKSPACE.
+ *   - The first call on each device resolves the array's device address and sets kernel
+ *     attributes (no allocation); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents (the
+ *     entry point re-zeroes the counters it needs on `stream` before launching). Two calls that
+ *     may overlap on the GPU (different streams without ordering) race on it: serialise them.
+ *   - Runs on the current device; every pointer must belong to it. No cudaMalloc, cudaFree or
+ *     allocating library routine is called. Errors: return code + fastocr_noalloc_last_error()
+ *     (thread-local string).
+ */
+#define FASTOCR_NOALLOC_MAX_UNITS 256
+fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, const void* q, const int32_t* idx,
+                                                  const int32_t* k, int32_t k_stride, void* out, int out_is_fp32,
+                                                  void* stream);
+const char* fastocr_noalloc_last_error(void);
+
+/*
  * Optional per-kernel timing (the paper has no counterpart; measurement aid). Between
  * fastocr_profile_begin and fastocr_profile_end every launch of this context is bracketed by CUDA
  * events on its stream. fastocr_profile_begin creates `max_launches` event pairs (not a hot-path

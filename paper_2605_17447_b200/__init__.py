@@ -4,6 +4,6 @@ marshals pointers. Importing it requires the built library (python -m paper_2605
 from .api import (  # noqa: F401
     Context, KVView, FastOCRError, kept_count, focal_layers, attn_flops, launch_count,
     fastocr_dense_decode_attn, fastocr_focal_scores, fastocr_select_topk, fastocr_sparse_decode_attn,
-    fastocr_decode_step, StepPlan, PROF_CLASSES,
+    fastocr_decode_step, fastocr_sparse_decode_attn_noalloc, StepPlan, PROF_CLASSES,
 )
 from .sharding import shard_sequences  # noqa: F401

@@ -195,6 +195,21 @@ def fastocr_sparse_decode_attn(ctx: Context, kv: KVView, q: torch.Tensor, idx: t
                                                   _stream(stream)))
 
 
+def fastocr_sparse_decode_attn_noalloc(kv: KVView, q: torch.Tensor, idx: torch.Tensor, k: torch.Tensor,
+                                       out: torch.Tensor, stream=None) -> None:
+    """Pruned attention for callers that may not allocate: no Context, the library's built-in scratch
+    array is used (batch * num_kv_heads <= 256; calls on one device must not overlap on the GPU)."""
+    _dev(q, torch.bfloat16, "q")
+    _dev(idx, torch.int32, "idx")
+    _dev(k, torch.int32, "k")
+    lib = _lib.load()
+    st = kv.struct()
+    rc = lib.fastocr_sparse_decode_attn_noalloc(C.byref(st), _ptr(q), _ptr(idx), _ptr(k), int(idx.shape[-1]), _ptr(out),
+                                                int(out.dtype == torch.float32), _stream(stream))
+    if rc != 0:
+        raise FastOCRError(rc, lib.fastocr_noalloc_last_error().decode())
+
+
 def fastocr_decode_step(ctx: Context, layers: Sequence[KVView], q: torch.Tensor, out: torch.Tensor,
                         is_focal: Sequence[bool], k: torch.Tensor, fixation: torch.Tensor, has_fixation: bool,
                         max_vis_len: int, max_kept: int = 0, stream=None) -> bool:

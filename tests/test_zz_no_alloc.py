@@ -1,0 +1,51 @@
+"""The allocation-free entry point (for callers that cannot call cudaMalloc: engines that own all of
+HBM, allocator-tracked frameworks) must give the same result as the context-based one. Collected
+last on purpose: a run that stops at the first failure has then already run every other test."""
+import pytest
+import torch
+
+from harness import make_case
+
+pytestmark = pytest.mark.gpu
+
+
+def _inputs(seed, spans, paged):
+    import oracle
+    case = make_case(seed, spans, page_size=16 if paged else 0)
+    kv = case.device_view()
+    g = torch.Generator().manual_seed(seed)
+    ks = [oracle.kept_count(n, 0.05) for n in case.vis_len]
+    idx = torch.zeros(case.B, max(max(ks), 1), dtype=torch.int32)
+    for b in range(case.B):
+        idx[b, :ks[b]] = torch.randperm(case.vis_len[b], generator=g)[:ks[b]].sort().values.int()
+    return case, kv, case.q.cuda(), idx.cuda(), torch.tensor(ks, dtype=torch.int32, device="cuda")
+
+
+def test_noalloc_matches_context_entry_point_twice_in_a_row():
+    import paper_2605_17447_b200 as fo
+    ctx = fo.Context(max_batch=8, num_q_heads=28, num_kv_heads=4, max_seq_len=8192, max_vis_len=4096)
+    # two different problems back to back: the second call finds the first one's leftovers in the scratch
+    for call, (seed, spans, paged) in enumerate(((901, [(16, 2500, 77), (16, 4097, 130)], False),
+                                                 (902, [(3, 700, 40), (9, 90, 5), (0, 333, 0)], True))):
+        case, kv, q, idx, kd = _inputs(seed, spans, paged)
+        ref = torch.empty(case.B, case.H, 128, dtype=torch.float32, device="cuda")
+        got = torch.full_like(ref, float("nan"))
+        fo.fastocr_sparse_decode_attn(ctx, kv, q, idx, kd, ref)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        fo.fastocr_sparse_decode_attn_noalloc(kv, q, idx, kd, got)
+        torch.cuda.synchronize()
+        if call == 1:        # once every kernel involved has been loaded, the driver's free memory must not shrink
+            assert torch.cuda.mem_get_info()[0] >= free_before
+        err = (got - ref).abs()
+        assert err.max() <= 1e-4 and err.mean() <= 1e-3, float(err.max())     # same tolerance as the parity tests
+    ctx.close()
+
+
+def test_noalloc_rejects_oversized_batches():
+    import paper_2605_17447_b200 as fo
+    case, kv, q, idx, kd = _inputs(903, [(4, 64, 4)], False)
+    kv.seq_len = torch.zeros(65, dtype=torch.int32, device="cuda")   # 65 sequences x 4 KV heads > 256 units
+    with pytest.raises(fo.FastOCRError) as e:
+        fo.fastocr_sparse_decode_attn_noalloc(kv, q, idx, kd, torch.empty(65, 28, 128, device="cuda"))
+    assert e.value.code == 3 and "256" in str(e.value)
