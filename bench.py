@@ -356,12 +356,17 @@ def main():
         dense_step(t)
     ms_dense = timed(dense_step, dense_steps, barrier) / dense_steps
 
-    # per-kernel average durations over the same steps (events around every launch)
+    # per-kernel average durations over the same steps, from CUDA events the library records on the
+    # launching stream: "in_situ" times each maximal run of same-kernel launches as one interval (the
+    # launches overlap exactly as in the timed region), "isolated" brackets every launch on its own
     prof_steps = min(args.steps, 50)
-    w.ctx.profile_begin(prof_steps * (w.L * 2 + 8))
-    for t in range(prof_steps):
-        fastocr_step(t)
-    prof = w.ctx.profile_end()
+    profs = {}
+    for mode, coalesce in (("in_situ", True), ("isolated", False)):
+        w.ctx.profile_begin(prof_steps * (w.L * 2 + 8), coalesce_runs=coalesce)
+        for t in range(prof_steps):
+            fastocr_step(t)
+        profs[mode] = w.ctx.profile_end()
+    prof = profs["in_situ"]
 
     if dist:
         tt = torch.tensor([ms, ms_dense], device=dev, dtype=torch.float64)
@@ -379,13 +384,18 @@ def main():
         tot, n = prof[name]
         if n:
             us = tot / n * 1e3
-            kern[name] = {"us_per_launch": us, "launches_per_step": n / prof_steps, "algorithmic_bytes": bytes_per,
+            iso_tot, iso_n = profs["isolated"][name]
+            kern[name] = {"us_per_launch": us, "us_per_launch_isolated": iso_tot / max(iso_n, 1) * 1e3,
+                          "launches_per_step": n / prof_steps, "algorithmic_bytes": bytes_per,
                           "gbs": bytes_per / us / 1e3, "frac_of_measured": bytes_per / us / 1e3 / peak,
                           "frac_of_8tbs": bytes_per / us / 1e3 / NOMINAL_HBM_GBS}
     for name in ("scores_finalize", "select_topk"):
         tot, n = prof[name]
         if n:
             kern[name] = {"us_per_launch": tot / n * 1e3, "launches_per_step": n / prof_steps}
+    total_prof = sum(v[0] for v in prof.values()) or 1.0
+    for name in kern:
+        kern[name]["share_of_step"] = prof[name][0] / total_prof
     share = {name: prof[name][0] for name in prof if prof[name][1]}
     dominant = max(("attn_sparse", "attn_dense"), key=lambda n: share.get(n, 0.0))
     traffic = None
@@ -394,7 +404,8 @@ def main():
         traffic = json.load(open(tpath)).get(dominant, {}).get("traffic_bytes_per_launch")
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kern[dominant]["gbs"], "peak": peak, "unit": "GB/s",
                 "frac": kern[dominant]["frac_of_measured"], "peak_kind": f"of {peak_kind}", "traffic": traffic,
-                "frac_of_8tbs": kern[dominant]["frac_of_8tbs"]}
+                "frac_of_8tbs": kern[dominant]["frac_of_8tbs"],
+                "timing": "CUDA events on the launching stream around each run of consecutive launches of this kernel, / launches"}
 
     # ---- end to end: per step, pinned-host queries + the new token's K/V rows in, outputs back ----
     e2e = None

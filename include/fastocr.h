@@ -207,11 +207,16 @@ const char* fastocr_noalloc_last_error(void);
 
 /*
  * Optional per-kernel timing (the paper has no counterpart; measurement aid). Between
- * fastocr_profile_begin and fastocr_profile_end every launch of this context is bracketed by CUDA
- * events on its stream. fastocr_profile_begin creates `max_launches` event pairs (not a hot-path
- * call; launches beyond that are not timed); fastocr_profile_end synchronises, adds up elapsed
- * milliseconds and launch counts per kernel class into the two host arrays of length
- * FASTOCR_PROF_CLASSES, and destroys the events. Do not use while a stream is being captured.
+ * fastocr_profile_begin and fastocr_profile_end the launches of this context are bracketed by CUDA
+ * events on their stream. With coalesce_runs == 0 every launch gets its own event pair: the figures
+ * are isolated-kernel times (the event records keep consecutive layers from overlapping and the
+ * interval includes launch latency). With coalesce_runs != 0 a maximal run of consecutive launches
+ * of the same class shares one pair, nothing is recorded inside the run, and total time / launches
+ * is the duration per launch as it occurs in an unprofiled step. fastocr_profile_begin creates
+ * `max_launches` event pairs (not a hot-path call; launches beyond that are not timed);
+ * fastocr_profile_end synchronises, adds up elapsed milliseconds and launch counts per kernel class
+ * into the two host arrays of length FASTOCR_PROF_CLASSES, and destroys the events. Use one stream
+ * between begin and end, and not while a stream is being captured.
  */
 enum {
   FASTOCR_PROF_ATTN_DENSE = 0,  /* split-KV attention kernel, full cache, K and V          */
@@ -222,7 +227,7 @@ enum {
   FASTOCR_PROF_MASS = 5,        /* image-mass reduction                                     */
   FASTOCR_PROF_CLASSES = 6
 };
-fastocr_status fastocr_profile_begin(fastocr_ctx* ctx, int32_t max_launches);
+fastocr_status fastocr_profile_begin(fastocr_ctx* ctx, int32_t max_launches, int coalesce_runs);
 fastocr_status fastocr_profile_end(fastocr_ctx* ctx, double* ms_per_class, int64_t* launches_per_class);
 
 /* Number of kernels this library has launched on any context since load (for bench accounting). */

@@ -48,7 +48,7 @@ EXPORTS = {
     "fastocr_sparse_decode_attn_noalloc": (C.c_int, [C.POINTER(KVViewStruct), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                                      C.c_void_p, C.c_int, C.c_void_p]),
     "fastocr_noalloc_last_error": (C.c_char_p, []),
-    "fastocr_profile_begin": (C.c_int, [C.c_void_p, C.c_int32]),
+    "fastocr_profile_begin": (C.c_int, [C.c_void_p, C.c_int32, C.c_int]),
     "fastocr_profile_end": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "fastocr_launch_count": (C.c_int64, []),
 }

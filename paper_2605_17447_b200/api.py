@@ -121,8 +121,10 @@ class Context:
     def device_faults(self) -> int:
         return int(self._lib.fastocr_device_faults(self._h))
 
-    def profile_begin(self, max_launches: int) -> None:
-        self.check(self._lib.fastocr_profile_begin(self._h, int(max_launches)))
+    def profile_begin(self, max_launches: int, coalesce_runs: bool = False) -> None:
+        """coalesce_runs: time maximal runs of same-class launches as one interval (in-situ durations)
+        instead of every launch on its own (isolated durations)."""
+        self.check(self._lib.fastocr_profile_begin(self._h, int(max_launches), int(bool(coalesce_runs))))
 
     def profile_end(self):
         """-> {class name: (total ms, launches)} for the launches since profile_begin."""

@@ -39,8 +39,12 @@ struct fastocr_ctx {
   // optional per-launch timing
   std::vector<cudaEvent_t> prof_ev;   // 2 per timed launch
   std::vector<int> prof_class;
+  std::vector<int64_t> prof_count;    // launches covered by each pair
   size_t prof_used = 0;
   bool prof_on = false;
+  bool prof_runs = false;             // one pair per run of same-class launches
+  bool prof_open = false;
+  cudaStream_t prof_stream = nullptr;
 };
 
 namespace {
@@ -126,15 +130,35 @@ fastocr_status cuda_fail(fastocr_ctx* ctx, cudaError_t e, const char* what) {
   return fail(ctx, FASTOCR_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
-// Brackets one launch with events when profiling is on.
+// Brackets launches with events when profiling is on. In per-launch mode every launch gets its own
+// event pair (the records between kernels keep consecutive layers from overlapping, so the figures
+// are isolated-kernel times including launch latency). In run mode a maximal run of consecutive
+// launches of the same class shares one pair: nothing is recorded between them, so they overlap
+// exactly as in an unprofiled step, and total time / launches is the in-situ duration.
 struct ProfScope {
   fastocr_ctx* ctx;
   cudaStream_t s;
   bool armed = false;
   ProfScope(fastocr_ctx* c, int cls, cudaStream_t st) : ctx(c), s(st) {
-    if (c->prof_on && c->prof_used + 2 <= c->prof_ev.size()) {
+    if (!c->prof_on) return;
+    if (c->prof_runs) {
+      if (c->prof_open && c->prof_class.back() == cls) {       // the run goes on
+        c->prof_count.back() += 1;
+        return;
+      }
+      close_run(c, st);
+      if (c->prof_used + 2 > c->prof_ev.size()) return;
+      c->prof_class.push_back(cls);
+      c->prof_count.push_back(1);
+      cudaEventRecord(c->prof_ev[c->prof_used], st);
+      c->prof_open = true;
+      c->prof_stream = st;
+      return;
+    }
+    if (c->prof_used + 2 <= c->prof_ev.size()) {
       armed = true;
       c->prof_class.push_back(cls);
+      c->prof_count.push_back(1);
       cudaEventRecord(c->prof_ev[c->prof_used], st);
     }
   }
@@ -143,6 +167,12 @@ struct ProfScope {
       cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s);
       ctx->prof_used += 2;
     }
+  }
+  static void close_run(fastocr_ctx* c, cudaStream_t st) {
+    if (!c->prof_open) return;
+    cudaEventRecord(c->prof_ev[c->prof_used + 1], st);
+    c->prof_used += 2;
+    c->prof_open = false;
   }
 };
 
@@ -386,7 +416,7 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
       // queries, index set and cache were all complete before), so the two may overlap
       st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, prev_was_pruned, s);
       if (st != FASTOCR_OK) return st;
-      prev_was_pruned = !ctx->prof_on;
+      prev_was_pruned = !ctx->prof_on || ctx->prof_runs;
     }
   }
   if (has_fixation_out != nullptr) *has_fixation_out = have ? 1 : 0;
@@ -422,7 +452,7 @@ double fastocr_attn_flops(double batch, double layers, double hidden, double seq
   return batch * layers * (8.0 * hidden * hidden + 4.0 * hidden * seq_len);
 }
 
-fastocr_status fastocr_profile_begin(fastocr_ctx* ctx, int32_t max_launches) {
+fastocr_status fastocr_profile_begin(fastocr_ctx* ctx, int32_t max_launches, int coalesce_runs) {
   if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
   if (max_launches <= 0 || ctx->prof_on) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "profile_begin: bad size or already profiling");
   cudaSetDevice(ctx->device);
@@ -430,7 +460,11 @@ fastocr_status fastocr_profile_begin(fastocr_ctx* ctx, int32_t max_launches) {
   for (auto& ev : ctx->prof_ev) FASTOCR_TRY_CUDA(cudaEventCreate(&ev), "cudaEventCreate");
   ctx->prof_class.clear();
   ctx->prof_class.reserve(max_launches);
+  ctx->prof_count.clear();
+  ctx->prof_count.reserve(max_launches);
   ctx->prof_used = 0;
+  ctx->prof_runs = coalesce_runs != 0;
+  ctx->prof_open = false;
   ctx->prof_on = true;
   return FASTOCR_OK;
 }
@@ -439,6 +473,7 @@ fastocr_status fastocr_profile_end(fastocr_ctx* ctx, double* ms_per_class, int64
   if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
   if (!ctx->prof_on || ms_per_class == nullptr || launches_per_class == nullptr)
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "profile_end: not profiling or NULL output");
+  ProfScope::close_run(ctx, ctx->prof_stream);
   ctx->prof_on = false;
   for (int c = 0; c < FASTOCR_PROF_CLASSES; ++c) {
     ms_per_class[c] = 0.0;
@@ -449,11 +484,12 @@ fastocr_status fastocr_profile_end(fastocr_ctx* ctx, double* ms_per_class, int64
     float ms = 0.f;
     e = cudaEventElapsedTime(&ms, ctx->prof_ev[i], ctx->prof_ev[i + 1]);
     ms_per_class[ctx->prof_class[i / 2]] += ms;
-    launches_per_class[ctx->prof_class[i / 2]] += 1;
+    launches_per_class[ctx->prof_class[i / 2]] += ctx->prof_count[i / 2];
   }
   for (auto ev : ctx->prof_ev) cudaEventDestroy(ev);
   ctx->prof_ev.clear();
   ctx->prof_class.clear();
+  ctx->prof_count.clear();
   ctx->prof_used = 0;
   if (e != cudaSuccess) return cuda_fail(ctx, e, "profile_end");
   return FASTOCR_OK;

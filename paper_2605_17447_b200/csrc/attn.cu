@@ -5,8 +5,9 @@
 // Work decomposition (stream-K over tokens). A unit is one (sequence, KV head) pair; its attended
 // tokens are cut into rows of 64 (one 16-token block per warp of a CTA). All rows of the launch
 // are laid end to end and divided into equal ranges, one per persistent CTA (two CTAs of four warps
-// per SM); when there are no more units than CTAs the number of active CTAs is rounded down to a
-// multiple of the unit count, so that equal-sized units are never shared between CTAs. Every CTA
+// per SM); when there are no more units than CTAs and the ranges are short, the number of active
+// CTAs is rounded down to a multiple of the unit count, so that equal-sized units are never shared
+// between CTAs. Every CTA
 // therefore streams the same number of rows, pays one pipeline prologue per launch and exits
 // without waiting for anyone. When a CTA's range leaves a unit, its four warps merge their
 // running (max, sum, output) through a 4 KB shared-memory buffer; a unit wholly inside the range is
@@ -50,6 +51,7 @@ constexpr int kBlockTokens = 16;                        // tokens per warp per p
 constexpr int kRowTokens = kAttnWarps * kBlockTokens;   // tokens per CTA per pipeline stage
 constexpr float kRescaleSlack = 8.0f;                   // log2 units
 constexpr int kMergeRound = 4;                          // partials fetched together by the merging CTA
+constexpr int kLongRangeRows = 32;                      // rows per CTA from which unit alignment is dropped
 
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -191,7 +193,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
   FASTOCR_TRACE_MARK(1);
   const int total_rows = prefix_s[units];
   const int grid = gridDim.x;
-  const int active = units <= grid ? units * (grid / units) : grid;
+  // short ranges: keep equal-sized units whole (no shared units, no global merge); long ranges:
+  // use every CTA, the few merges are negligible against the stream
+  const int active = (units <= grid && total_rows < kLongRangeRows * grid) ? units * (grid / units) : grid;
   const int per_cta = (total_rows + active - 1) / active;
   const int r0 = blockIdx.x * per_cta;
   const int r1 = min(total_rows, r0 + per_cta);
