@@ -120,7 +120,7 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
 #else
   a.trace = nullptr;
 #endif
-  a.wait_at_start = 1;
+  a.wait_point = fastocr::kWaitAtStart;
   a.grid_ctas = ctx->sm_count * ctx->ctas_per_sm;
   (void)max_len;
   return a;
@@ -184,7 +184,7 @@ struct ProfScope {
 
 // dense pass (+ optional fused scoring) without re-validating the view
 fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, void* out, int out_is_fp32,
-                          float* scores_out, int32_t n_stride, int32_t max_vis, cudaStream_t s) {
+                          float* scores_out, int32_t n_stride, int32_t max_vis, int wait_point, cudaStream_t s) {
   AttnLaunch a = make_launch(ctx, kv, q, /*with_v=*/out != nullptr, kv->max_seq_len);
   const bool want_scores = scores_out != nullptr;
   if (want_scores) {
@@ -193,6 +193,7 @@ fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
   }
   a.out = out;
   a.out_is_fp32 = out_is_fp32;
+  a.wait_point = wait_point;
   a.stats = want_scores ? ctx->stats : nullptr;
   {
     ProfScope p(ctx, out != nullptr ? FASTOCR_PROF_ATTN_DENSE : FASTOCR_PROF_ATTN_KEYS, s);
@@ -207,17 +208,17 @@ fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
   return FASTOCR_OK;
 }
 
-// inputs_settled: nothing this launch reads (lengths, index list, queries, cache) was written by
-// the launch issued just before it on the stream, so it may start while that one drains.
+// wait_point: how much of this launch may run while earlier kernels of the stream are still
+// draining (fastocr::kWait...), i.e. which of its inputs could have been written just before.
 fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, const int32_t* idx,
                            const int32_t* k, int32_t k_stride, int32_t max_kept, void* out, int out_is_fp32,
-                           bool inputs_settled, cudaStream_t s) {
+                           int wait_point, cudaStream_t s) {
   const int max_len = (max_kept > 0 && max_kept < kv->max_seq_len) ? max_kept : kv->max_seq_len;
   AttnLaunch a = make_launch(ctx, kv, q, true, max_len);
   a.idx = idx;
   a.kcount = k;
   a.k_stride = k_stride;
-  a.wait_at_start = inputs_settled ? 0 : 1;
+  a.wait_point = wait_point;
   a.out = out;
   a.out_is_fp32 = out_is_fp32;
   {
@@ -325,7 +326,7 @@ fastocr_status fastocr_dense_decode_attn(fastocr_ctx* ctx, const fastocr_kv_view
     max_vis = n_stride < ctx->lim.max_vis_len ? n_stride : ctx->lim.max_vis_len;
     if (ctx->lim.max_vis_len <= 0) return fail(ctx, FASTOCR_ERR_WORKSPACE, "context was created with max_vis_len = 0");
   }
-  return dense_impl(ctx, kv, q, out, out_is_fp32, scores_out, n_stride, max_vis, static_cast<cudaStream_t>(stream));
+  return dense_impl(ctx, kv, q, out, out_is_fp32, scores_out, n_stride, max_vis, fastocr::kWaitAtStart, static_cast<cudaStream_t>(stream));
 }
 
 fastocr_status fastocr_focal_scores(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, float* scores_out,
@@ -336,7 +337,7 @@ fastocr_status fastocr_focal_scores(fastocr_ctx* ctx, const fastocr_kv_view* kv,
   if (ctx->lim.max_vis_len <= 0) return fail(ctx, FASTOCR_ERR_WORKSPACE, "context was created with max_vis_len = 0");
   const int32_t max_vis = n_stride < ctx->lim.max_vis_len ? n_stride : ctx->lim.max_vis_len;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  st = dense_impl(ctx, kv, q, nullptr, 0, scores_out, n_stride, max_vis, s);
+  st = dense_impl(ctx, kv, q, nullptr, 0, scores_out, n_stride, max_vis, fastocr::kWaitAtStart, s);
   if (st != FASTOCR_OK) return st;
   if (image_mass_out != nullptr) {
     ProfScope p(ctx, FASTOCR_PROF_MASS, s);
@@ -369,7 +370,7 @@ fastocr_status fastocr_sparse_decode_attn(fastocr_ctx* ctx, const fastocr_kv_vie
   if (st != FASTOCR_OK) return st;
   if (idx == nullptr || k == nullptr || out == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL idx, k or out");
   if (k_stride <= 0 || max_kept < 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "k_stride must be positive, max_kept non-negative");
-  return sparse_impl(ctx, kv, q, idx, k, k_stride, max_kept, out, out_is_fp32, false, static_cast<cudaStream_t>(stream));
+  return sparse_impl(ctx, kv, q, idx, k, k_stride, max_kept, out, out_is_fp32, fastocr::kWaitAtStart, static_cast<cudaStream_t>(stream));
 }
 
 fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
@@ -393,15 +394,21 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
   const int64_t per_layer = static_cast<int64_t>(layers[0].batch) * layers[0].num_q_heads * fastocr::kHeadDim;
   const size_t q_bytes = per_layer * 2, o_bytes = per_layer * (out_is_fp32 ? 4 : 2);
   bool have = has_fixation != 0;
-  bool prev_was_pruned = false;   // the launch just before was a pruned-attention kernel of this step
+  // What the launch issued just before the next one was: nothing of this step yet, a pruned or
+  // dense attention kernel of this step (it wrote an output slice and the split workspace, neither
+  // of which the next attention kernel reads), or the selection kernel (it wrote the index set).
+  enum { kOther, kAttention, kSelection } prev = kOther;
   for (int l = 0; l < num_layers; ++l) {
     const void* ql = static_cast<const char*>(q) + l * q_bytes;
     void* ol = static_cast<char*>(out) + l * o_bytes;
     const bool focal = is_focal[l] != 0;
+    const bool chained = prev != kOther && (!ctx->prof_on || ctx->prof_runs);
     fastocr_status st;
     if (focal || (l == 0 && !have)) {
-      // full attention + scoring + selection; the refreshed set replaces the current one
-      st = dense_impl(ctx, &layers[l], ql, ol, out_is_fp32, ctx->scores, ctx->lim.max_vis_len, max_vis_len, s);
+      // full attention + scoring + selection; the refreshed set replaces the current one.
+      // The logits workspace is written from the first block on: wait before the stream starts.
+      st = dense_impl(ctx, &layers[l], ql, ol, out_is_fp32, ctx->scores, ctx->lim.max_vis_len, max_vis_len,
+                      chained ? fastocr::kWaitAfterSetup : fastocr::kWaitAtStart, s);
       if (st != FASTOCR_OK) return st;
       {
         ProfScope p(ctx, FASTOCR_PROF_TOPK, s);
@@ -410,13 +417,15 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
                          "top-k launch");
       }
       have = true;
-      prev_was_pruned = false;
+      prev = kSelection;
     } else {
-      // a pruned layer that follows another pruned layer reads nothing the latter wrote (its
-      // queries, index set and cache were all complete before), so the two may overlap
-      st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, prev_was_pruned, s);
+      // a pruned layer that follows another attention layer reads nothing the latter wrote (its
+      // queries, index set and cache were complete before), so the two may overlap; right after
+      // a selection only the set-up (lengths, kept counts) may run ahead
+      const int wp = !chained ? fastocr::kWaitAtStart : (prev == kAttention ? fastocr::kWaitBeforeWrites : fastocr::kWaitAfterSetup);
+      st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, wp, s);
       if (st != FASTOCR_OK) return st;
-      prev_was_pruned = !ctx->prof_on || ctx->prof_runs;
+      prev = kAttention;
     }
   }
   if (has_fixation_out != nullptr) *has_fixation_out = have ? 1 : 0;

@@ -84,17 +84,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// Programmatic dependent launch: a launch of this kernel may begin while the previous kernel in the
-// stream is still draining. dependents_may_launch() lets the next kernel's CTAs be scheduled as
-// soon as resources free up; wait_for_prior_grids() blocks until every earlier kernel has finished
-// and its writes are visible (a no-op when the launch carried no such attribute).
-#ifdef FASTOCR_NO_LAUNCH_DEPENDENTS
-__device__ __forceinline__ void dependents_may_launch() {}
-#else
-__device__ __forceinline__ void dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
-#endif
-__device__ __forceinline__ void wait_for_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 // two adjacent outputs (even index), bf16 or fp32
 __device__ __forceinline__ void store_pair(void* out, int is_fp32, int64_t index, float x, float y) {
   if (is_fp32) *reinterpret_cast<float2*>(reinterpret_cast<float*>(out) + index) = make_float2(x, y);
@@ -161,9 +150,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
   const int units = a.batch * Hkv;                     // unit u = (sequence u / Hkv, KV head u % Hkv)
 
   FASTOCR_TRACE_MARK(0);
-  // Everything read before the first wait_for_prior_grids() (lengths, index list, queries, cache)
-  // must not have been produced by the kernel launched just before this one; the host says so.
-  if (a.wait_at_start) wait_for_prior_grids();
+  // Everything read before the first wait_for_prior_grids() must not have been produced by a
+  // kernel that may still be running; the host says how much that is (AttnLaunch::wait_point).
+  if (a.wait_point == kWaitAtStart) wait_for_prior_grids();
   dependents_may_launch();
 
   // ---- set-up: prefix of 64-token rows over units (warp 0) -------------------------------------
@@ -220,6 +209,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
     u = lo;
   }
   int seg_begin = r0;
+  if (a.wait_point == kWaitAfterSetup) wait_for_prior_grids();   // before index-list reads and logits writes
 #pragma unroll 1
   while (per_cta > 0 && seg_begin < r1) {
     while (prefix_s[u + 1] <= seg_begin) ++u;          // skip empty units
@@ -552,6 +542,8 @@ __global__ void __launch_bounds__(kFinalizeThreads) scores_finalize_kernel(
     const float* __restrict__ logits, const float* __restrict__ stats, const int32_t* __restrict__ vis_len,
     int num_q_heads, int n_stride_logits, float* __restrict__ scores, int n_stride) {
   extern __shared__ float st[];                        // [H][2]: max, 1/sum
+  wait_for_prior_grids();
+  dependents_may_launch();
   const int b = blockIdx.y;
   const int N = vis_len[b];
   for (int i = threadIdx.x; i < num_q_heads; i += blockDim.x) {
@@ -563,13 +555,23 @@ __global__ void __launch_bounds__(kFinalizeThreads) scores_finalize_kernel(
   if (i >= N || i >= n_stride || i >= n_stride_logits) return;
   const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + i;
   float s = 0.f;
-  for (int h = 0; h < num_q_heads; ++h) s += exp2f(lp[static_cast<int64_t>(h) * n_stride_logits] - st[2 * h]) * st[2 * h + 1];
+  int h = 0;
+  for (; h + 4 <= num_q_heads; h += 4) {               // four loads in flight; summed in head order
+    float x[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) x[j] = lp[static_cast<int64_t>(h + j) * n_stride_logits];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) s += exp2f(x[j] - st[2 * (h + j)]) * st[2 * (h + j) + 1];
+  }
+  for (; h < num_q_heads; ++h) s += exp2f(lp[static_cast<int64_t>(h) * n_stride_logits] - st[2 * h]) * st[2 * h + 1];
   scores[static_cast<int64_t>(b) * n_stride + i] = s / static_cast<float>(num_q_heads);
 }
 
 __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restrict__ scores, int n_stride,
                                                           const int32_t* __restrict__ vis_len, float* __restrict__ mass) {
   __shared__ float red[32];
+  wait_for_prior_grids();
+  dependents_may_launch();
   const int b = blockIdx.x, N = vis_len[b];
   float s = 0.f;
   for (int i = threadIdx.x; i < N; i += blockDim.x) s += scores[static_cast<int64_t>(b) * n_stride + i];
@@ -587,17 +589,7 @@ __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restric
 
 template <int G, bool HAS_V>
 cudaError_t launch_partial_t(const AttnLaunch& a, cudaStream_t s) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(a.grid_ctas);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = Smem<HAS_V>::total;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, attn_stream_kernel<G, HAS_V>, a);
+  const cudaError_t e = launch_pdl(attn_stream_kernel<G, HAS_V>, dim3(a.grid_ctas), dim3(kThreads), Smem<HAS_V>::total, s, a);
   count_launches(1);
   return e;
 }
@@ -645,17 +637,17 @@ cudaError_t launch_scores_finalize(const float* logits, const float* stats, cons
                                    int32_t n_stride, cudaStream_t s) {
   if (max_vis_len <= 0) return cudaSuccess;
   dim3 grid((max_vis_len + kFinalizeThreads - 1) / kFinalizeThreads, batch);
-  scores_finalize_kernel<<<grid, kFinalizeThreads, num_q_heads * 2 * sizeof(float), s>>>(
-      logits, stats, vis_len, num_q_heads, n_stride_logits, scores, n_stride);
+  const cudaError_t e = launch_pdl(scores_finalize_kernel, grid, dim3(kFinalizeThreads), num_q_heads * 2 * sizeof(float), s,
+                                   logits, stats, vis_len, num_q_heads, n_stride_logits, scores, n_stride);
   count_launches(1);
-  return cudaGetLastError();
+  return e;
 }
 
 cudaError_t launch_image_mass(const float* scores, int32_t n_stride, const int32_t* vis_len, int32_t batch, float* mass,
                               cudaStream_t s) {
-  image_mass_kernel<<<batch, 1024, 0, s>>>(scores, n_stride, vis_len, mass);
+  const cudaError_t e = launch_pdl(image_mass_kernel, dim3(batch), dim3(1024), 0, s, scores, n_stride, vis_len, mass);
   count_launches(1);
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace fastocr

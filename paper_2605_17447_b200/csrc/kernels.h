@@ -11,6 +11,37 @@ constexpr int kAttnWarps = 4;         // autonomous warps per persistent attenti
 constexpr int kMaxUnits = 1024;       // sequences x KV heads per launch (their row prefix lives in shared memory)
 constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
 
+// Programmatic dependent launch. Every kernel of this library is launched with the "programmatic
+// stream serialization" attribute and (i) lets its successor's CTAs be scheduled as soon as SM
+// resources free up (dependents_may_launch), (ii) calls wait_for_prior_grids() before it touches
+// anything an earlier kernel may have written or may still be reading; the wait returns when all
+// earlier kernels in the stream have completed and their writes are visible. A predecessor that is
+// not one of these kernels never triggers early, so ordinary stream order applies to it.
+#ifdef __CUDACC__
+__device__ __forceinline__ void dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void wait_for_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
+// AttnLaunch::wait_point
+constexpr int kWaitBeforeWrites = 0;  // inputs settled long ago: wait only before results / shared workspace are written
+constexpr int kWaitAtStart = 1;       // anything may have just been written: wait first
+constexpr int kWaitAfterSetup = 2;    // lengths and kept counts are settled, index list / logits workspace are not
+
 struct AttnLaunch {
   // cache view
   const void* k;
@@ -30,7 +61,7 @@ struct AttnLaunch {
   const int32_t* kcount;
   int32_t k_stride;
   int32_t grid_ctas;          // persistent CTAs (kAttnWarps warps each)
-  int32_t wait_at_start;      // 0: no input of this launch was written by the launch just before it
+  int32_t wait_point;         // where the kernel waits for earlier kernels: kWaitAtStart / kWaitAfterSetup / kWaitBeforeWrites
   // workspace
   float* part_acc;            // [slots][8][128], slot = CTA index + unit index (unit = sequence * Hkv + KV head)
   float* part_ml;             // [slots][8][2]  (max, sum) in the log2 domain

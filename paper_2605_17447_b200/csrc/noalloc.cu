@@ -123,7 +123,7 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   a.kcount = k;
   a.k_stride = k_stride;
   a.grid_ctas = grid;
-  a.wait_at_start = 1;
+  a.wait_point = fastocr::kWaitAtStart;
   a.part_acc = reinterpret_cast<float*>(s.scratch);
   a.part_ml = reinterpret_cast<float*>(s.scratch + kAccBytes);
   a.counters = reinterpret_cast<int32_t*>(counters);

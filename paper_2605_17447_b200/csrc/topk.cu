@@ -31,6 +31,8 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   __shared__ uint32_t warp_gt[kTopkWarps], warp_eq[kTopkWarps];
   __shared__ uint32_t sel_prefix, sel_remaining;
 
+  wait_for_prior_grids();
+  dependents_may_launch();
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = min(vis_len[b], kTopkMaxN);
   int k = kreq[b];
@@ -57,12 +59,17 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
       const int i = base + lane;
       const uint32_t key = i < N ? keys[i] : 0u;
       const bool in = i < N && (key & hi_mask) == prefix;
-      // aggregate identical digits inside the warp before touching shared memory
       const uint32_t digit = (key >> shift) & 0xffu;
-      const uint32_t active = __ballot_sync(0xffffffffu, in);
-      if (in) {
-        const uint32_t peers = __match_any_sync(active, digit);
-        if ((__ffs(peers) - 1) == lane) atomicAdd(&hist[digit], __popc(peers));
+      if (pass == 0) {
+        // the leading byte (sign and most of the exponent) is heavily clustered: aggregate
+        // identical digits inside the warp before touching shared memory
+        const uint32_t active = __ballot_sync(0xffffffffu, in);
+        if (in) {
+          const uint32_t peers = __match_any_sync(active, digit);
+          if ((__ffs(peers) - 1) == lane) atomicAdd(&hist[digit], __popc(peers));
+        }
+      } else if (in) {                                 // later bytes are spread out and few keys are left
+        atomicAdd(&hist[digit], 1u);
       }
     }
     __syncthreads();
@@ -158,17 +165,20 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
 }  // namespace
 
 cudaError_t configure_topk() {
-  return cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkMaxN * 4);
+  cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkMaxN * 4);
+  if (e != cudaSuccess) return e;
+  // same shared-memory carve-out as the attention kernel: no reconfiguration between them
+  return cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
 }
 
 cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int32_t* vis_len, const int32_t* k,
                                int32_t batch, int32_t max_vis_len, int32_t* idx_out, int32_t k_stride,
                                cudaStream_t s) {
   if (batch <= 0 || max_vis_len <= 0) return cudaSuccess;
-  select_topk_kernel<<<batch, kTopkThreads, static_cast<size_t>(max_vis_len) * 4, s>>>(scores, n_stride, vis_len, k,
-                                                                                       idx_out, k_stride);
+  const cudaError_t e = launch_pdl(select_topk_kernel, dim3(batch), dim3(kTopkThreads), static_cast<size_t>(max_vis_len) * 4, s,
+                                   scores, n_stride, vis_len, k, idx_out, k_stride);
   count_launches(1);
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace fastocr
