@@ -1,18 +1,27 @@
 // TopK of Eq. 2: exact selection of the k best-scored image tokens of every sequence.
 //
-// One CTA per sequence. The scores are mapped to order-preserving 32-bit keys held in shared
-// memory (up to 32768 keys = 128 KB), the key of the k-th largest score is found with a four-pass
-// MSB-first radix select (8 bits per pass, 256-bin histogram in shared memory), and the result is
-// emitted by an in-order compaction: every key above the threshold, plus the first r keys equal to
-// it, where r is what is left of k. Walking the indices in ascending order gives both the
-// "lower index wins ties" rule and the ascending output order with no sort.
+// One thread-block cluster per sequence (1, 2, 4 or 8 CTAs, chosen so that a launch fills the GPU
+// even for small batches); CTA c of the cluster owns the contiguous slice c of the sequence's
+// scores. The scores are mapped to order-preserving 32-bit keys held in shared memory, the key of
+// the k-th largest score is found with a four-pass MSB-first radix select (8 bits per pass: every
+// CTA histograms its slice, the 256 bin totals are summed across the cluster through distributed
+// shared memory, and every CTA walks the same totals), and the result is emitted by an in-order
+// compaction: every key above the threshold, plus the first r keys equal to it, where r is what is
+// left of k. Walking the indices in ascending order gives both the "lower index wins ties" rule
+// and the ascending output order with no sort; a CTA learns how many selected keys precede its
+// slice from the other CTAs' totals.
 #include "kernels.h"
+
+#include <cooperative_groups.h>
+
+namespace cg = cooperative_groups;
 
 namespace fastocr {
 namespace {
 
 constexpr int kTopkThreads = 1024;
 constexpr int kTopkWarps = kTopkThreads / 32;
+constexpr int kTopkMaxCluster = 8;
 
 // larger float <=> larger key; -0 == +0; NaN below everything.
 __device__ __forceinline__ uint32_t score_key(float s) {
@@ -25,23 +34,32 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* __restrict__ scores, int n_stride,
                                                                    const int32_t* __restrict__ vis_len,
                                                                    const int32_t* __restrict__ kreq,
-                                                                   int32_t* __restrict__ idx_out, int k_stride) {
-  extern __shared__ uint32_t keys[];                    // [N]
-  __shared__ uint32_t hist[256];
+                                                                   int32_t* __restrict__ idx_out, int k_stride, int n_cap) {
+  extern __shared__ uint32_t keys[];                    // this CTA's slice of the keys
+  __shared__ uint32_t hist[256];                        // this CTA's histogram (read by the whole cluster)
+  __shared__ uint32_t hist_all[256];                    // cluster totals
   __shared__ uint32_t warp_gt[kTopkWarps], warp_eq[kTopkWarps];
+  __shared__ uint32_t slice_tot[2];                     // selected-candidate counts of this slice: above, equal
   __shared__ uint32_t sel_prefix, sel_remaining;
 
   wait_for_prior_grids();
   dependents_may_launch();
-  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int N = min(vis_len[b], kTopkMaxN);
+  cg::cluster_group cluster = cg::this_cluster();
+  const int C = static_cast<int>(cluster.num_blocks());
+  const int c = static_cast<int>(cluster.block_rank());
+  const int b = blockIdx.x / C, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int N = min(vis_len[b], n_cap);                 // n_cap: what the launch sized the key slices for
   int k = kreq[b];
   k = k < 0 ? 0 : (k > N ? N : k);
   k = min(k, k_stride);
-  if (k == 0) return;
+  if (k == 0) return;                                   // the same decision in every CTA of the cluster
 
-  const float* sp = scores + static_cast<int64_t>(b) * n_stride;
-  for (int i = tid; i < N; i += kTopkThreads) keys[i] = score_key(sp[i]);
+  // slice [lo_i, hi_i) of the sequence, a multiple of 32 keys per CTA
+  const int per_cta = (((N + C - 1) / C) + 31) & ~31;
+  const int lo_i = min(c * per_cta, N), hi_i = min(lo_i + per_cta, N);
+  const int n_loc = hi_i - lo_i;
+  const float* sp = scores + static_cast<int64_t>(b) * n_stride + lo_i;
+  for (int i = tid; i < n_loc; i += kTopkThreads) keys[i] = score_key(sp[i]);
   if (tid == 0) {
     sel_prefix = 0u;
     sel_remaining = static_cast<uint32_t>(k);
@@ -55,10 +73,10 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
     const uint32_t prefix = sel_prefix;
     const uint32_t remaining = sel_remaining;
     const uint32_t hi_mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-    for (int base = warp * 32; base < N; base += kTopkThreads) {     // warp-uniform trip count
+    for (int base = warp * 32; base < n_loc; base += kTopkThreads) {   // warp-uniform trip count
       const int i = base + lane;
-      const uint32_t key = i < N ? keys[i] : 0u;
-      const bool in = i < N && (key & hi_mask) == prefix;
+      const uint32_t key = i < n_loc ? keys[i] : 0u;
+      const bool in = i < n_loc && (key & hi_mask) == prefix;
       const uint32_t digit = (key >> shift) & 0xffu;
       if (pass == 0) {
         // the leading byte (sign and most of the exponent) is heavily clustered: aggregate
@@ -68,19 +86,25 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
           const uint32_t peers = __match_any_sync(active, digit);
           if ((__ffs(peers) - 1) == lane) atomicAdd(&hist[digit], __popc(peers));
         }
-      } else if (in) {                                 // later bytes are spread out and few keys are left
+      } else if (in) {                                  // later bytes are spread out and few keys are left
         atomicAdd(&hist[digit], 1u);
       }
     }
-    __syncthreads();
+    cluster.sync();                                     // every slice's histogram is complete
+    if (tid < 256) {
+      uint32_t t = 0;
+      for (int r = 0; r < C; ++r) t += *cluster.map_shared_rank(&hist[tid], r);
+      hist_all[tid] = t;
+    }
+    cluster.sync();                                     // totals read: the histograms may be cleared again
     // one warp walks the bins from the top: find the digit where the running count reaches k
     if (warp == 0) {
-      uint32_t above = 0;                              // keys with a larger digit
+      uint32_t above = 0;                               // keys with a larger digit
       uint32_t found_digit = 0, found_above = 0;
       bool found = false;
       for (int base = 224; base >= 0 && !found; base -= 32) {
-        const uint32_t cnt = hist[base + (31 - lane)]; // lane 0 holds the largest digit of the group
-        uint32_t incl = cnt;                           // inclusive scan, largest digit first
+        const uint32_t cnt = hist_all[base + (31 - lane)];   // lane 0 holds the largest digit of the group
+        uint32_t incl = cnt;                            // inclusive scan, largest digit first
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
           const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
@@ -108,8 +132,8 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   const uint32_t take_eq = sel_remaining;               // how many keys equal to thr are selected
 
   // ---- in-order compaction --------------------------------------------------------------------
-  const int per = (N + kTopkThreads - 1) / kTopkThreads;
-  const int lo = min(tid * per, N), hi = min(lo + per, N);
+  const int per = (n_loc + kTopkThreads - 1) / kTopkThreads;
+  const int lo = min(tid * per, n_loc), hi = min(lo + per, n_loc);
   uint32_t gt = 0, eq = 0;
   for (int i = lo; i < hi; ++i) {
     const uint32_t key = keys[i];
@@ -120,10 +144,10 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const uint32_t a = __shfl_up_sync(0xffffffffu, gt_incl, o);
-    const uint32_t c = __shfl_up_sync(0xffffffffu, eq_incl, o);
+    const uint32_t e = __shfl_up_sync(0xffffffffu, eq_incl, o);
     if (lane >= o) {
       gt_incl += a;
-      eq_incl += c;
+      eq_incl += e;
     }
   }
   if (lane == 31) {
@@ -132,34 +156,44 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   }
   __syncthreads();
   if (warp == 0) {
-    uint32_t a = warp_gt[lane], c = warp_eq[lane];
-    uint32_t ai = a, ci = c;
+    uint32_t a = warp_gt[lane], e = warp_eq[lane];
+    uint32_t ai = a, ei = e;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const uint32_t ta = __shfl_up_sync(0xffffffffu, ai, o);
-      const uint32_t tc = __shfl_up_sync(0xffffffffu, ci, o);
+      const uint32_t te = __shfl_up_sync(0xffffffffu, ei, o);
       if (lane >= o) {
         ai += ta;
-        ci += tc;
+        ei += te;
       }
     }
-    warp_gt[lane] = ai - a;                            // exclusive
-    warp_eq[lane] = ci - c;
+    warp_gt[lane] = ai - a;                             // exclusive
+    warp_eq[lane] = ei - e;
+    if (lane == 31) {
+      slice_tot[0] = ai;
+      slice_tot[1] = ei;
+    }
   }
-  __syncthreads();
+  cluster.sync();                                       // also orders warp_gt / warp_eq inside the CTA
   uint32_t gt_before = warp_gt[warp] + gt_incl - gt;
   uint32_t eq_before = warp_eq[warp] + eq_incl - eq;
+  for (int r = 0; r < c; ++r) {                         // candidates in the slices before this one
+    const uint32_t* t = cluster.map_shared_rank(slice_tot, r);
+    gt_before += t[0];
+    eq_before += t[1];
+  }
   int32_t* op = idx_out + static_cast<int64_t>(b) * k_stride;
   for (int i = lo; i < hi; ++i) {
     const uint32_t key = keys[i];
     if (key > thr) {
-      op[gt_before + min(eq_before, take_eq)] = i;
+      op[gt_before + min(eq_before, take_eq)] = lo_i + i;
       ++gt_before;
     } else if (key == thr) {
-      if (eq_before < take_eq) op[gt_before + eq_before] = i;
+      if (eq_before < take_eq) op[gt_before + eq_before] = lo_i + i;
       ++eq_before;
     }
   }
+  cluster.sync();                                       // nobody leaves while its shared memory may still be read
 }
 
 }  // namespace
@@ -175,8 +209,28 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
                                int32_t batch, int32_t max_vis_len, int32_t* idx_out, int32_t k_stride,
                                cudaStream_t s) {
   if (batch <= 0 || max_vis_len <= 0) return cudaSuccess;
-  const cudaError_t e = launch_pdl(select_topk_kernel, dim3(batch), dim3(kTopkThreads), static_cast<size_t>(max_vis_len) * 4, s,
-                                   scores, n_stride, vis_len, k, idx_out, k_stride);
+  // cluster size: enough CTAs to cover the GPU for small batches, at least 1024 keys per CTA
+  int device = 0, sms = 148;
+  if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+  int C = 1;
+  while (C < kTopkMaxCluster && batch * C * 2 <= sms && max_vis_len / (C * 2) >= 1024) C *= 2;
+  const int per_cta = (((max_vis_len + C - 1) / C) + 31) & ~31;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(batch * C);
+  cfg.blockDim = dim3(kTopkThreads);
+  cfg.dynamicSmemBytes = static_cast<size_t>(per_cta) * 4;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = C;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, select_topk_kernel, scores, n_stride, vis_len, k, idx_out, k_stride,
+                                           static_cast<int>(max_vis_len));
   count_launches(1);
   return e;
 }
