@@ -187,7 +187,7 @@ double fastocr_attn_flops(double batch, double layers, double hidden, double seq
  * counterpart; this exists for callers that cannot call cudaMalloc: engines that give all of HBM
  * to their own pool at start-up, allocator-tracked frameworks, decode loops that must stay out of
  * the driver's allocator). Same computation and arguments as fastocr_sparse_decode_attn, but the
- * scratch of the split merge is a fixed array inside the library (about 2.7 MB of device memory
+ * scratch of the split merge is a fixed array inside the library (about 3.1 MB of device memory
  * on every GPU that loads it, held until the process exits) instead of a context's workspace.
  *   - Limit: batch * num_kv_heads <= FASTOCR_NOALLOC_MAX_UNITS, else FASTOCR_ERR_WORKSPACE.
  *   - The first call on each device resolves the array's device address and sets kernel

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -32,7 +33,10 @@ struct fastocr_ctx {
   float* stats = nullptr;       // [max_batch][H][2]
   float* scores = nullptr;      // [max_batch][max_vis_len] (decode_step scratch)
   unsigned long long* faults = nullptr;
-  int ctas_per_sm = 2;          // persistent attention CTAs per SM
+  // persistent attention CTAs per SM brought by one launch: a full cache pass takes every slot,
+  // a pruned pass leaves one free (so that the next layer's launch can start beside it)
+  int dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
+  int sparse_ctas_per_sm = fastocr::kAttnCtasPerSm - 1;
   unsigned long long* trace = nullptr;   // set only by debug builds
   unsigned trace_seq = 0;
   char err[512] = {0};
@@ -121,7 +125,7 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
   a.trace = nullptr;
 #endif
   a.wait_point = fastocr::kWaitAtStart;
-  a.grid_ctas = ctx->sm_count * ctx->ctas_per_sm;
+  a.grid_ctas = ctx->sm_count * ctx->dense_ctas_per_sm;
   (void)max_len;
   return a;
 }
@@ -218,6 +222,7 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
   a.idx = idx;
   a.kcount = k;
   a.k_stride = k_stride;
+  a.grid_ctas = ctx->sm_count * ctx->sparse_ctas_per_sm;
   a.wait_point = wait_point;
   a.out = out;
   a.out_is_fp32 = out_is_fp32;
@@ -261,7 +266,11 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   }
   ctx->sm_count = sm > 0 ? sm : 148;
   // one partial slot per (CTA, unit) pair that can occur: CTAs + units
-  ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * ctx->ctas_per_sm +
+  if (const char* v = std::getenv("FASTOCR_DENSE_CTAS_PER_SM")) ctx->dense_ctas_per_sm = std::atoi(v);     // tuning knobs,
+  if (const char* v = std::getenv("FASTOCR_SPARSE_CTAS_PER_SM")) ctx->sparse_ctas_per_sm = std::atoi(v);   // read once here
+  if (ctx->dense_ctas_per_sm < 1 || ctx->dense_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
+  if (ctx->sparse_ctas_per_sm < 1 || ctx->sparse_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->sparse_ctas_per_sm = fastocr::kAttnCtasPerSm - 1;
+  ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * fastocr::kAttnCtasPerSm +
                    static_cast<int64_t>(lim->max_batch) * lim->num_kv_heads + 64;
   const int64_t nvis = lim->max_vis_len > 0 ? lim->max_vis_len : 1;
   const size_t bytes_acc = static_cast<size_t>(ctx->cap_items) * fastocr::kMaxGroup * fastocr::kHeadDim * sizeof(float);

@@ -3,16 +3,17 @@
 // set K = T u F (Eq. 2, non-focal case), on contiguous or paged caches.
 //
 // Work decomposition (stream-K over tokens). A unit is one (sequence, KV head) pair; its attended
-// tokens are cut into rows of 64 (one 16-token block per warp of a CTA). All rows of the launch
-// are laid end to end and divided into equal ranges, one per persistent CTA (two CTAs of four warps
-// per SM); when there are no more units than CTAs and the ranges are short, the number of active
-// CTAs is rounded down to a multiple of the unit count, so that equal-sized units are never shared
-// between CTAs. Every CTA
-// therefore streams the same number of rows, pays one pipeline prologue per launch and exits
-// without waiting for anyone. When a CTA's range leaves a unit, its four warps merge their
-// running (max, sum, output) through a 4 KB shared-memory buffer; a unit wholly inside the range is
-// normalised and written at once, a unit shared by several CTAs goes through global partials and
-// is merged by whichever CTA arrives last (one atomic arrival counter per unit, no spinning).
+// tokens are cut into rows of 32 (one 16-token block per warp of a CTA). The rows of the launch
+// are divided among persistent CTAs of two warps: equal parts of every unit when the units are of
+// similar length and no more numerous than the CTAs (no CTA then straddles two units), else
+// equal ranges of all rows laid end to end. Four CTAs fit an SM; a full-cache pass brings all four,
+// a pruned pass three, so that the next layer's launch (which starts early through programmatic
+// dependent launch) can run its prologue beside it. Every CTA streams about the same number of
+// rows, pays one pipeline prologue per unit piece and exits without waiting for anyone. When a
+// CTA leaves a unit, its warps merge their running (max, sum, output) through a 4 KB shared-memory
+// buffer; a unit held by one CTA is normalised and written at once, a unit shared by several CTAs
+// goes through global partials and is merged by whichever CTA arrives last (one atomic arrival
+// counter per unit, no spinning).
 //
 // Data path: a block's 16 K rows and 16 V rows (256 bytes each) travel HBM -> shared memory with
 // 16-byte cp.async, one full row per half-warp per instruction (so every request covers whole
@@ -51,7 +52,7 @@ constexpr int kBlockTokens = 16;                        // tokens per warp per p
 constexpr int kRowTokens = kAttnWarps * kBlockTokens;   // tokens per CTA per pipeline stage
 constexpr float kRescaleSlack = 8.0f;                   // log2 units
 constexpr int kMergeRound = 4;                          // partials fetched together by the merging CTA
-constexpr int kLongRangeRows = 32;                      // rows per CTA from which unit alignment is dropped
+constexpr int kLongRangeRows = 128;                     // rows per CTA from which unit alignment is dropped
 
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -141,7 +142,7 @@ __device__ __forceinline__ unsigned long long trace_now() {
 #endif
 
 template <int G, bool HAS_V>
-__global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaunch a) {
+__global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(const AttnLaunch a) {
   extern __shared__ __align__(16) unsigned char smem[];
   using L = Smem<HAS_V>;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -152,8 +153,11 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
   FASTOCR_TRACE_MARK(0);
   // Everything read before the first wait_for_prior_grids() must not have been produced by a
   // kernel that may still be running; the host says how much that is (AttnLaunch::wait_point).
+  // The next kernel is let in only once this one's own early reads are known to be safe: a kernel
+  // whose inputs were settled before it started says so at once, the others after their wait
+  // (their successor may assume that whatever they waited for has completed).
   if (a.wait_point == kWaitAtStart) wait_for_prior_grids();
-  dependents_may_launch();
+  if (a.wait_point != kWaitAfterSetup) dependents_may_launch();
 
   // ---- set-up: prefix of 64-token rows over units (warp 0) -------------------------------------
   int* prefix_s = reinterpret_cast<int*>(smem + L::prefix);
@@ -162,11 +166,12 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
   float* mrg_o = mrg_m + 16;                                   // [8][128]
   int* mrg_flag = reinterpret_cast<int*>(mrg_o + kMaxGroup * kHeadDim);
   if (warp == 0) {
-    int carry = 0;
+    int carry = 0, longest = 0;
     for (int u0 = 0; u0 < units; u0 += 32) {
       const int u = u0 + lane;
       int n = 0;
       if (u < units) n = (load_geom(a, u / Hkv).n_tok + kRowTokens - 1) / kRowTokens;
+      longest = max(longest, n);
       int incl = n;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -176,18 +181,39 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
       if (u < units) prefix_s[u] = carry + incl - n;
       carry += __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (lane == 0) prefix_s[units] = carry;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) longest = max(longest, __shfl_xor_sync(0xffffffffu, longest, o));
+    if (lane == 0) {
+      prefix_s[units] = carry;
+      mrg_flag[1] = longest;
+    }
   }
   __syncthreads();
   FASTOCR_TRACE_MARK(1);
-  const int total_rows = prefix_s[units];
+  const int total_rows = prefix_s[units], longest_unit = mrg_flag[1];
   const int grid = gridDim.x;
-  // short ranges: keep equal-sized units whole (no shared units, no global merge); long ranges:
-  // use every CTA, the few merges are negligible against the stream
-  const int active = (units <= grid && total_rows < kLongRangeRows * grid) ? units * (grid / units) : grid;
-  const int per_cta = (total_rows + active - 1) / active;
-  const int r0 = blockIdx.x * per_cta;
-  const int r1 = min(total_rows, r0 + per_cta);
+  // Two ways to hand out rows. Short ranges over at most `grid` units of similar length: every unit
+  // is cut into the same number of equal parts, one per CTA, so no CTA straddles two units (no
+  // pipeline refill) and a unit that fits one CTA needs no global merge. Otherwise (ragged
+  // batches, more units than CTAs, or long ranges where a few merges are negligible): all rows
+  // laid end to end and cut into equal ranges.
+  const bool split_units = units <= grid && total_rows < kLongRangeRows * grid &&
+                           static_cast<int64_t>(longest_unit) * units <= static_cast<int64_t>(total_rows) + total_rows / 8;
+  const int parts = split_units ? grid / units : 1;     // CTAs per unit
+  const int per_cta = (total_rows + grid - 1) / grid;   // rows per CTA (equal-range mode)
+  int r0 = 0, r1 = 0, first_unit = 0;
+  if (split_units) {
+    first_unit = blockIdx.x / parts;
+    if (first_unit < units) {
+      const int ub = prefix_s[first_unit], ue = prefix_s[first_unit + 1];
+      const int per = (ue - ub + parts - 1) / parts;
+      r0 = min(ue, ub + (blockIdx.x - first_unit * parts) * per);
+      r1 = min(ue, r0 + per);
+    }
+  } else {
+    r0 = min(total_rows, blockIdx.x * per_cta);
+    r1 = min(total_rows, r0 + per_cta);
+  }
 
   const float scale_log2 = a.sm_scale * 1.4426950408889634f;
   const int64_t row_elems = static_cast<int64_t>(Hkv) * kHeadDim;
@@ -199,8 +225,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
   FASTOCR_TRACE_MARK(2);
 
   // ---- the CTA's range, one unit segment after the other --------------------------------------
-  int u = 0;
-  if (per_cta > 0 && r0 < r1) {
+  int u = first_unit;
+  if (!split_units && r0 < r1) {
     int lo = 0, hi = units;                            // largest u with prefix[u] <= r0
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
@@ -209,9 +235,12 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
     u = lo;
   }
   int seg_begin = r0;
-  if (a.wait_point == kWaitAfterSetup) wait_for_prior_grids();   // before index-list reads and logits writes
+  if (a.wait_point == kWaitAfterSetup) {               // before index-list reads and logits writes
+    wait_for_prior_grids();
+    dependents_may_launch();
+  }
 #pragma unroll 1
-  while (per_cta > 0 && seg_begin < r1) {
+  while (seg_begin < r1) {
     while (prefix_s[u + 1] <= seg_begin) ++u;          // skip empty units
     const int ubeg = prefix_s[u], uend = prefix_s[u + 1];
     const int seg_rows = min(uend, r1) - seg_begin;    // rows of unit u inside this range
@@ -388,7 +417,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
     cp_async_wait<0>();
     FASTOCR_TRACE_MARK(4);
 
-    // ---- leaving the unit (all four warps get here together: they walk the same rows) ----------
+    // ---- leaving the unit (all warps of the CTA get here together: they walk the same rows) ----------
     wait_for_prior_grids();                            // results and the shared workspace are written from here on
     float l = l_part;
     l += __shfl_xor_sync(0xffffffffu, l, 1);
@@ -396,7 +425,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
     // this warp's maxima for the two heads whose outputs the lane holds
     const float mA = __shfl_sync(0xffffffffu, m_ref, 8 * t4), mB = __shfl_sync(0xffffffffu, m_ref, 8 * t4 + 4);
     __syncthreads();                                   // the merge buffer is free again
-    // the four warps fold their state into the shared buffer, one after the other
+    // the warps fold their state into the shared buffer, one after the other
 #pragma unroll 1
     for (int w = 0; w < kAttnWarps; ++w) {
       if (warp == w) {
@@ -429,30 +458,46 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
       }
       __syncthreads();
     }
-    // thread (h, d8) owns head h, dims d8 .. d8 + 7 of the CTA's result
+    // item e = (head e / 16, dims 8 (e % 16) .. + 7) of the CTA's result; kItems items per thread
     {
-      const int h = tid >> 4, d8 = (tid & 15) * 8;
-      const bool h_ok = h < G;
-      float M = mrg_m[h], den = mrg_l[h];
-      float num[8];
-      if (HAS_V) {
-        const float4 x0 = *reinterpret_cast<const float4*>(mrg_o + h * kHeadDim + d8);
-        const float4 x1 = *reinterpret_cast<const float4*>(mrg_o + h * kHeadDim + d8 + 4);
-        num[0] = x0.x; num[1] = x0.y; num[2] = x0.z; num[3] = x0.w;
-        num[4] = x1.x; num[5] = x1.y; num[6] = x1.z; num[7] = x1.w;
+      constexpr int kItems = kMaxGroup * 16 / kThreads;
+      float M[kItems], den[kItems], num[kItems][8];
+#pragma unroll
+      for (int it = 0; it < kItems; ++it) {
+        const int e = it * kThreads + tid, h = e >> 4, d8 = (e & 15) * 8;
+        M[it] = mrg_m[h];
+        den[it] = mrg_l[h];
+        if (HAS_V) {
+          const float4 x0 = *reinterpret_cast<const float4*>(mrg_o + h * kHeadDim + d8);
+          const float4 x1 = *reinterpret_cast<const float4*>(mrg_o + h * kHeadDim + d8 + 4);
+          num[it][0] = x0.x; num[it][1] = x0.y; num[it][2] = x0.z; num[it][3] = x0.w;
+          num[it][4] = x1.x; num[it][5] = x1.y; num[it][6] = x1.z; num[it][7] = x1.w;
+        }
       }
-      const int c_lo = ubeg / per_cta, c_hi = (uend - 1) / per_cta;
+      // the CTAs that hold a piece of this unit: [c_lo, c_hi]
+      int c_lo, c_hi;
+      if (split_units) {
+        const int per = (uend - ubeg + parts - 1) / parts;
+        c_lo = u * parts;
+        c_hi = c_lo + (uend - ubeg + per - 1) / per - 1;
+      } else {
+        c_lo = ubeg / per_cta;
+        c_hi = (uend - 1) / per_cta;
+      }
       const int64_t head0 = static_cast<int64_t>(u) * G;
       bool finish = true;
       if (c_lo != c_hi) {                              // the unit is shared with other CTAs
         const int64_t slot = static_cast<int64_t>(blockIdx.x) + u;
-        if (h_ok) {
+#pragma unroll
+        for (int it = 0; it < kItems; ++it) {
+          const int e = it * kThreads + tid, h = e >> 4, d8 = (e & 15) * 8;
+          if (h >= G) continue;
           if (HAS_V) {
             float4* dst = reinterpret_cast<float4*>(a.part_acc + (slot * kMaxGroup + h) * kHeadDim + d8);
-            dst[0] = make_float4(num[0], num[1], num[2], num[3]);
-            dst[1] = make_float4(num[4], num[5], num[6], num[7]);
+            dst[0] = make_float4(num[it][0], num[it][1], num[it][2], num[it][3]);
+            dst[1] = make_float4(num[it][4], num[it][5], num[it][6], num[it][7]);
           }
-          if ((tid & 15) == 0) *reinterpret_cast<float2*>(a.part_ml + (slot * kMaxGroup + h) * 2) = make_float2(M, den);
+          if ((e & 15) == 0) *reinterpret_cast<float2*>(a.part_ml + (slot * kMaxGroup + h) * 2) = make_float2(M[it], den[it]);
         }
         __threadfence();                               // partial visible before the arrival is counted
         __syncthreads();
@@ -466,51 +511,68 @@ __global__ void __launch_bounds__(kThreads, 2) attn_stream_kernel(const AttnLaun
         finish = *mrg_flag != 0;
         if (finish) {                                  // the last CTA to arrive merges all partials
           __threadfence();
-          M = -INFINITY;
-          den = 0.f;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) num[i] = 0.f;
 #pragma unroll 1
-          for (int c0 = c_lo; c0 <= c_hi; c0 += kMergeRound) {
-            float2 ml[kMergeRound];
-            float4 x0[kMergeRound], x1[kMergeRound];
+          for (int it = 0; it < kItems; ++it) {
+            const int e = it * kThreads + tid, h = e >> 4, d8 = (e & 15) * 8;
+            const int hh = h < G ? h : 0;
+            float Mm = -INFINITY, dd = 0.f, nn[8];
 #pragma unroll
-            for (int r = 0; r < kMergeRound; ++r) {    // a short tail re-reads the last partial (ignored below)
-              const int64_t sl = static_cast<int64_t>(min(c0 + r, c_hi)) + u;
-              const int hh = h_ok ? h : 0;
-              ml[r] = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (sl * kMaxGroup + hh) * 2));
-              x0[r] = x1[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (HAS_V) {
-                const float4* srcp = reinterpret_cast<const float4*>(a.part_acc + (sl * kMaxGroup + hh) * kHeadDim + d8);
-                x0[r] = __ldcg(srcp);
-                x1[r] = __ldcg(srcp + 1);
+            for (int i = 0; i < 8; ++i) nn[i] = 0.f;
+#pragma unroll 1
+            for (int c0 = c_lo; c0 <= c_hi; c0 += kMergeRound) {
+              float2 ml[kMergeRound];
+              float4 x0[kMergeRound], x1[kMergeRound];
+#pragma unroll
+              for (int r = 0; r < kMergeRound; ++r) {  // a short tail re-reads the last partial (ignored below)
+                const int64_t sl = static_cast<int64_t>(min(c0 + r, c_hi)) + u;
+                ml[r] = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (sl * kMaxGroup + hh) * 2));
+                x0[r] = x1[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (HAS_V) {
+                  const float4* srcp = reinterpret_cast<const float4*>(a.part_acc + (sl * kMaxGroup + hh) * kHeadDim + d8);
+                  x0[r] = __ldcg(srcp);
+                  x1[r] = __ldcg(srcp + 1);
+                }
+              }
+#pragma unroll
+              for (int r = 0; r < kMergeRound; ++r) {
+                if (c0 + r > c_hi || ml[r].x == -INFINITY) continue;
+                const float Mn = fmaxf(Mm, ml[r].x);
+                const float so = (Mm == -INFINITY) ? 0.f : exp2f(Mm - Mn), sn = exp2f(ml[r].x - Mn);
+                nn[0] = nn[0] * so + x0[r].x * sn; nn[1] = nn[1] * so + x0[r].y * sn;
+                nn[2] = nn[2] * so + x0[r].z * sn; nn[3] = nn[3] * so + x0[r].w * sn;
+                nn[4] = nn[4] * so + x1[r].x * sn; nn[5] = nn[5] * so + x1[r].y * sn;
+                nn[6] = nn[6] * so + x1[r].z * sn; nn[7] = nn[7] * so + x1[r].w * sn;
+                dd = dd * so + ml[r].y * sn;
+                Mm = Mn;
               }
             }
+            // (kItems is 1 or 2: select the slot without indexing registers dynamically)
 #pragma unroll
-            for (int r = 0; r < kMergeRound; ++r) {
-              if (c0 + r > c_hi || ml[r].x == -INFINITY) continue;
-              const float Mn = fmaxf(M, ml[r].x);
-              const float so = (M == -INFINITY) ? 0.f : exp2f(M - Mn), sn = exp2f(ml[r].x - Mn);
-              num[0] = num[0] * so + x0[r].x * sn; num[1] = num[1] * so + x0[r].y * sn;
-              num[2] = num[2] * so + x0[r].z * sn; num[3] = num[3] * so + x0[r].w * sn;
-              num[4] = num[4] * so + x1[r].x * sn; num[5] = num[5] * so + x1[r].y * sn;
-              num[6] = num[6] * so + x1[r].z * sn; num[7] = num[7] * so + x1[r].w * sn;
-              den = den * so + ml[r].y * sn;
-              M = Mn;
-            }
+            for (int jt = 0; jt < kItems; ++jt)
+              if (jt == it) {
+                M[jt] = Mm;
+                den[jt] = dd;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) num[jt][i] = nn[i];
+              }
           }
         }
       }
-      if (finish && h_ok) {
-        if (HAS_V) {
-          const float inv = den > 0.f ? 1.f / den : 0.f;
-          const int64_t oi = (head0 + h) * kHeadDim + d8;
+      if (finish) {
 #pragma unroll
-          for (int i = 0; i < 8; i += 2) store_pair(a.out, a.out_is_fp32, oi + i, num[i] * inv, num[i + 1] * inv);
-        }
-        if ((tid & 15) == 0 && a.stats != nullptr) {
-          a.stats[(head0 + h) * 2 + 0] = M;
-          a.stats[(head0 + h) * 2 + 1] = den;
+        for (int it = 0; it < kItems; ++it) {
+          const int e = it * kThreads + tid, h = e >> 4, d8 = (e & 15) * 8;
+          if (h >= G) continue;
+          if (HAS_V) {
+            const float inv = den[it] > 0.f ? 1.f / den[it] : 0.f;
+            const int64_t oi = (head0 + h) * kHeadDim + d8;
+#pragma unroll
+            for (int i = 0; i < 8; i += 2) store_pair(a.out, a.out_is_fp32, oi + i, num[it][i] * inv, num[it][i + 1] * inv);
+          }
+          if ((e & 15) == 0 && a.stats != nullptr) {
+            a.stats[(head0 + h) * 2 + 0] = M[it];
+            a.stats[(head0 + h) * 2 + 1] = den[it];
+          }
         }
       }
     }

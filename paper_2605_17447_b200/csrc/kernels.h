@@ -7,18 +7,26 @@ namespace fastocr {
 
 constexpr int kHeadDim = 128;
 constexpr int kMaxGroup = 8;          // query heads per KV head handled by one CTA
-constexpr int kAttnWarps = 4;         // autonomous warps per persistent attention CTA (two CTAs per SM)
-constexpr int kMaxUnits = 1024;       // sequences x KV heads per launch (their row prefix lives in shared memory)
+constexpr int kAttnWarps = 2;         // warps per persistent attention CTA
+constexpr int kAttnCtasPerSm = 4;     // resident CTAs per SM (shared memory); a launch uses half of them
+constexpr int kMaxUnits = 512;        // sequences x KV heads per launch (their row prefix lives in shared memory)
 constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
 
 // Programmatic dependent launch. Every kernel of this library is launched with the "programmatic
 // stream serialization" attribute and (i) lets its successor's CTAs be scheduled as soon as SM
 // resources free up (dependents_may_launch), (ii) calls wait_for_prior_grids() before it touches
 // anything an earlier kernel may have written or may still be reading; the wait returns when all
-// earlier kernels in the stream have completed and their writes are visible. A predecessor that is
-// not one of these kernels never triggers early, so ordinary stream order applies to it.
+// earlier kernels in the stream have completed and their writes are visible. A kernel that has to
+// wait before reading some input triggers its successor only after that wait: the successor may
+// be told (by the host) that the same input is settled, which is true only from then on. A
+// predecessor that is not one of these kernels never triggers early, so ordinary stream order
+// applies to it.
 #ifdef __CUDACC__
+#ifdef FASTOCR_NO_EARLY_LAUNCH   // debug builds: every kernel starts after its predecessor has finished
+__device__ __forceinline__ void dependents_may_launch() {}
+#else
 __device__ __forceinline__ void dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+#endif
 __device__ __forceinline__ void wait_for_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>

@@ -15,14 +15,14 @@
 
 namespace {
 
-constexpr int kNoallocMaxSlots = FASTOCR_NOALLOC_MAX_UNITS + 2 * 192;   // units + persistent CTAs (<= 192 SMs)
+constexpr int kNoallocMaxSlots = FASTOCR_NOALLOC_MAX_UNITS + 3 * 160;   // units + persistent CTAs (3 per SM, <= 160 SMs)
 constexpr size_t kAccBytes = static_cast<size_t>(kNoallocMaxSlots) * fastocr::kMaxGroup * fastocr::kHeadDim * sizeof(float);
 constexpr size_t kMlBytes = static_cast<size_t>(kNoallocMaxSlots) * fastocr::kMaxGroup * 2 * sizeof(float);
 constexpr size_t kCounterBytes = static_cast<size_t>(FASTOCR_NOALLOC_MAX_UNITS) * sizeof(int32_t);
 constexpr size_t kFaultBytes = 256;
 constexpr size_t kScratchBytes = kAccBytes + kMlBytes + kCounterBytes + kFaultBytes;
 
-// The scratch itself: about 2.7 MB held by every GPU that loads the library, until exit.
+// The scratch itself: about 3.1 MB held by every GPU that loads the library, until exit.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
 struct DeviceSetup {
@@ -94,7 +94,7 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   fastocr_status st = setup_current_device(device);
   if (st != FASTOCR_OK) return st;
   const DeviceSetup& s = g_setup[device];
-  const int grid = 2 * s.sm_count;
+  const int grid = 3 * s.sm_count;
   if (units + grid > kNoallocMaxSlots) return fail(FASTOCR_ERR_WORKSPACE, "this GPU has more SMs than the built-in scratch was sized for");
 
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
