@@ -48,6 +48,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=None, help="override the number of layer caches")
     ap.add_argument("--distinct-steps", type=int, default=16, help="length of the replayed fixation track")
     ap.add_argument("--focal", default=None, help="comma-separated focal layers (skips Focal Layer Selection)")
+    ap.add_argument("--sweep", action="store_true", help="roofline sweep over N and tau (7B-shaped layer, batch 64); prints one JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
@@ -301,8 +302,65 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_sweep(args):
+    """Roofline sweep of the benchmark's config 4: per (N, tau), the pruned layer and the dense layer
+    timed back to back over 8 distinct layer caches (so every launch reads cold data), plus
+    scoring + selection, as us per layer and GB/s of algorithmic bytes."""
+    import paper_2605_17447_b200 as fo
+    peak, peak_kind = measured_peaks()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    points = []
+    reps = 20
+    for N in (1024, 4096, 8192, 16384, 32768):
+        for tau in (0.02, 0.05, 0.10, 0.20, 1.0):
+            cfg = get_config("cfg4", N=N, batch=args.batch, layers=8, tau=tau)
+            if tau == 0.02:                       # one data set per N; tau only changes k
+                w = Workload(cfg, 2, dev)
+            else:
+                w.cfg.tau = tau
+                w.k = [fo.kept_count(n, tau) for n in w.vis_len]
+                w.k_d.copy_(torch.tensor(w.k, dtype=torch.int32))
+                w.fix = torch.zeros(w.B, max(w.k), dtype=torch.int32, device=dev)
+            w.max_kept = max(k + t for k, t in zip(w.k, w.text0)) + w.nd
+            out = torch.empty(w.L, w.B, w.H, cfg.head_dim, dtype=torch.bfloat16, device=dev)
+            q = w.q_all[0]
+            w.set_step(0)
+            # a real selection for this tau: one focal pass on layer 0
+            sel = fo.StepPlan(w.ctx, w.views[:1], [True], w.k_d, w.fix, max(w.vis_len))
+            sel.run(q[:1], out[:1], False)
+            chain = fo.StepPlan(w.ctx, w.views, [False] * w.L, w.k_d, w.fix, max(w.vis_len), w.max_kept)
+            def sparse_chain(t):
+                chain.run(q, out, True)
+            def dense_chain(t):
+                for l in range(w.L):
+                    fo.fastocr_dense_decode_attn(w.ctx, w.views[l], q[l], out[l])
+            scores = torch.zeros(w.B, max(w.vis_len), dtype=torch.float32, device=dev)
+            def select_only(t):
+                fo.fastocr_focal_scores(w.ctx, w.views[t % w.L], q[t % w.L], scores)
+                fo.fastocr_select_topk(w.ctx, scores, w.vis_len_d, w.k_d, w.fix, max(w.vis_len))
+            res = {}
+            for name, fn, per in (("sparse", sparse_chain, w.L), ("dense", dense_chain, w.L), ("scores_topk", select_only, 1)):
+                for t in range(3):
+                    fn(t)
+                res[name] = timed(fn, reps, lambda: None) / reps / per * 1e3
+            sel.run(q[:1], out[:1], False)        # leave a valid selection behind
+            sb, db = w.sparse_bytes(0), w.dense_bytes(0)
+            points.append({"N": N, "tau": tau, "k": w.k[0], "sparse_us": res["sparse"], "dense_us": res["dense"],
+                           "scores_topk_us": res["scores_topk"], "sparse_gbs": sb / res["sparse"] / 1e3,
+                           "dense_gbs": db / res["dense"] / 1e3, "sparse_frac_of_8tbs": sb / res["sparse"] / 1e3 / NOMINAL_HBM_GBS,
+                           "sparse_frac_of_measured": sb / res["sparse"] / 1e3 / peak, "dense_frac_of_measured": db / res["dense"] / 1e3 / peak,
+                           "layer_speedup": res["dense"] / res["sparse"]})
+        del w
+        torch.cuda.empty_cache()
+    print(json.dumps({"sweep": "cfg4", "batch": args.batch, "layers_cycled": 8, "peak_gbs": peak, "peak_kind": peak_kind, "points": points}))
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

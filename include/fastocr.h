@@ -141,8 +141,8 @@ fastocr_status fastocr_select_topk(fastocr_ctx* ctx, const float* scores, int32_
  * K = T u F only: every text position plus positions vis_start + idx[b][i], i < k[b].
  *   idx device int32 [B][k_stride] (values in [0, vis_len[b]); need not be sorted, must be distinct)
  *   k   device int32 [B]
- *   max_kept host-known bound on k[b] + seq_len[b] - vis_len[b], or 0 if unknown (a sizing hint;
- *            the current kernels balance the work from the device-side lengths and ignore it)
+ *   max_kept host-known bound on k[b] + seq_len[b] - vis_len[b], or 0 if unknown; only used to
+ *            size the launch (a long pass takes every CTA slot, a short one leaves room for the next layer)
  * A sequence whose kept set is empty yields zeros.
  */
 fastocr_status fastocr_sparse_decode_attn(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q,

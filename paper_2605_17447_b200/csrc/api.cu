@@ -222,7 +222,13 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
   a.idx = idx;
   a.kcount = k;
   a.k_stride = k_stride;
-  a.grid_ctas = ctx->sm_count * ctx->sparse_ctas_per_sm;
+  // Leave a slot per SM free for the next layer's launch unless the pass is long enough (per the
+  // caller's bound on kept tokens) for the overlap not to matter: then take every slot.
+  {
+    const int64_t rows = static_cast<int64_t>(kv->batch) * kv->num_kv_heads * ((max_len + 31) / 32);
+    const bool long_pass = max_kept > 0 && rows >= static_cast<int64_t>(64) * ctx->sm_count * fastocr::kAttnCtasPerSm;
+    a.grid_ctas = ctx->sm_count * (long_pass ? ctx->dense_ctas_per_sm : ctx->sparse_ctas_per_sm);
+  }
   a.wait_point = wait_point;
   a.out = out;
   a.out_is_fp32 = out_is_fp32;
