@@ -126,6 +126,7 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
 #endif
   a.wait_point = fastocr::kWaitAtStart;
   a.grid_ctas = ctx->sm_count * ctx->dense_ctas_per_sm;
+  a.active_ctas = a.grid_ctas;
   (void)max_len;
   return a;
 }
@@ -228,6 +229,11 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
     const int64_t rows = static_cast<int64_t>(kv->batch) * kv->num_kv_heads * ((max_len + 31) / 32);
     const bool long_pass = max_kept > 0 && rows >= static_cast<int64_t>(64) * ctx->sm_count * fastocr::kAttnCtasPerSm;
     a.grid_ctas = ctx->sm_count * (long_pass ? ctx->dense_ctas_per_sm : ctx->sparse_ctas_per_sm);
+    // no idle CTAs: when every unit gets the same number of CTAs (the kernel's choice for batches
+    // of similar sequences), a grid that is a multiple of the unit count has none left over
+    const int units = kv->batch * kv->num_kv_heads;
+    if (!long_pass && units <= a.grid_ctas) a.grid_ctas = units * (a.grid_ctas / units);
+    a.active_ctas = a.grid_ctas;
   }
   a.wait_point = wait_point;
   a.out = out;

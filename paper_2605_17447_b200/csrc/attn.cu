@@ -191,7 +191,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   __syncthreads();
   FASTOCR_TRACE_MARK(1);
   const int total_rows = prefix_s[units], longest_unit = mrg_flag[1];
-  const int grid = gridDim.x;
+  const int grid = min(static_cast<int>(gridDim.x), a.active_ctas);
   // Two ways to hand out rows. Short ranges over at most `grid` units of similar length: every unit
   // is cut into the same number of equal parts, one per CTA, so no CTA straddles two units (no
   // pipeline refill) and a unit that fits one CTA needs no global merge. Otherwise (ragged
@@ -202,7 +202,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   const int parts = split_units ? grid / units : 1;     // CTAs per unit
   const int per_cta = (total_rows + grid - 1) / grid;   // rows per CTA (equal-range mode)
   int r0 = 0, r1 = 0, first_unit = 0;
-  if (split_units) {
+  if (static_cast<int>(blockIdx.x) >= grid) {
+    // a spare CTA: launched only so that the launch claims the whole shared-memory array of every SM
+  } else if (split_units) {
     first_unit = blockIdx.x / parts;
     if (first_unit < units) {
       const int ub = prefix_s[first_unit], ue = prefix_s[first_unit + 1];
@@ -418,7 +420,6 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     FASTOCR_TRACE_MARK(4);
 
     // ---- leaving the unit (all warps of the CTA get here together: they walk the same rows) ----------
-    wait_for_prior_grids();                            // results and the shared workspace are written from here on
     float l = l_part;
     l += __shfl_xor_sync(0xffffffffu, l, 1);
     l += __shfl_xor_sync(0xffffffffu, l, 2);
@@ -487,6 +488,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       const int64_t head0 = static_cast<int64_t>(u) * G;
       bool finish = true;
       if (c_lo != c_hi) {                              // the unit is shared with other CTAs
+        wait_for_prior_grids();                        // the split workspace may still be in use by the previous kernel
         const int64_t slot = static_cast<int64_t>(blockIdx.x) + u;
 #pragma unroll
         for (int it = 0; it < kItems; ++it) {
@@ -581,6 +583,11 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   }
   FASTOCR_TRACE_MARK(5);
 
+  // A kernel of this library must not complete before its predecessor has (later kernels rely on
+  // "my predecessor is done, hence everything before it"). CTAs that wrote only their own output
+  // slice did not have to wait; one CTA anchors the chain, the others free their SM slots at once.
+  if (blockIdx.x == 0) wait_for_prior_grids();
+
   // ---- sequences with nothing to attend get zeros (rare; kept off the main path) ---------------
   if (blockIdx.x == 0) {
     for (int e = 0; e < units; ++e) {
@@ -658,8 +665,11 @@ cudaError_t launch_partial_t(const AttnLaunch& a, cudaStream_t s) {
 
 template <int G, bool HAS_V>
 cudaError_t configure_t() {
-  return cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Smem<HAS_V>::total);
+  cudaError_t e = cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       Smem<HAS_V>::total);
+  if (e != cudaSuccess) return e;
+  // all of the SM's L1/shared array as shared memory: four CTAs must fit
+  return cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
 }
 
 }  // namespace
@@ -693,6 +703,17 @@ cudaError_t configure_kernels() {
 #undef X
   return cudaSuccess;
 }
+
+#ifdef FASTOCR_TRACE
+// debug builds: resident CTAs per SM the runtime grants the 7-head attention kernel
+extern "C" int fastocr_debug_occupancy() {
+  int n = -1;
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_stream_kernel<7, true>, kThreads, Smem<true>::total);
+  cudaFuncAttributes fa;
+  cudaFuncGetAttributes(&fa, attn_stream_kernel<7, true>);
+  return n * 1000 + fa.numRegs;
+}
+#endif
 
 cudaError_t launch_scores_finalize(const float* logits, const float* stats, const int32_t* vis_len, int32_t batch,
                                    int32_t num_q_heads, int32_t n_stride_logits, int32_t max_vis_len, float* scores,

@@ -68,7 +68,8 @@ struct AttnLaunch {
   const int32_t* idx;
   const int32_t* kcount;
   int32_t k_stride;
-  int32_t grid_ctas;          // persistent CTAs (kAttnWarps warps each)
+  int32_t grid_ctas;          // CTAs launched (kAttnWarps warps each)
+  int32_t active_ctas;        // CTAs that take work (<= grid_ctas); the rest exit at once
   int32_t wait_point;         // where the kernel waits for earlier kernels: kWaitAtStart / kWaitAfterSetup / kWaitBeforeWrites
   // workspace
   float* part_acc;            // [slots][8][128], slot = CTA index + unit index (unit = sequence * Hkv + KV head)
