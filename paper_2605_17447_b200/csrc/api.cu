@@ -126,6 +126,13 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
 #endif
   a.wait_point = fastocr::kWaitAtStart;
   a.grid_ctas = ctx->sm_count * ctx->dense_ctas_per_sm;
+  {
+    // small batches: the kernel gives every unit at most kMaxPartsPerUnit CTAs; launch no more
+    const int units = kv->batch * kv->num_kv_heads;
+    const int64_t rows = static_cast<int64_t>(units) * ((max_len + 31) / 32);
+    if (units * fastocr::kMaxPartsPerUnit < a.grid_ctas && rows < static_cast<int64_t>(128) * a.grid_ctas)
+      a.grid_ctas = units * fastocr::kMaxPartsPerUnit;
+  }
   a.active_ctas = a.grid_ctas;
   (void)max_len;
   return a;
@@ -232,7 +239,13 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
     // no idle CTAs: when every unit gets the same number of CTAs (the kernel's choice for batches
     // of similar sequences), a grid that is a multiple of the unit count has none left over
     const int units = kv->batch * kv->num_kv_heads;
-    if (!long_pass && units <= a.grid_ctas) a.grid_ctas = units * (a.grid_ctas / units);
+    if (!long_pass && units <= a.grid_ctas) {
+      int parts = a.grid_ctas / units;
+      const int max_rows = (max_len + 31) / 32;          // a unit cannot feed more CTAs than it has rows
+      if (parts > max_rows) parts = max_rows;
+      if (parts > fastocr::kMaxPartsPerUnit) parts = fastocr::kMaxPartsPerUnit;
+      a.grid_ctas = units * parts;
+    }
     a.active_ctas = a.grid_ctas;
   }
   a.wait_point = wait_point;

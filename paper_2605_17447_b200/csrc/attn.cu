@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   // laid end to end and cut into equal ranges.
   const bool split_units = units <= grid && total_rows < kLongRangeRows * grid &&
                            static_cast<int64_t>(longest_unit) * units <= static_cast<int64_t>(total_rows) + total_rows / 8;
-  const int parts = split_units ? grid / units : 1;     // CTAs per unit
+  const int parts = split_units ? min(grid / units, kMaxPartsPerUnit) : 1;     // CTAs per unit
   const int per_cta = (total_rows + grid - 1) / grid;   // rows per CTA (equal-range mode)
   int r0 = 0, r1 = 0, first_unit = 0;
   if (static_cast<int>(blockIdx.x) >= grid) {
@@ -513,50 +513,49 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
         finish = *mrg_flag != 0;
         if (finish) {                                  // the last CTA to arrive merges all partials
           __threadfence();
-#pragma unroll 1
-          for (int it = 0; it < kItems; ++it) {
-            const int e = it * kThreads + tid, h = e >> 4, d8 = (e & 15) * 8;
-            const int hh = h < G ? h : 0;
-            float Mm = -INFINITY, dd = 0.f, nn[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) nn[i] = 0.f;
+          for (int it = 0; it < kItems; ++it) {
+            M[it] = -INFINITY;
+            den[it] = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) num[it][i] = 0.f;
+          }
+          // kMergeRound partials of every item of this thread are fetched together, then folded in
 #pragma unroll 1
-            for (int c0 = c_lo; c0 <= c_hi; c0 += kMergeRound) {
-              float2 ml[kMergeRound];
-              float4 x0[kMergeRound], x1[kMergeRound];
+          for (int c0 = c_lo; c0 <= c_hi; c0 += kMergeRound) {
+            float2 ml[kItems][kMergeRound];
+            float4 x0[kItems][kMergeRound], x1[kItems][kMergeRound];
+#pragma unroll
+            for (int it = 0; it < kItems; ++it) {
+              const int e = it * kThreads + tid, h = e >> 4, d8 = (e & 15) * 8;
+              const int hh = h < G ? h : 0;
 #pragma unroll
               for (int r = 0; r < kMergeRound; ++r) {  // a short tail re-reads the last partial (ignored below)
                 const int64_t sl = static_cast<int64_t>(min(c0 + r, c_hi)) + u;
-                ml[r] = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (sl * kMaxGroup + hh) * 2));
-                x0[r] = x1[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                ml[it][r] = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (sl * kMaxGroup + hh) * 2));
+                x0[it][r] = x1[it][r] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (HAS_V) {
                   const float4* srcp = reinterpret_cast<const float4*>(a.part_acc + (sl * kMaxGroup + hh) * kHeadDim + d8);
-                  x0[r] = __ldcg(srcp);
-                  x1[r] = __ldcg(srcp + 1);
+                  x0[it][r] = __ldcg(srcp);
+                  x1[it][r] = __ldcg(srcp + 1);
                 }
               }
+            }
+#pragma unroll
+            for (int it = 0; it < kItems; ++it) {
 #pragma unroll
               for (int r = 0; r < kMergeRound; ++r) {
-                if (c0 + r > c_hi || ml[r].x == -INFINITY) continue;
-                const float Mn = fmaxf(Mm, ml[r].x);
-                const float so = (Mm == -INFINITY) ? 0.f : exp2f(Mm - Mn), sn = exp2f(ml[r].x - Mn);
-                nn[0] = nn[0] * so + x0[r].x * sn; nn[1] = nn[1] * so + x0[r].y * sn;
-                nn[2] = nn[2] * so + x0[r].z * sn; nn[3] = nn[3] * so + x0[r].w * sn;
-                nn[4] = nn[4] * so + x1[r].x * sn; nn[5] = nn[5] * so + x1[r].y * sn;
-                nn[6] = nn[6] * so + x1[r].z * sn; nn[7] = nn[7] * so + x1[r].w * sn;
-                dd = dd * so + ml[r].y * sn;
-                Mm = Mn;
+                if (c0 + r > c_hi || ml[it][r].x == -INFINITY) continue;
+                const float Mn = fmaxf(M[it], ml[it][r].x);
+                const float so = (M[it] == -INFINITY) ? 0.f : exp2f(M[it] - Mn), sn = exp2f(ml[it][r].x - Mn);
+                num[it][0] = num[it][0] * so + x0[it][r].x * sn; num[it][1] = num[it][1] * so + x0[it][r].y * sn;
+                num[it][2] = num[it][2] * so + x0[it][r].z * sn; num[it][3] = num[it][3] * so + x0[it][r].w * sn;
+                num[it][4] = num[it][4] * so + x1[it][r].x * sn; num[it][5] = num[it][5] * so + x1[it][r].y * sn;
+                num[it][6] = num[it][6] * so + x1[it][r].z * sn; num[it][7] = num[it][7] * so + x1[it][r].w * sn;
+                den[it] = den[it] * so + ml[it][r].y * sn;
+                M[it] = Mn;
               }
             }
-            // (kItems is 1 or 2: select the slot without indexing registers dynamically)
-#pragma unroll
-            for (int jt = 0; jt < kItems; ++jt)
-              if (jt == it) {
-                M[jt] = Mm;
-                den[jt] = dd;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) num[jt][i] = nn[i];
-              }
           }
         }
       }
