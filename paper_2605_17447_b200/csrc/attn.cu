@@ -43,6 +43,8 @@
 
 #include <cuda_bf16.h>
 
+#include <climits>
+
 namespace fastocr {
 namespace {
 
@@ -133,12 +135,21 @@ __device__ __forceinline__ unsigned long long trace_now() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
   return t;
 }
+#define FASTOCR_TRACE_CLK(var) const long long var = clock64()
+#define FASTOCR_TRACE_CYC(slot)                                                                             \
+  do {                                                                                                      \
+    if (a.trace != nullptr && lane == 0) a.trace[(blockIdx.x * kAttnWarps + warp) * 16 + (slot)] = clock64(); \
+  } while (0)
+#define FASTOCR_TRACE_ADD(acc, t1, t0) acc += static_cast<unsigned>((t1) - (t0))
 #define FASTOCR_TRACE_MARK(slot)                                                                            \
   do {                                                                                                      \
-    if (a.trace != nullptr && lane == 0) a.trace[(blockIdx.x * kAttnWarps + warp) * 8 + (slot)] = trace_now(); \
+    if (a.trace != nullptr && lane == 0) a.trace[(blockIdx.x * kAttnWarps + warp) * 16 + (slot)] = trace_now(); \
   } while (0)
 #else
 #define FASTOCR_TRACE_MARK(slot) do { } while (0)
+#define FASTOCR_TRACE_CLK(var) do { } while (0)
+#define FASTOCR_TRACE_CYC(slot) do { } while (0)
+#define FASTOCR_TRACE_ADD(acc, t1, t0) do { } while (0)
 #endif
 
 template <int G, bool HAS_V>
@@ -151,45 +162,88 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   const int units = a.batch * Hkv;                     // unit u = (sequence u / Hkv, KV head u % Hkv)
 
   FASTOCR_TRACE_MARK(0);
+  FASTOCR_TRACE_CYC(8);
+#ifdef FASTOCR_TRACE
+  unsigned trace_wait = 0, trace_qk = 0, trace_look = 0, trace_pv = 0;   // cycles, summed over the main loop
+#endif
   // Everything read before the first wait_for_prior_grids() must not have been produced by a
   // kernel that may still be running; the host says how much that is (AttnLaunch::wait_point).
   // The next kernel is let in only once this one's own early reads are known to be safe: a kernel
   // whose inputs were settled before it started says so at once, the others after their wait
   // (their successor may assume that whatever they waited for has completed).
+  // When it does so on top of that is a matter of pacing: a successor that streams the same amount
+  // of data should begin its set-up while this kernel is in mid-stream, so that one kernel's idle
+  // set-up phase falls into the other's streaming phase instead of all CTAs of the GPU setting up
+  // (memory idle) and then streaming (memory saturated) in step.
+  const bool trigger_early = a.trigger_q8 <= 0;
   if (a.wait_point == kWaitAtStart) wait_for_prior_grids();
-  if (a.wait_point != kWaitAfterSetup) dependents_may_launch();
+  if (a.wait_point != kWaitAfterSetup && trigger_early) dependents_may_launch();
 
-  // ---- set-up: prefix of 64-token rows over units (warp 0) -------------------------------------
+  // ---- set-up: prefix of the units' row counts ----------------------------------------------------
+  // Every thread fetches the lengths of up to kMaxUnits / kThreads units at once (one round trip to
+  // L2 for the whole table), warp 0 then scans the counts in shared memory.
   int* prefix_s = reinterpret_cast<int*>(smem + L::prefix);
   float* mrg_m = reinterpret_cast<float*>(smem + L::merge);   // [8]
   float* mrg_l = mrg_m + 8;                                    // [8]
   float* mrg_o = mrg_m + 16;                                   // [8][128]
   int* mrg_flag = reinterpret_cast<int*>(mrg_o + kMaxGroup * kHeadDim);
-  if (warp == 0) {
-    int carry = 0, longest = 0;
-    for (int u0 = 0; u0 < units; u0 += 32) {
-      const int u = u0 + lane;
-      int n = 0;
-      if (u < units) n = (load_geom(a, u / Hkv).n_tok + kRowTokens - 1) / kRowTokens;
-      longest = max(longest, n);
-      int incl = n;
+  // every unit's geometry, kept in the (still unused) ring until the CTA has picked up that of its
+  // first unit: saves that unit a second round trip to L2
+  int4* geom_s = reinterpret_cast<int4*>(smem + L::ring);
+  static_assert(kMaxUnits * 16 <= L::kRingBytes, "the geometry table must fit the ring");
+  {
+    constexpr int kPerThread = kMaxUnits / kThreads;
+    int rows_of[kPerThread];
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
+    for (int i = 0; i < kPerThread; ++i) {
+      const int uu = i * kThreads + tid;
+      rows_of[i] = 0;
+      if (uu < units) {
+        const SeqGeom sg = load_geom(a, uu / Hkv);
+        rows_of[i] = (sg.n_tok + kRowTokens - 1) / kRowTokens;
+        geom_s[uu] = make_int4(sg.vs, sg.N, sg.kept_vis, sg.n_tok);
       }
-      if (u < units) prefix_s[u] = carry + incl - n;
-      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    int longest = 0;
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+      const int uu = i * kThreads + tid;
+      if (uu < units) prefix_s[uu + 1] = rows_of[i];
+      longest = max(longest, rows_of[i]);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) longest = max(longest, __shfl_xor_sync(0xffffffffu, longest, o));
+    if (lane == 0) mrg_flag[1 + warp] = longest;
+  }
+  FASTOCR_TRACE_CYC(9);
+  __syncthreads();
+  if (warp == 0) {                                     // lane l owns units [l * chunk, (l + 1) * chunk)
+    const int chunk = (units + 31) >> 5;
+    const int u_lo = lane * chunk, u_hi = min(units, u_lo + chunk);
+    int sum = 0;
+    for (int uu = u_lo; uu < u_hi; ++uu) sum += prefix_s[uu + 1];
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    int run = incl - sum;
+    for (int uu = u_lo; uu < u_hi; ++uu) {
+      run += prefix_s[uu + 1];
+      prefix_s[uu + 1] = run;
+    }
     if (lane == 0) {
-      prefix_s[units] = carry;
+      prefix_s[0] = 0;
+      int longest = mrg_flag[1];
+#pragma unroll
+      for (int w = 1; w < kAttnWarps; ++w) longest = max(longest, mrg_flag[1 + w]);
       mrg_flag[1] = longest;
     }
   }
   __syncthreads();
   FASTOCR_TRACE_MARK(1);
+  FASTOCR_TRACE_CYC(10);
   const int total_rows = prefix_s[units], longest_unit = mrg_flag[1];
   const int grid = min(static_cast<int>(gridDim.x), a.active_ctas);
   // Two ways to hand out rows. Short ranges over at most `grid` units of similar length: every unit
@@ -224,7 +278,13 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   const uint32_t smem_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
   const uint32_t ring_warp = smem_u32 + L::ring + warp * kStages * L::kStageBytes;
   const bool head_ok = g8 < G;
-  FASTOCR_TRACE_MARK(2);
+#ifdef FASTOCR_TRACE
+  if (a.trace != nullptr && lane == 0) {               // slot 2: the SM this CTA runs on
+    unsigned smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    a.trace[(blockIdx.x * kAttnWarps + warp) * 16 + 2] = smid + 1;
+  }
+#endif
 
   // ---- the CTA's range, one unit segment after the other --------------------------------------
   int u = first_unit;
@@ -239,15 +299,24 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   int seg_begin = r0;
   if (a.wait_point == kWaitAfterSetup) {               // before index-list reads and logits writes
     wait_for_prior_grids();
-    dependents_may_launch();
+    if (trigger_early) dependents_may_launch();
   }
+  // the row of this CTA's range at which it triggers (a CTA without rows triggers by exiting)
+  const int trigger_row = trigger_early ? INT_MIN : r0 + min(((r1 - r0) * min(a.trigger_q8, 256)) >> 8, r1 - r0 - 1);
 #pragma unroll 1
   while (seg_begin < r1) {
     while (prefix_s[u + 1] <= seg_begin) ++u;          // skip empty units
     const int ubeg = prefix_s[u], uend = prefix_s[u + 1];
     const int seg_rows = min(uend, r1) - seg_begin;    // rows of unit u inside this range
     const int b = u / Hkv, g = u - b * Hkv;
-    const SeqGeom sg = load_geom(a, b);
+    SeqGeom sg;
+    if (seg_begin == r0) {                             // first segment: from the table in shared memory
+      const int4 gq = geom_s[u];
+      sg.vs = gq.x; sg.N = gq.y; sg.kept_vis = gq.z; sg.n_tok = gq.w;
+      __syncthreads();                                 // both warps have read it: the ring may be written
+    } else {
+      sg = load_geom(a, b);
+    }
     const int tok0 = (seg_begin - ubeg) * kRowTokens + warp * kBlockTokens;   // this warp's first token of the segment
     const __nv_bfloat16* kptr = reinterpret_cast<const __nv_bfloat16*>(a.k) + b * seq_elems + g * kHeadDim + 8 * c16;
     const __nv_bfloat16* vptr =
@@ -276,64 +345,26 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     // the iteration that loads it): P (row n+4) logical position of token `lane` (< 16) of this
     // warp's block, a load from the index list for selected image tokens; R (row n+3) physical
     // cache row, a block-table load for paged caches; I (row n+2) the cp.async copies; C (row n)
-    // the arithmetic. The first four iterations (n < 0) only fill the stages.
-    int pos_p = 0, row_p = 0;
-    bool idx_p = false;                                // pos_p is a raw index-list entry, checked in stage R
-#pragma unroll 1
-    for (int n = -4; n < seg_rows; ++n) {
-      const bool real = n >= 0;
-      if (real) {
-        cp_async_wait<kStages - 2>();
-        __syncwarp();                                  // every lane's copies of this block have landed
-      }
-      if (n == 0) FASTOCR_TRACE_MARK(3);
-      const uint32_t src = ring_warp + ((n + kStages) % kStages) * L::kStageBytes;
-      const int j0 = tok0 + n * kRowTokens;
-      const bool live = real && j0 < sg.n_tok;         // the block holds at least one attended token
-      float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
-      uint4 vw[4][2];
-      if (live) {
-        // ---- S^T = Q K^T for the two 8-token tiles --------------------------------------------
-        // lane (g8, t4) reads chunk 4j + t4 of rows g8 and 8 + g8: per 8-lane phase two rows whose
-        // swizzles differ in bit 2, i.e. eight distinct 16-byte bank groups
-        const uint32_t krow = src + g8 * 256;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const uint32_t coff = ((4 * j + t4) ^ k_swz(g8)) << 4;    // k_swz(8 + g8) == k_swz(g8)
-          const uint4 ka = lds128(krow + coff), kb = lds128(krow + 8 * 256 + coff);
-          mma_bf16(sa, qw[j][0], 0u, qw[j][1], 0u, ka.x, ka.y);
-          mma_bf16(sa, qw[j][2], 0u, qw[j][3], 0u, ka.z, ka.w);
-          mma_bf16(sb, qw[j][0], 0u, qw[j][1], 0u, kb.x, kb.y);
-          mma_bf16(sb, qw[j][2], 0u, qw[j][3], 0u, kb.z, kb.w);
-        }
-        if (HAS_V) {
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {                // rows {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4}, chunks g8 and 8 + g8
-            const int tk = 2 * t4 + (v & 1) + 8 * (v >> 1);
-            const uint32_t vrow = src + L::kTileBytes + tk * 256;
-            vw[v][0] = lds128(vrow + ((g8 ^ v_swz(tk)) << 4));
-            vw[v][1] = lds128(vrow + (((8 + g8) ^ v_swz(tk)) << 4));
+    // the arithmetic.
+    auto stage_p = [&](int r, int& pos, bool& is_idx) {      // is_idx: pos is a raw index-list entry, checked in stage R
+      is_idx = false;
+      const int jr = tok0 + r * kRowTokens;
+      if (r < seg_rows && jr < sg.n_tok && lane < kBlockTokens) {
+        const int j = min(jr + lane, sg.n_tok - 1);
+        pos = j;
+        if (a.idx != nullptr) {                        // kept set: text before | selected image | text after
+          if (j >= sg.vs + sg.kept_vis) {
+            pos = j - sg.kept_vis + sg.N;
+          } else if (j >= sg.vs) {
+            pos = __ldg(a.idx + static_cast<int64_t>(b) * a.k_stride + (j - sg.vs));
+            is_idx = true;
           }
         }
       }
-      // ---- stage I: copies of row n + 2 ---------------------------------------------------------
-      if (n >= -2) {
-        if (n + 2 < seg_rows && j0 + 2 * kRowTokens < sg.n_tok) {
-          const uint32_t dst = ring_warp + ((n + 2 + kStages) % kStages) * L::kStageBytes;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {                // rows 2i (lanes 0-15) and 2i + 1 (lanes 16-31)
-            const int tok = 2 * i + half;
-            const int64_t roff = __shfl_sync(0xffffffffu, row_p, tok) * row_elems;
-            cp_async16(dst + tok * 256 + ((c16 ^ k_swz(tok)) << 4), kptr + roff);
-            if (HAS_V) cp_async16(dst + L::kTileBytes + tok * 256 + ((c16 ^ v_swz(tok)) << 4), vptr + roff);
-          }
-        }
-        cp_async_commit();
-      }
-      // ---- stage R: cache row of row n + 3 ------------------------------------------------------
-      if (n + 3 < seg_rows && j0 + 3 * kRowTokens < sg.n_tok && lane < kBlockTokens) {
-        int pos = pos_p;
-        if (idx_p) {
+    };
+    auto stage_r = [&](int r, int pos, bool is_idx, int& row) {
+      if (r < seg_rows && tok0 + r * kRowTokens < sg.n_tok && lane < kBlockTokens) {
+        if (is_idx) {
           if (pos < 0 || pos >= sg.N) {                // never read outside the image span
             atomicAdd(a.fault_counter, 1ULL);
             pos = pos < 0 ? 0 : sg.N - 1;
@@ -344,23 +375,113 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           const int page = __ldg(a.block_table + static_cast<int64_t>(b) * a.max_pages + pos / a.page_size);
           pos = page * a.page_size + pos % a.page_size;
         }
-        row_p = pos;
+        row = pos;
       }
-      // ---- stage P: position of row n + 4 (nothing may depend on the loaded value here) ---------
-      idx_p = false;
-      if (n + 4 < seg_rows && j0 + 4 * kRowTokens < sg.n_tok && lane < kBlockTokens) {
-        const int j = min(j0 + 4 * kRowTokens + lane, sg.n_tok - 1);
-        pos_p = j;
-        if (a.idx != nullptr) {                        // kept set: text before | selected image | text after
-          if (j >= sg.vs + sg.kept_vis) {
-            pos_p = j - sg.kept_vis + sg.N;
-          } else if (j >= sg.vs) {
-            pos_p = __ldg(a.idx + static_cast<int64_t>(b) * a.k_stride + (j - sg.vs));
-            idx_p = true;
+    };
+    auto stage_i = [&](int r, int row) {
+      if (r < seg_rows && tok0 + r * kRowTokens < sg.n_tok) {
+        const uint32_t dst = ring_warp + (r % kStages) * L::kStageBytes;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {                  // rows 2i (lanes 0-15) and 2i + 1 (lanes 16-31)
+          const int tok = 2 * i + half;
+          const int64_t roff = __shfl_sync(0xffffffffu, row, tok) * row_elems;
+          cp_async16(dst + tok * 256 + ((c16 ^ k_swz(tok)) << 4), kptr + roff);
+          if (HAS_V) cp_async16(dst + L::kTileBytes + tok * 256 + ((c16 ^ v_swz(tok)) << 4), vptr + roff);
+        }
+      }
+      cp_async_commit();
+    };
+    // Address translation: a pruned pass touches a handful of rows in every 2 MiB page of the
+    // sequence's cache span, and the first touch of a page by this SM costs a translation miss in
+    // the middle of the stream. Touch every page of the span now, all at once (one line each, L2
+    // only): lanes 0-15 of warp 0 for K, lanes 16-31 for V.
+    if (a.idx != nullptr && a.page_size == 0 && warp == 0) {
+      const int64_t span = static_cast<int64_t>(sg.n_tok - sg.kept_vis + sg.N) * row_elems * 2;   // bytes, whole sequence
+      const char* base = reinterpret_cast<const char*>(half ? static_cast<const void*>(a.v) : a.k) +
+                         (b * seq_elems + g * kHeadDim) * 2;
+      int64_t off = static_cast<int64_t>(c16) << 21;
+      if (c16 == 15) off = span - 256;
+      if (off >= 0 && off < span && (HAS_V || half == 0)) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
+    }
+    // Filling the stages: the lookups of the first rows are issued together (one round trip for
+    // the index-list entries of rows 0-3, one for the block-table entries of rows 0-2) instead of
+    // one after the other, then the copies of rows 0 and 1 go out.
+    int pos_p = 0, row_p = 0;
+    bool idx_p = false;
+    FASTOCR_TRACE_CYC(11);
+    {
+      int pos0 = 0, pos1 = 0, pos2 = 0, row0 = 0, row1 = 0;
+      bool ix0, ix1, ix2;
+      stage_p(0, pos0, ix0);
+      stage_p(1, pos1, ix1);
+      stage_p(2, pos2, ix2);
+      stage_p(3, pos_p, idx_p);
+      stage_r(0, pos0, ix0, row0);
+      stage_r(1, pos1, ix1, row1);
+      stage_r(2, pos2, ix2, row_p);
+      FASTOCR_TRACE_CYC(12);
+      stage_i(0, row0);
+      stage_i(1, row1);
+      FASTOCR_TRACE_CYC(13);
+    }
+#pragma unroll 1
+    for (int n = 0; n < seg_rows; ++n) {
+      if (seg_begin + n == trigger_row) dependents_may_launch();
+      const int j0 = tok0 + n * kRowTokens;
+      FASTOCR_TRACE_CLK(c_top);
+      cp_async_wait<kStages - 2>();
+      __syncwarp();                                    // every lane's copies of this block have landed
+      FASTOCR_TRACE_CLK(c_waited);
+      FASTOCR_TRACE_ADD(trace_wait, c_waited, c_top);
+      if (n == 0) { FASTOCR_TRACE_MARK(3); FASTOCR_TRACE_CYC(14); }
+      const uint32_t src = ring_warp + (n % kStages) * L::kStageBytes;
+      const bool live = j0 < sg.n_tok;         // the block holds at least one attended token
+      // two accumulators per 8-token tile (even / odd 32-dim pieces): dependent MMA chains of four
+      float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+      float sa2[4] = {0.f, 0.f, 0.f, 0.f}, sb2[4] = {0.f, 0.f, 0.f, 0.f};
+      uint4 vw[4][2];
+      if (live) {
+        // ---- S^T = Q K^T for the two 8-token tiles --------------------------------------------
+        // lane (g8, t4) reads chunk 4j + t4 of rows g8 and 8 + g8: per 8-lane phase two rows whose
+        // swizzles differ in bit 2, i.e. eight distinct 16-byte bank groups
+        const uint32_t krow = src + g8 * 256;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t coff = ((4 * j + t4) ^ k_swz(g8)) << 4;    // k_swz(8 + g8) == k_swz(g8)
+          const uint4 ka = lds128(krow + coff), kb = lds128(krow + 8 * 256 + coff);
+          if (j & 1) {
+            mma_bf16(sa2, qw[j][0], 0u, qw[j][1], 0u, ka.x, ka.y);
+            mma_bf16(sb2, qw[j][0], 0u, qw[j][1], 0u, kb.x, kb.y);
+            mma_bf16(sa2, qw[j][2], 0u, qw[j][3], 0u, ka.z, ka.w);
+            mma_bf16(sb2, qw[j][2], 0u, qw[j][3], 0u, kb.z, kb.w);
+          } else {
+            mma_bf16(sa, qw[j][0], 0u, qw[j][1], 0u, ka.x, ka.y);
+            mma_bf16(sb, qw[j][0], 0u, qw[j][1], 0u, kb.x, kb.y);
+            mma_bf16(sa, qw[j][2], 0u, qw[j][3], 0u, ka.z, ka.w);
+            mma_bf16(sb, qw[j][2], 0u, qw[j][3], 0u, kb.z, kb.w);
+          }
+        }
+        sa[0] += sa2[0]; sa[1] += sa2[1]; sb[0] += sb2[0]; sb[1] += sb2[1];   // rows 8-15 of the tiles are padding
+        if (HAS_V) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {                // rows {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4}, chunks g8 and 8 + g8
+            const int tk = 2 * t4 + (v & 1) + 8 * (v >> 1);
+            const uint32_t vrow = src + L::kTileBytes + tk * 256;
+            vw[v][0] = lds128(vrow + ((g8 ^ v_swz(tk)) << 4));
+            vw[v][1] = lds128(vrow + (((8 + g8) ^ v_swz(tk)) << 4));
           }
         }
       }
+      FASTOCR_TRACE_CLK(c_qk);
+      FASTOCR_TRACE_ADD(trace_qk, c_qk, c_waited);
+      // ---- stages I, R, P for rows n + 2, n + 3, n + 4 (the ring slot of row n + 2 is the one row
+      // n - 1 was read from; the __syncwarp above separates those reads from these writes) -------
+      stage_i(n + 2, row_p);
+      stage_r(n + 3, pos_p, idx_p, row_p);
+      stage_p(n + 4, pos_p, idx_p);
 
+      FASTOCR_TRACE_CLK(c_look);
+      FASTOCR_TRACE_ADD(trace_look, c_look, c_qk);
       if (live) {
         // ---- online softmax for head g8, tokens j0 + {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4} -----
         float x[4] = {sa[0] * scale_log2, sa[1] * scale_log2, sb[0] * scale_log2, sb[1] * scale_log2};
@@ -415,9 +536,12 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           }
         }
       }
+      FASTOCR_TRACE_CLK(c_end);
+      FASTOCR_TRACE_ADD(trace_pv, c_end, c_look);
     }
     cp_async_wait<0>();
     FASTOCR_TRACE_MARK(4);
+    FASTOCR_TRACE_CYC(15);
 
     // ---- leaving the unit (all warps of the CTA get here together: they walk the same rows) ----------
     float l = l_part;
@@ -581,6 +705,12 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     ++u;
   }
   FASTOCR_TRACE_MARK(5);
+#ifdef FASTOCR_TRACE
+  if (a.trace != nullptr && lane == 0) {
+    a.trace[(blockIdx.x * kAttnWarps + warp) * 16 + 6] = (static_cast<unsigned long long>(trace_wait) << 32) | trace_qk;
+    a.trace[(blockIdx.x * kAttnWarps + warp) * 16 + 7] = (static_cast<unsigned long long>(trace_look) << 32) | trace_pv;
+  }
+#endif
 
   // A kernel of this library must not complete before its predecessor has (later kernels rely on
   // "my predecessor is done, hence everything before it"). CTAs that wrote only their own output
