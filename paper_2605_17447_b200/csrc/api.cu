@@ -197,10 +197,13 @@ struct ProfScope {
   } while (0)
 
 // dense pass (+ optional fused scoring) without re-validating the view
+// scores_out == NULL with logits_only: logits and per-head statistics are left in the context's
+// workspace for a consumer that forms the scores itself (the selection kernel)
 fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, void* out, int out_is_fp32,
-                          float* scores_out, int32_t n_stride, int32_t max_vis, int wait_point, cudaStream_t s) {
+                          float* scores_out, int32_t n_stride, int32_t max_vis, int wait_point, cudaStream_t s,
+                          bool logits_only = false) {
   AttnLaunch a = make_launch(ctx, kv, q, /*with_v=*/out != nullptr, kv->max_seq_len);
-  const bool want_scores = scores_out != nullptr;
+  const bool want_scores = scores_out != nullptr || logits_only;
   if (want_scores) {
     a.logits = ctx->logits;
     a.n_stride = ctx->lim.max_vis_len;
@@ -213,7 +216,7 @@ fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
     ProfScope p(ctx, out != nullptr ? FASTOCR_PROF_ATTN_DENSE : FASTOCR_PROF_ATTN_KEYS, s);
     FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
   }
-  if (want_scores) {
+  if (want_scores && !logits_only) {
     ProfScope p(ctx, FASTOCR_PROF_FINALIZE, s);
     FASTOCR_TRY_CUDA(fastocr::launch_scores_finalize(ctx->logits, ctx->stats, kv->vis_len, kv->batch, kv->num_q_heads,
                                                      ctx->lim.max_vis_len, max_vis, scores_out, n_stride, s),
@@ -248,6 +251,7 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
       if (parts > fastocr::kMaxPartsPerUnit) parts = fastocr::kMaxPartsPerUnit;
       a.grid_ctas = units * parts;
     }
+    if (const char* v = std::getenv("FASTOCR_SPARSE_GRID")) a.grid_ctas = std::atoi(v);   // EXPERIMENT
     a.active_ctas = a.grid_ctas;
   }
   a.wait_point = wait_point;
@@ -397,7 +401,7 @@ fastocr_status fastocr_select_topk(fastocr_ctx* ctx, const float* scores, int32_
     return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "max_vis_len %d exceeds %d", max_vis_len, fastocr::kTopkMaxN);
   ProfScope p(ctx, FASTOCR_PROF_TOPK, static_cast<cudaStream_t>(stream));
   FASTOCR_TRY_CUDA(fastocr::launch_select_topk(scores, n_stride, vis_len, k, batch, max_vis_len, idx_out, k_stride,
-                                               static_cast<cudaStream_t>(stream)),
+                                               nullptr, nullptr, 0, 0, static_cast<cudaStream_t>(stream)),
                    "top-k launch");
   return FASTOCR_OK;
 }
@@ -446,13 +450,17 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
     if (focal || (l == 0 && !have)) {
       // full attention + scoring + selection; the refreshed set replaces the current one.
       // The logits workspace is written from the first block on: wait before the stream starts.
-      st = dense_impl(ctx, &layers[l], ql, ol, out_is_fp32, ctx->scores, ctx->lim.max_vis_len, max_vis_len,
-                      chained ? fastocr::kWaitAfterSetup : fastocr::kWaitAtStart, s);
+      // The selection kernel forms the scores from the logits itself (no score array, one launch
+      // less) unless there are more heads than it has room for.
+      const bool fused = layers[l].num_q_heads <= fastocr::kTopkMaxHeads;
+      st = dense_impl(ctx, &layers[l], ql, ol, out_is_fp32, fused ? nullptr : ctx->scores, ctx->lim.max_vis_len, max_vis_len,
+                      chained ? fastocr::kWaitAfterSetup : fastocr::kWaitAtStart, s, fused);
       if (st != FASTOCR_OK) return st;
       {
         ProfScope p(ctx, FASTOCR_PROF_TOPK, s);
         FASTOCR_TRY_CUDA(fastocr::launch_select_topk(ctx->scores, ctx->lim.max_vis_len, layers[l].vis_len, k, layers[l].batch,
-                                                     max_vis_len, fixation, k_stride, s),
+                                                     max_vis_len, fixation, k_stride, fused ? ctx->logits : nullptr, ctx->stats,
+                                                     layers[l].num_q_heads, ctx->lim.max_vis_len, s),
                          "top-k launch");
       }
       have = true;

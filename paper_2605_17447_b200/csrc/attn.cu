@@ -53,6 +53,7 @@ constexpr int kThreads = kAttnWarps * 32;
 constexpr int kBlockTokens = 16;                        // tokens per warp per pipeline stage
 constexpr int kRowTokens = kAttnWarps * kBlockTokens;   // tokens per CTA per pipeline stage
 constexpr float kRescaleSlack = 8.0f;                   // log2 units
+constexpr int kMergePitch = kHeadDim + 4;                // floats per head in the CTA's merge buffer (bank spread)
 constexpr int kMergeRound = 4;                          // partials fetched together by the merging CTA
 constexpr int kLongRangeRows = 128;                     // rows per CTA from which unit alignment is dropped
 
@@ -73,6 +74,21 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 r;
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr) : "memory");
   return r;
+}
+// four 8x8 b16 matrices from shared memory (lane l supplies the address of row l % 8 of matrix l / 8)
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+// transpose of an 8x8 b16 matrix held one row per lane group (the MMA fragment layout)
+__device__ __forceinline__ uint32_t movm_trans(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
 }
 // D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -112,10 +128,9 @@ __device__ __forceinline__ SeqGeom load_geom(const AttnLaunch& a, int b) {
   return s;
 }
 
-// chunk swizzles of a staged row (16 chunks of 16 bytes): K fragments are read by (token g8,
-// chunk 4j + t4), V fragments by (token pair index t4, chunk g8); see the bank analysis in the reads
-__device__ __forceinline__ int k_swz(int tok) { return (tok & 1) << 2; }
-__device__ __forceinline__ int v_swz(int tok) { return ((tok >> 1) & 3) << 1; }
+// chunk swizzle of a staged row (16 chunks of 16 bytes): the eight rows of an ldmatrix 8x8 matrix
+// (eight consecutive tokens, same chunk) land in eight different 16-byte bank groups
+__device__ __forceinline__ int row_swz(int tok) { return tok & 7; }
 
 // shared-memory carve-up (bytes). A stage holds a 16 x 256 B K tile (+ the same for V) per warp.
 template <bool HAS_V>
@@ -126,7 +141,7 @@ struct Smem {
   static constexpr int ring = 0;
   static constexpr int prefix = kRingBytes;                          // int32 [kMaxUnits + 1], rows before each unit
   static constexpr int merge = prefix + ((kMaxUnits + 1) * 4 + 15) / 16 * 16;   // float m[8], l[8], o[8][128], int flag
-  static constexpr int total = merge + (16 + kMaxGroup * kHeadDim + 4) * 4;
+  static constexpr int total = merge + (16 + kMaxGroup * (kHeadDim + 4) + 4) * 4;
 };
 
 #ifdef FASTOCR_TRACE
@@ -185,8 +200,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   int* prefix_s = reinterpret_cast<int*>(smem + L::prefix);
   float* mrg_m = reinterpret_cast<float*>(smem + L::merge);   // [8]
   float* mrg_l = mrg_m + 8;                                    // [8]
-  float* mrg_o = mrg_m + 16;                                   // [8][128]
-  int* mrg_flag = reinterpret_cast<int*>(mrg_o + kMaxGroup * kHeadDim);
+  float* mrg_o = mrg_m + 16;                                   // [8][kMergePitch]
+  int* mrg_flag = reinterpret_cast<int*>(mrg_o + kMaxGroup * kMergePitch);
   // every unit's geometry, kept in the (still unused) ring until the CTA has picked up that of its
   // first unit: saves that unit a second round trip to L2
   int4* geom_s = reinterpret_cast<int4*>(smem + L::ring);
@@ -322,24 +337,33 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     const __nv_bfloat16* vptr =
         HAS_V ? reinterpret_cast<const __nv_bfloat16*>(a.v) + b * seq_elems + g * kHeadDim + 8 * c16 : nullptr;
 
-    // A fragments of Q: head g8, dims 32j + 8 t4 .. + 8
-    uint32_t qw[4][4];
+    // B fragments of Q^T for the eight 16-dim steps: head g8, dims 16 s + {2 t4, 2 t4 + 1} and 16 s + 8 + {2 t4, 2 t4 + 1}
+    uint32_t qb[8][2];
     {
-      const uint4* qp = reinterpret_cast<const uint4*>(a.q) + (static_cast<int64_t>(u) * G + g8) * (kHeadDim / 8) + t4;
+      const uint32_t* qp = reinterpret_cast<const uint32_t*>(a.q) + (static_cast<int64_t>(u) * G + g8) * (kHeadDim / 2) + t4;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        uint4 w = make_uint4(0u, 0u, 0u, 0u);
-        if (head_ok) w = __ldg(qp + 4 * j);
-        qw[j][0] = w.x; qw[j][1] = w.y; qw[j][2] = w.z; qw[j][3] = w.w;
+      for (int st = 0; st < 8; ++st) {
+        qb[st][0] = head_ok ? __ldg(qp + 8 * st) : 0u;
+        qb[st][1] = head_ok ? __ldg(qp + 8 * st + 4) : 0u;
       }
     }
-    float o[8][4];                                     // O^T tiles: dims {64 (j>>2) + 8 g8 + 2 (j&3) + (0|1)} x heads {2 t4, 2 t4 + 1}
+    // The lane's share of the state: heads hA = 2 t4 and hB = 2 t4 + 1.
+    float o[8][4];                                     // O^T tile j: dims {16 j + g8, 16 j + 8 + g8} x heads {hA, hB}
 #pragma unroll
     for (int j = 0; j < 8; ++j)
 #pragma unroll
       for (int i = 0; i < 4; ++i) o[j][i] = 0.f;
-    float m_ref = -INFINITY, l_part = 0.f;             // head g8 (identical in the 4 lanes of a group)
-    float* logit_row = (a.logits != nullptr && head_ok) ? a.logits + (static_cast<int64_t>(u) * G + g8) * a.n_stride : nullptr;
+    float mA = -INFINITY, mB = -INFINITY;              // reference maxima (identical in the 8 lanes that share t4)
+    float lA = 0.f, lB = 0.f;                          // this lane's part of the sums (tokens g8, 8 + g8 of every block)
+    const bool okA = 2 * t4 < G, okB = 2 * t4 + 1 < G;
+    float* logitA = (a.logits != nullptr && okA) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4) * a.n_stride : nullptr;
+    float* logitB = (a.logits != nullptr && okB) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4 + 1) * a.n_stride : nullptr;
+    // ldmatrix row addresses inside a tile. K (A operand of S = K Q^T, tokens on M): matrix l / 8 =
+    // (tokens 8 (i & 1) .., chunk 2 s + (i >> 1)); V (A operand of O^T = V^T P through .trans):
+    // matrix i = (tokens 8 (i >> 1) .., chunk 2 j + (i & 1)).
+    const int lm_r = lane & 7, lm_i = lane >> 3;
+    const uint32_t k_lm = (lm_r + 8 * (lm_i & 1)) * 256, k_lm_c = lm_i >> 1;
+    const uint32_t v_lm = (lm_r + 8 * (lm_i >> 1)) * 256, v_lm_c = lm_i & 1;
 
     // Look-ahead stages, each one row behind the previous (so that no loaded value is needed in
     // the iteration that loads it): P (row n+4) logical position of token `lane` (< 16) of this
@@ -385,8 +409,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
         for (int i = 0; i < 8; ++i) {                  // rows 2i (lanes 0-15) and 2i + 1 (lanes 16-31)
           const int tok = 2 * i + half;
           const int64_t roff = __shfl_sync(0xffffffffu, row, tok) * row_elems;
-          cp_async16(dst + tok * 256 + ((c16 ^ k_swz(tok)) << 4), kptr + roff);
-          if (HAS_V) cp_async16(dst + L::kTileBytes + tok * 256 + ((c16 ^ v_swz(tok)) << 4), vptr + roff);
+          cp_async16(dst + tok * 256 + ((c16 ^ row_swz(tok)) << 4), kptr + roff);
+          if (HAS_V) cp_async16(dst + L::kTileBytes + tok * 256 + ((c16 ^ row_swz(tok)) << 4), vptr + roff);
         }
       }
       cp_async_commit();
@@ -436,41 +460,19 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       if (n == 0) { FASTOCR_TRACE_MARK(3); FASTOCR_TRACE_CYC(14); }
       const uint32_t src = ring_warp + (n % kStages) * L::kStageBytes;
       const bool live = j0 < sg.n_tok;         // the block holds at least one attended token
-      // two accumulators per 8-token tile (even / odd 32-dim pieces): dependent MMA chains of four
-      float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
-      float sa2[4] = {0.f, 0.f, 0.f, 0.f}, sb2[4] = {0.f, 0.f, 0.f, 0.f};
-      uint4 vw[4][2];
+      // two accumulators (even / odd 16-dim steps): dependent MMA chains of four
+      float sc[4] = {0.f, 0.f, 0.f, 0.f}, sc2[4] = {0.f, 0.f, 0.f, 0.f};
       if (live) {
-        // ---- S^T = Q K^T for the two 8-token tiles --------------------------------------------
-        // lane (g8, t4) reads chunk 4j + t4 of rows g8 and 8 + g8: per 8-lane phase two rows whose
-        // swizzles differ in bit 2, i.e. eight distinct 16-byte bank groups
-        const uint32_t krow = src + g8 * 256;
+        // ---- S = K Q^T: tokens j0 + {g8, 8 + g8} x heads {hA, hB} ---------------------------------
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const uint32_t coff = ((4 * j + t4) ^ k_swz(g8)) << 4;    // k_swz(8 + g8) == k_swz(g8)
-          const uint4 ka = lds128(krow + coff), kb = lds128(krow + 8 * 256 + coff);
-          if (j & 1) {
-            mma_bf16(sa2, qw[j][0], 0u, qw[j][1], 0u, ka.x, ka.y);
-            mma_bf16(sb2, qw[j][0], 0u, qw[j][1], 0u, kb.x, kb.y);
-            mma_bf16(sa2, qw[j][2], 0u, qw[j][3], 0u, ka.z, ka.w);
-            mma_bf16(sb2, qw[j][2], 0u, qw[j][3], 0u, kb.z, kb.w);
-          } else {
-            mma_bf16(sa, qw[j][0], 0u, qw[j][1], 0u, ka.x, ka.y);
-            mma_bf16(sb, qw[j][0], 0u, qw[j][1], 0u, kb.x, kb.y);
-            mma_bf16(sa, qw[j][2], 0u, qw[j][3], 0u, ka.z, ka.w);
-            mma_bf16(sb, qw[j][2], 0u, qw[j][3], 0u, kb.z, kb.w);
-          }
+        for (int st = 0; st < 8; ++st) {
+          uint32_t ka[4];
+          ldsm_x4(ka, src + k_lm + (((2 * st + k_lm_c) ^ lm_r) << 4));
+          if (st & 1) mma_bf16(sc2, ka[0], ka[1], ka[2], ka[3], qb[st][0], qb[st][1]);
+          else mma_bf16(sc, ka[0], ka[1], ka[2], ka[3], qb[st][0], qb[st][1]);
         }
-        sa[0] += sa2[0]; sa[1] += sa2[1]; sb[0] += sb2[0]; sb[1] += sb2[1];   // rows 8-15 of the tiles are padding
-        if (HAS_V) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {                // rows {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4}, chunks g8 and 8 + g8
-            const int tk = 2 * t4 + (v & 1) + 8 * (v >> 1);
-            const uint32_t vrow = src + L::kTileBytes + tk * 256;
-            vw[v][0] = lds128(vrow + ((g8 ^ v_swz(tk)) << 4));
-            vw[v][1] = lds128(vrow + (((8 + g8) ^ v_swz(tk)) << 4));
-          }
-        }
+        for (int i = 0; i < 4; ++i) sc[i] += sc2[i];
       }
       FASTOCR_TRACE_CLK(c_qk);
       FASTOCR_TRACE_ADD(trace_qk, c_qk, c_waited);
@@ -483,56 +485,60 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       FASTOCR_TRACE_CLK(c_look);
       FASTOCR_TRACE_ADD(trace_look, c_look, c_qk);
       if (live) {
-        // ---- online softmax for head g8, tokens j0 + {2 t4, 2 t4 + 1, 8 + 2 t4, 9 + 2 t4} -----
-        float x[4] = {sa[0] * scale_log2, sa[1] * scale_log2, sb[0] * scale_log2, sb[1] * scale_log2};
+        // ---- online softmax: x[0], x[1] token j0 + g8 (heads hA, hB); x[2], x[3] token j0 + 8 + g8 ------
+        float x[4] = {sc[0] * scale_log2, sc[1] * scale_log2, sc[2] * scale_log2, sc[3] * scale_log2};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int tok = j0 + 2 * t4 + (i & 1) + 8 * (i >> 1);     // index in the unit's attended list
-          const bool valid = head_ok && tok < sg.n_tok;
+          const int tok = j0 + g8 + 8 * (i >> 1);      // index in the unit's attended list
+          const bool valid = ((i & 1) ? okB : okA) && tok < sg.n_tok;
           x[i] = valid ? x[i] : -INFINITY;
-          if (logit_row != nullptr && valid) {         // dense / scoring mode: position == list index
+          float* lrow = (i & 1) ? logitB : logitA;
+          if (lrow != nullptr && valid) {              // dense / scoring mode: position == list index
             const int rel = tok - sg.vs;
-            if (rel >= 0 && rel < sg.N && rel < a.n_stride) logit_row[rel] = x[i];
+            if (rel >= 0 && rel < sg.N && rel < a.n_stride) lrow[rel] = x[i];
           }
         }
-        float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-        if (__any_sync(0xffffffffu, mx > m_ref + kRescaleSlack)) {
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-          const bool raise = mx > m_ref + kRescaleSlack;
-          const float alpha = raise ? fast_exp2(m_ref - mx) : 1.f; // m_ref = -inf gives 0
-          if (raise) m_ref = mx;
-          l_part *= alpha;
+        float mxA = fmaxf(x[0], x[2]), mxB = fmaxf(x[1], x[3]);
+        if (__any_sync(0xffffffffu, mxA > mA + kRescaleSlack || mxB > mB + kRescaleSlack)) {
+#pragma unroll
+          for (int off = 4; off < 32; off <<= 1) {     // over the 8 lanes that share t4
+            mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, off));
+            mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, off));
+          }
+          const bool raiseA = mxA > mA + kRescaleSlack, raiseB = mxB > mB + kRescaleSlack;
+          const float alA = raiseA ? fast_exp2(mA - mxA) : 1.f;   // m = -inf gives 0
+          const float alB = raiseB ? fast_exp2(mB - mxB) : 1.f;
+          if (raiseA) mA = mxA;
+          if (raiseB) mB = mxB;
+          lA *= alA;
+          lB *= alB;
           if (HAS_V) {
-            const float a0 = __shfl_sync(0xffffffffu, alpha, 8 * t4);     // head 2 t4 lives in group 2 t4
-            const float a1 = __shfl_sync(0xffffffffu, alpha, 8 * t4 + 4); // head 2 t4 + 1
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1;
+              o[j][0] *= alA; o[j][1] *= alB; o[j][2] *= alA; o[j][3] *= alB;
             }
           }
         }
         float p[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          p[i] = (x[i] == -INFINITY) ? 0.f : fast_exp2(x[i] - m_ref);
-          l_part += p[i];
-        }
+        for (int i = 0; i < 4; ++i) p[i] = (x[i] == -INFINITY) ? 0.f : fast_exp2(x[i] - ((i & 1) ? mB : mA));
+        lA += p[0] + p[2];
+        lB += p[1] + p[3];
         if (HAS_V) {
-          // B fragments of P (tokens on K, head g8 on N): high bf16 part and remainder
-          const uint32_t ph0 = pack_bf16(p[0], p[1]), ph1 = pack_bf16(p[2], p[3]);
-          const uint32_t pl0 = pack_bf16(p[0] - __uint_as_float(ph0 << 16), p[1] - __uint_as_float(ph0 & 0xffff0000u));
-          const uint32_t pl1 = pack_bf16(p[2] - __uint_as_float(ph1 << 16), p[3] - __uint_as_float(ph1 & 0xffff0000u));
+          // P as the B operand of O^T += V^T P (tokens on K, head g8 on N) is the transpose of what the
+          // lanes hold (token g8, heads hA hB): one movmatrix per 8-token half, for the bf16 high
+          // part and for the remainder
+          const uint32_t h0 = pack_bf16(p[0], p[1]), h1 = pack_bf16(p[2], p[3]);
+          const uint32_t r0w = pack_bf16(p[0] - __uint_as_float(h0 << 16), p[1] - __uint_as_float(h0 & 0xffff0000u));
+          const uint32_t r1w = pack_bf16(p[2] - __uint_as_float(h1 << 16), p[3] - __uint_as_float(h1 & 0xffff0000u));
+          const uint32_t ph0 = movm_trans(h0), ph1 = movm_trans(h1), pl0 = movm_trans(r0w), pl1 = movm_trans(r1w);
+          const uint32_t vt = src + L::kTileBytes + v_lm;
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const int piece = j >> 2, i = j & 3;
-            const uint32_t w0 = (&vw[0][piece].x)[i], w1 = (&vw[1][piece].x)[i];
-            const uint32_t w2 = (&vw[2][piece].x)[i], w3 = (&vw[3][piece].x)[i];
-            // A fragment of V^T: rows = (even dim, odd dim), columns = token pairs
-            const uint32_t a0 = __byte_perm(w0, w1, 0x5410), a1 = __byte_perm(w0, w1, 0x7632);
-            const uint32_t a2 = __byte_perm(w2, w3, 0x5410), a3 = __byte_perm(w2, w3, 0x7632);
-            mma_bf16(o[j], a0, a1, a2, a3, ph0, ph1);
-            mma_bf16(o[j], a0, a1, a2, a3, pl0, pl1);
+            uint32_t va[4];                            // A fragment of V^T: dims 16 j .. + 15 x the block's 16 tokens
+            ldsm_x4_trans(va, vt + (((2 * j + v_lm_c) ^ lm_r) << 4));
+            mma_bf16(o[j], va[0], va[1], va[2], va[3], ph0, ph1);
+            mma_bf16(o[j], va[0], va[1], va[2], va[3], pl0, pl1);
           }
         }
       }
@@ -544,40 +550,41 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     FASTOCR_TRACE_CYC(15);
 
     // ---- leaving the unit (all warps of the CTA get here together: they walk the same rows) ----------
-    float l = l_part;
-    l += __shfl_xor_sync(0xffffffffu, l, 1);
-    l += __shfl_xor_sync(0xffffffffu, l, 2);
-    // this warp's maxima for the two heads whose outputs the lane holds
-    const float mA = __shfl_sync(0xffffffffu, m_ref, 8 * t4), mB = __shfl_sync(0xffffffffu, m_ref, 8 * t4 + 4);
+    // sums over the block's tokens: the 8 lanes that share t4 hold parts for heads hA, hB
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+      lA += __shfl_xor_sync(0xffffffffu, lA, off);
+      lB += __shfl_xor_sync(0xffffffffu, lB, off);
+    }
     __syncthreads();                                   // the merge buffer is free again
     // the warps fold their state into the shared buffer, one after the other
 #pragma unroll 1
     for (int w = 0; w < kAttnWarps; ++w) {
       if (warp == w) {
-        float sbA = 0.f, swA = 1.f, sbB = 0.f, swB = 1.f, sb8 = 0.f, sw8 = 1.f, Mn8 = m_ref;
+        float sbA = 0.f, swA = 1.f, sbB = 0.f, swB = 1.f, MnA = mA, MnB = mB;
         if (w > 0) {
-          const float bA = mrg_m[2 * t4], bB = mrg_m[2 * t4 + 1], b8 = mrg_m[g8];
-          const float MnA = fmaxf(bA, mA), MnB = fmaxf(bB, mB);
-          Mn8 = fmaxf(b8, m_ref);
+          const float bA = mrg_m[2 * t4], bB = mrg_m[2 * t4 + 1];
+          MnA = fmaxf(bA, mA);
+          MnB = fmaxf(bB, mB);
           sbA = bA == -INFINITY ? 0.f : exp2f(bA - MnA); swA = mA == -INFINITY ? 0.f : exp2f(mA - MnA);
           sbB = bB == -INFINITY ? 0.f : exp2f(bB - MnB); swB = mB == -INFINITY ? 0.f : exp2f(mB - MnB);
-          sb8 = b8 == -INFINITY ? 0.f : exp2f(b8 - Mn8); sw8 = m_ref == -INFINITY ? 0.f : exp2f(m_ref - Mn8);
         }
         __syncwarp();                                  // every lane has read the old maxima
-        if (t4 == 0) {
-          mrg_l[g8] = (w > 0 ? mrg_l[g8] * sb8 : 0.f) + l * sw8;
-          mrg_m[g8] = Mn8;
+        if (g8 == 0) {
+          mrg_l[2 * t4] = (w > 0 ? mrg_l[2 * t4] * sbA : 0.f) + lA * swA;
+          mrg_l[2 * t4 + 1] = (w > 0 ? mrg_l[2 * t4 + 1] * sbB : 0.f) + lB * swB;
+          mrg_m[2 * t4] = MnA;
+          mrg_m[2 * t4 + 1] = MnB;
         }
         if (HAS_V) {
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const int d0 = 64 * (j >> 2) + 8 * g8 + 2 * (j & 3);
-            float2* pa = reinterpret_cast<float2*>(mrg_o + (2 * t4) * kHeadDim + d0);
-            float2* pb = reinterpret_cast<float2*>(mrg_o + (2 * t4 + 1) * kHeadDim + d0);
-            float2 va = make_float2(0.f, 0.f), vb = make_float2(0.f, 0.f);
-            if (w > 0) { va = *pa; vb = *pb; }
-            *pa = make_float2(va.x * sbA + o[j][0] * swA, va.y * sbA + o[j][2] * swA);
-            *pb = make_float2(vb.x * sbB + o[j][1] * swB, vb.y * sbB + o[j][3] * swB);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {              // (dim 16 j + 8 (i >> 1) + g8, head 2 t4 + (i & 1)): 32 distinct banks
+              float* pa = mrg_o + (2 * t4 + (i & 1)) * kMergePitch + 16 * j + 8 * (i >> 1) + g8;
+              const float old = w > 0 ? *pa : 0.f;
+              *pa = old * ((i & 1) ? sbB : sbA) + o[j][i] * ((i & 1) ? swB : swA);
+            }
           }
         }
       }
@@ -593,8 +600,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
         M[it] = mrg_m[h];
         den[it] = mrg_l[h];
         if (HAS_V) {
-          const float4 x0 = *reinterpret_cast<const float4*>(mrg_o + h * kHeadDim + d8);
-          const float4 x1 = *reinterpret_cast<const float4*>(mrg_o + h * kHeadDim + d8 + 4);
+          const float4 x0 = *reinterpret_cast<const float4*>(mrg_o + h * kMergePitch + d8);
+          const float4 x1 = *reinterpret_cast<const float4*>(mrg_o + h * kMergePitch + d8 + 4);
           num[it][0] = x0.x; num[it][1] = x0.y; num[it][2] = x0.z; num[it][3] = x0.w;
           num[it][4] = x1.x; num[it][5] = x1.y; num[it][6] = x1.z; num[it][7] = x1.w;
         }
@@ -759,10 +766,10 @@ __global__ void __launch_bounds__(kFinalizeThreads) scores_finalize_kernel(
 #pragma unroll
     for (int j = 0; j < 4; ++j) x[j] = lp[static_cast<int64_t>(h + j) * n_stride_logits];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) s += exp2f(x[j] - st[2 * (h + j)]) * st[2 * (h + j) + 1];
+    for (int j = 0; j < 4; ++j) s = score_add_head(s, x[j], st[2 * (h + j)], st[2 * (h + j) + 1]);
   }
-  for (; h < num_q_heads; ++h) s += exp2f(lp[static_cast<int64_t>(h) * n_stride_logits] - st[2 * h]) * st[2 * h + 1];
-  scores[static_cast<int64_t>(b) * n_stride + i] = s / static_cast<float>(num_q_heads);
+  for (; h < num_q_heads; ++h) s = score_add_head(s, lp[static_cast<int64_t>(h) * n_stride_logits], st[2 * h], st[2 * h + 1]);
+  scores[static_cast<int64_t>(b) * n_stride + i] = score_finish(s, num_q_heads);
 }
 
 __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restrict__ scores, int n_stride,

@@ -12,6 +12,7 @@ constexpr int kAttnCtasPerSm = 4;     // resident CTAs per SM (shared memory); a
 constexpr int kMaxUnits = 512;        // sequences x KV heads per launch (their row prefix lives in shared memory)
 constexpr int kMaxPartsPerUnit = 16;  // CTAs sharing one unit in split mode (bounds the last CTA's merge)
 constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
+constexpr int kTopkMaxHeads = 128;    // query heads the selection kernel can score by itself
 
 // Programmatic dependent launch. Every kernel of this library is launched with the "programmatic
 // stream serialization" attribute and (i) lets its successor's CTAs be scheduled as soon as SM
@@ -44,6 +45,17 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
+#endif
+
+#ifdef __CUDACC__
+// One head's term of a focal score (Section 3.1.1: post-softmax weight, averaged over heads):
+// logit and maximum in the log2 domain, inv_sum = 1 / softmax denominator. Heads are added in
+// ascending order and the total divided by H; every kernel that forms scores goes through these
+// two functions, so that they all produce the same bits.
+__device__ __forceinline__ float score_add_head(float acc, float logit, float max_log2, float inv_sum) {
+  return acc + exp2f(logit - max_log2) * inv_sum;
+}
+__device__ __forceinline__ float score_finish(float acc, int num_q_heads) { return acc / static_cast<float>(num_q_heads); }
 #endif
 
 // AttnLaunch::wait_point
@@ -99,8 +111,11 @@ cudaError_t launch_scores_finalize(const float* logits, const float* stats, cons
 cudaError_t launch_image_mass(const float* scores, int32_t n_stride, const int32_t* vis_len, int32_t batch,
                               float* mass, cudaStream_t s);
 
+// Scores come either from `scores` ([B][n_stride]) or, when `logits` is not NULL, are formed on the fly
+// from the attention kernel's logits ([B][H][n_stride_logits]) and per-head (max, sum) statistics.
 cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int32_t* vis_len, const int32_t* k,
                                int32_t batch, int32_t max_vis_len, int32_t* idx_out, int32_t k_stride,
+                               const float* logits, const float* stats, int32_t num_q_heads, int32_t n_stride_logits,
                                cudaStream_t s);
 
 cudaError_t configure_kernels();   // one-time cudaFuncSetAttribute calls (current device)

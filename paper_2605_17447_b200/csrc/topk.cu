@@ -34,8 +34,12 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* __restrict__ scores, int n_stride,
                                                                    const int32_t* __restrict__ vis_len,
                                                                    const int32_t* __restrict__ kreq,
-                                                                   int32_t* __restrict__ idx_out, int k_stride, int n_cap) {
+                                                                   int32_t* __restrict__ idx_out, int k_stride, int n_cap,
+                                                                   const float* __restrict__ logits,
+                                                                   const float* __restrict__ stats, int num_q_heads,
+                                                                   int n_stride_logits) {
   extern __shared__ uint32_t keys[];                    // this CTA's slice of the keys
+  __shared__ float head_st[2 * kTopkMaxHeads];          // scoring mode: per head (max, 1 / sum)
   __shared__ uint32_t hist[256];                        // this CTA's histogram (read by the whole cluster)
   __shared__ uint32_t hist_all[256];                    // cluster totals
   __shared__ uint32_t warp_gt[kTopkWarps], warp_eq[kTopkWarps];
@@ -58,8 +62,56 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   const int per_cta = (((N + C - 1) / C) + 31) & ~31;
   const int lo_i = min(c * per_cta, N), hi_i = min(lo_i + per_cta, N);
   const int n_loc = hi_i - lo_i;
-  const float* sp = scores + static_cast<int64_t>(b) * n_stride + lo_i;
-  for (int i = tid; i < n_loc; i += kTopkThreads) keys[i] = score_key(sp[i]);
+  if (logits == nullptr) {
+    const float* sp = scores + static_cast<int64_t>(b) * n_stride + lo_i;
+    for (int i = tid; i < n_loc; i += kTopkThreads) keys[i] = score_key(sp[i]);
+  } else {
+    // Scores formed here from the focal layer's logits (the same arithmetic as the stand-alone
+    // scoring kernel, head by head in ascending order): four tokens per thread, eight heads' loads
+    // in flight. The logits were written by the kernel just before and are read from L2.
+    for (int i = tid; i < num_q_heads; i += kTopkThreads) {
+      head_st[2 * i] = stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2];
+      head_st[2 * i + 1] = 1.0f / stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2 + 1];
+    }
+    __syncthreads();
+    const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + lo_i;
+    const bool vec = (n_stride_logits & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;   // lo_i is a multiple of 32
+    for (int i0 = tid * 4; i0 < n_loc; i0 += kTopkThreads * 4) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      const bool full = vec && i0 + 4 <= n_loc;
+      for (int h0 = 0; h0 < num_q_heads; h0 += 8) {
+        float4 x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          x[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (h0 + j < num_q_heads) {
+            const float* src = lp + static_cast<int64_t>(h0 + j) * n_stride_logits + i0;
+            if (full) {
+              x[j] = __ldcg(reinterpret_cast<const float4*>(src));
+            } else {
+              x[j].x = __ldcg(src);
+              if (i0 + 1 < n_loc) x[j].y = __ldcg(src + 1);
+              if (i0 + 2 < n_loc) x[j].z = __ldcg(src + 2);
+              if (i0 + 3 < n_loc) x[j].w = __ldcg(src + 3);
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (h0 + j < num_q_heads) {
+            const float m = head_st[2 * (h0 + j)], inv = head_st[2 * (h0 + j) + 1];
+            acc[0] = score_add_head(acc[0], x[j].x, m, inv);
+            acc[1] = score_add_head(acc[1], x[j].y, m, inv);
+            acc[2] = score_add_head(acc[2], x[j].z, m, inv);
+            acc[3] = score_add_head(acc[3], x[j].w, m, inv);
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (i0 + j < n_loc) keys[i0 + j] = score_key(score_finish(acc[j], num_q_heads));
+    }
+  }
   if (tid == 0) {
     sel_prefix = 0u;
     sel_remaining = static_cast<uint32_t>(k);
@@ -207,8 +259,10 @@ cudaError_t configure_topk() {
 
 cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int32_t* vis_len, const int32_t* k,
                                int32_t batch, int32_t max_vis_len, int32_t* idx_out, int32_t k_stride,
+                               const float* logits, const float* stats, int32_t num_q_heads, int32_t n_stride_logits,
                                cudaStream_t s) {
   if (batch <= 0 || max_vis_len <= 0) return cudaSuccess;
+  if (logits != nullptr && (num_q_heads <= 0 || num_q_heads > kTopkMaxHeads)) return cudaErrorInvalidValue;
   // cluster size: enough CTAs to cover the GPU for small batches, at least 1024 keys per CTA
   int device = 0, sms = 148;
   if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
@@ -230,7 +284,8 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   const cudaError_t e = cudaLaunchKernelEx(&cfg, select_topk_kernel, scores, n_stride, vis_len, k, idx_out, k_stride,
-                                           static_cast<int>(max_vis_len));
+                                           static_cast<int>(max_vis_len), logits, stats, static_cast<int>(num_q_heads),
+                                           static_cast<int>(n_stride_logits));
   count_launches(1);
   return e;
 }
