@@ -38,6 +38,7 @@ struct fastocr_ctx {
   int dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
   int sparse_ctas_per_sm = fastocr::kAttnCtasPerSm - 1;
   int sparse_trigger_q8 = 0;
+  int dense_depth = 2, sparse_depth = 3;
   unsigned long long* trace = nullptr;   // set only by debug builds
   unsigned trace_seq = 0;
   char err[512] = {0};
@@ -127,6 +128,7 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
 #endif
   a.wait_point = fastocr::kWaitAtStart;
   a.trigger_q8 = 0;
+  a.depth = ctx->dense_depth;
   a.grid_ctas = ctx->sm_count * ctx->dense_ctas_per_sm;
   {
     // small batches: the kernel gives every unit at most kMaxPartsPerUnit CTAs; launch no more
@@ -255,6 +257,7 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
     a.active_ctas = a.grid_ctas;
   }
   a.wait_point = wait_point;
+  a.depth = ctx->sparse_depth;
   a.trigger_q8 = ctx->sparse_trigger_q8;   // the next layer's pruned pass sets up while this one is in mid-stream
   a.out = out;
   a.out_is_fp32 = out_is_fp32;
@@ -300,6 +303,8 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   // one partial slot per (CTA, unit) pair that can occur: CTAs + units
   if (const char* v = std::getenv("FASTOCR_DENSE_CTAS_PER_SM")) ctx->dense_ctas_per_sm = std::atoi(v);     // tuning knobs,
   if (const char* v = std::getenv("FASTOCR_SPARSE_CTAS_PER_SM")) ctx->sparse_ctas_per_sm = std::atoi(v);   // read once here
+  if (const char* v = std::getenv("FASTOCR_DENSE_DEPTH")) ctx->dense_depth = std::atoi(v);
+  if (const char* v = std::getenv("FASTOCR_SPARSE_DEPTH")) ctx->sparse_depth = std::atoi(v);
   if (const char* v = std::getenv("FASTOCR_SPARSE_TRIGGER_Q8")) ctx->sparse_trigger_q8 = std::atoi(v);
   if (ctx->sparse_trigger_q8 < 0 || ctx->sparse_trigger_q8 > 256) ctx->sparse_trigger_q8 = 0;
   if (ctx->dense_ctas_per_sm < 1 || ctx->dense_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->dense_ctas_per_sm = fastocr::kAttnCtasPerSm;

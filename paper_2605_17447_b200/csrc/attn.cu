@@ -62,8 +62,20 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+// Cache rows are read once per layer: they go through L2 marked evict-first, so that streaming a
+// gigabyte of them does not push out what is read again soon (the logits of a focal layer, the
+// index list, the queries).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint64_t policy) {
+#ifdef FASTOCR_NO_EVICT_FIRST
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+#else
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
+#endif
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -167,8 +179,10 @@ __device__ __forceinline__ unsigned long long trace_now() {
 #define FASTOCR_TRACE_ADD(acc, t1, t0) do { } while (0)
 #endif
 
-template <int G, bool HAS_V>
+// kDepth: how many blocks ahead of its use a copy is issued (1 .. kStages)
+template <int G, bool HAS_V, int kDepth>
 __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(const AttnLaunch a) {
+  static_assert(kDepth >= 1 && kDepth <= kStages, "copy distance");
   extern __shared__ __align__(16) unsigned char smem[];
   using L = Smem<HAS_V>;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -293,6 +307,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   const uint32_t smem_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
   const uint32_t ring_warp = smem_u32 + L::ring + warp * kStages * L::kStageBytes;
   const bool head_ok = g8 < G;
+  const uint64_t stream_policy = l2_evict_first_policy();
 #ifdef FASTOCR_TRACE
   if (a.trace != nullptr && lane == 0) {               // slot 2: the SM this CTA runs on
     unsigned smid;
@@ -402,19 +417,37 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
         row = pos;
       }
     };
-    auto stage_i = [&](int r, int row) {
+    // The copies of a block: its 16 K rows are one cp.async group, its 16 V rows another (K is
+    // needed at the top of the block's iteration, V only after the softmax, and each tile's ring
+    // slot is free again as soon as the fragments of the block that used it last are in registers).
+    auto stage_ik = [&](int r, int row) {
       if (r < seg_rows && tok0 + r * kRowTokens < sg.n_tok) {
         const uint32_t dst = ring_warp + (r % kStages) * L::kStageBytes;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {                  // rows 2i (lanes 0-15) and 2i + 1 (lanes 16-31)
           const int tok = 2 * i + half;
           const int64_t roff = __shfl_sync(0xffffffffu, row, tok) * row_elems;
-          cp_async16(dst + tok * 256 + ((c16 ^ row_swz(tok)) << 4), kptr + roff);
-          if (HAS_V) cp_async16(dst + L::kTileBytes + tok * 256 + ((c16 ^ row_swz(tok)) << 4), vptr + roff);
+          cp_async16(dst + tok * 256 + ((c16 ^ row_swz(tok)) << 4), kptr + roff, stream_policy);
         }
       }
       cp_async_commit();
     };
+    auto stage_iv = [&](int r, int row) {
+      if (!HAS_V) return;
+      if (r < seg_rows && tok0 + r * kRowTokens < sg.n_tok) {
+        const uint32_t dst = ring_warp + (r % kStages) * L::kStageBytes + L::kTileBytes;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int tok = 2 * i + half;
+          const int64_t roff = __shfl_sync(0xffffffffu, row, tok) * row_elems;
+          cp_async16(dst + tok * 256 + ((c16 ^ row_swz(tok)) << 4), vptr + roff, stream_policy);
+        }
+      }
+      cp_async_commit();
+    };
+    // groups younger than the one waited for: K(n) at the top of iteration n, V(n) before P.V
+    constexpr int kWaitK = HAS_V ? 2 * kDepth - 1 : kDepth - 1;
+    constexpr int kWaitV = 2 * kDepth - 1;
     // Address translation: a pruned pass touches a handful of rows in every 2 MiB page of the
     // sequence's cache span, and the first touch of a page by this SM costs a translation miss in
     // the middle of the stream. Touch every page of the span now, all at once (one line each, L2
@@ -428,24 +461,33 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       if (off >= 0 && off < span && (HAS_V || half == 0)) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
     }
     // Filling the stages: the lookups of the first rows are issued together (one round trip for
-    // the index-list entries of rows 0-3, one for the block-table entries of rows 0-2) instead of
-    // one after the other, then the copies of rows 0 and 1 go out.
+    // the index-list entries, one for the block-table entries) instead of one after the other,
+    // then the copies of the first kDepth rows go out.
     int pos_p = 0, row_p = 0;
     bool idx_p = false;
     FASTOCR_TRACE_CYC(11);
     {
-      int pos0 = 0, pos1 = 0, pos2 = 0, row0 = 0, row1 = 0;
-      bool ix0, ix1, ix2;
-      stage_p(0, pos0, ix0);
-      stage_p(1, pos1, ix1);
-      stage_p(2, pos2, ix2);
-      stage_p(3, pos_p, idx_p);
-      stage_r(0, pos0, ix0, row0);
-      stage_r(1, pos1, ix1, row1);
-      stage_r(2, pos2, ix2, row_p);
+      int posq[kDepth + 2], rowq[kDepth + 1];
+      bool ixq[kDepth + 2];
+#pragma unroll
+      for (int r = 0; r < kDepth + 2; ++r) {
+        posq[r] = 0;
+        stage_p(r, posq[r], ixq[r]);
+      }
+#pragma unroll
+      for (int r = 0; r < kDepth + 1; ++r) {
+        rowq[r] = 0;
+        stage_r(r, posq[r], ixq[r], rowq[r]);
+      }
       FASTOCR_TRACE_CYC(12);
-      stage_i(0, row0);
-      stage_i(1, row1);
+#pragma unroll
+      for (int r = 0; r < kDepth; ++r) {
+        stage_ik(r, rowq[r]);
+        stage_iv(r, rowq[r]);
+      }
+      row_p = rowq[kDepth];
+      pos_p = posq[kDepth + 1];
+      idx_p = ixq[kDepth + 1];
       FASTOCR_TRACE_CYC(13);
     }
 #pragma unroll 1
@@ -453,8 +495,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       if (seg_begin + n == trigger_row) dependents_may_launch();
       const int j0 = tok0 + n * kRowTokens;
       FASTOCR_TRACE_CLK(c_top);
-      cp_async_wait<kStages - 2>();
-      __syncwarp();                                    // every lane's copies of this block have landed
+      cp_async_wait<kWaitK>();
+      __syncwarp();                                    // every lane's K copies of this block have landed
       FASTOCR_TRACE_CLK(c_waited);
       FASTOCR_TRACE_ADD(trace_wait, c_waited, c_top);
       if (n == 0) { FASTOCR_TRACE_MARK(3); FASTOCR_TRACE_CYC(14); }
@@ -476,11 +518,13 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       }
       FASTOCR_TRACE_CLK(c_qk);
       FASTOCR_TRACE_ADD(trace_qk, c_qk, c_waited);
-      // ---- stages I, R, P for rows n + 2, n + 3, n + 4 (the ring slot of row n + 2 is the one row
-      // n - 1 was read from; the __syncwarp above separates those reads from these writes) -------
-      stage_i(n + 2, row_p);
-      stage_r(n + 3, pos_p, idx_p, row_p);
-      stage_p(n + 4, pos_p, idx_p);
+      // ---- look-ahead: K copies of block n + kDepth into the slot block n's K tile just left, then
+      // stages R and P one and two blocks further ---------------------------------------------------
+      __syncwarp();                                    // every lane has this block's K fragments
+      stage_ik(n + kDepth, row_p);
+      const int row_v = row_p;
+      stage_r(n + kDepth + 1, pos_p, idx_p, row_p);
+      stage_p(n + kDepth + 2, pos_p, idx_p);
 
       FASTOCR_TRACE_CLK(c_look);
       FASTOCR_TRACE_ADD(trace_look, c_look, c_qk);
@@ -532,16 +576,22 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           const uint32_t r0w = pack_bf16(p[0] - __uint_as_float(h0 << 16), p[1] - __uint_as_float(h0 & 0xffff0000u));
           const uint32_t r1w = pack_bf16(p[2] - __uint_as_float(h1 << 16), p[3] - __uint_as_float(h1 & 0xffff0000u));
           const uint32_t ph0 = movm_trans(h0), ph1 = movm_trans(h1), pl0 = movm_trans(r0w), pl1 = movm_trans(r1w);
+          cp_async_wait<kWaitV>();
+          __syncwarp();                                // every lane's V copies of this block have landed
           const uint32_t vt = src + L::kTileBytes + v_lm;
+          uint32_t va[8][4];                           // A fragments of V^T: dims 16 j .. + 15 x the block's 16 tokens
+#pragma unroll
+          for (int j = 0; j < 8; ++j) ldsm_x4_trans(va[j], vt + (((2 * j + v_lm_c) ^ lm_r) << 4));
+          __syncwarp();                                // the V tile's slot is free: copies of block n + kDepth
+          stage_iv(n + kDepth, row_v);                 // go out while the tensor cores work
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            uint32_t va[4];                            // A fragment of V^T: dims 16 j .. + 15 x the block's 16 tokens
-            ldsm_x4_trans(va, vt + (((2 * j + v_lm_c) ^ lm_r) << 4));
-            mma_bf16(o[j], va[0], va[1], va[2], va[3], ph0, ph1);
-            mma_bf16(o[j], va[0], va[1], va[2], va[3], pl0, pl1);
+            mma_bf16(o[j], va[j][0], va[j][1], va[j][2], va[j][3], ph0, ph1);
+            mma_bf16(o[j], va[j][0], va[j][1], va[j][2], va[j][3], pl0, pl1);
           }
         }
       }
+      if (HAS_V && !live) stage_iv(n + kDepth, row_v);   // keeps the group count in step (nothing to copy any more)
       FASTOCR_TRACE_CLK(c_end);
       FASTOCR_TRACE_ADD(trace_pv, c_end, c_look);
     }
@@ -792,20 +842,20 @@ __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restric
   }
 }
 
-template <int G, bool HAS_V>
+template <int G, bool HAS_V, int DEPTH>
 cudaError_t launch_partial_t(const AttnLaunch& a, cudaStream_t s) {
-  const cudaError_t e = launch_pdl(attn_stream_kernel<G, HAS_V>, dim3(a.grid_ctas), dim3(kThreads), Smem<HAS_V>::total, s, a);
+  const cudaError_t e = launch_pdl(attn_stream_kernel<G, HAS_V, DEPTH>, dim3(a.grid_ctas), dim3(kThreads), Smem<HAS_V>::total, s, a);
   count_launches(1);
   return e;
 }
 
-template <int G, bool HAS_V>
+template <int G, bool HAS_V, int DEPTH>
 cudaError_t configure_t() {
-  cudaError_t e = cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V, DEPTH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        Smem<HAS_V>::total);
   if (e != cudaSuccess) return e;
   // all of the SM's L1/shared array as shared memory: four CTAs must fit
-  return cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+  return cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V, DEPTH>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
 }
 
 }  // namespace
@@ -816,9 +866,10 @@ cudaError_t launch_attn_partial(const AttnLaunch& a, cudaStream_t s) {
   const int G = a.num_q_heads / a.num_kv_heads;
   const bool has_v = a.v != nullptr;
   switch (G) {
-#define X(g) \
-  case g:    \
-    return has_v ? launch_partial_t<g, true>(a, s) : launch_partial_t<g, false>(a, s);
+#define X(g)                                                                                  \
+  case g:                                                                                     \
+    if (!has_v) return launch_partial_t<g, false, 2>(a, s);                                   \
+    return a.depth >= 3 ? launch_partial_t<g, true, 3>(a, s) : launch_partial_t<g, true, 2>(a, s);
     FASTOCR_FOR_EACH_GROUP(X)
 #undef X
     default:
@@ -832,9 +883,10 @@ cudaError_t configure_kernels() {
   // kernels in between do not trigger a reconfiguration
   if ((e = cudaFuncSetAttribute(scores_finalize_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(image_mass_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
-#define X(g)                                                \
-  if ((e = configure_t<g, true>()) != cudaSuccess) return e; \
-  if ((e = configure_t<g, false>()) != cudaSuccess) return e;
+#define X(g)                                                   \
+  if ((e = configure_t<g, true, 2>()) != cudaSuccess) return e;  \
+  if ((e = configure_t<g, true, 3>()) != cudaSuccess) return e;  \
+  if ((e = configure_t<g, false, 2>()) != cudaSuccess) return e;
   FASTOCR_FOR_EACH_GROUP(X)
 #undef X
   return cudaSuccess;
@@ -844,9 +896,9 @@ cudaError_t configure_kernels() {
 // debug builds: resident CTAs per SM the runtime grants the 7-head attention kernel
 extern "C" int fastocr_debug_occupancy() {
   int n = -1;
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_stream_kernel<7, true>, kThreads, Smem<true>::total);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_stream_kernel<7, true, 2>, kThreads, Smem<true>::total);
   cudaFuncAttributes fa;
-  cudaFuncGetAttributes(&fa, attn_stream_kernel<7, true>);
+  cudaFuncGetAttributes(&fa, attn_stream_kernel<7, true, 2>);
   return n * 1000 + fa.numRegs;
 }
 #endif

@@ -3,9 +3,9 @@
 // One thread-block cluster per sequence (1, 2, 4 or 8 CTAs, chosen so that a launch fills the GPU
 // even for small batches); CTA c of the cluster owns the contiguous slice c of the sequence's
 // scores. The scores are mapped to order-preserving 32-bit keys held in shared memory, the key of
-// the k-th largest score is found with a four-pass MSB-first radix select (8 bits per pass: every
-// CTA histograms its slice, the 256 bin totals are summed across the cluster through distributed
-// shared memory, and every CTA walks the same totals), and the result is emitted by an in-order
+// the k-th largest score is found with a three-pass MSB-first radix select (digits of 11, 11 and 10
+// bits: every CTA histograms its slice, the bin totals are summed across the cluster through
+// distributed shared memory, and every CTA scans the same totals), and the result is emitted by an in-order
 // compaction: every key above the threshold, plus the first r keys equal to it, where r is what is
 // left of k. Walking the indices in ascending order gives both the "lower index wins ties" rule
 // and the ascending output order with no sort; a CTA learns how many selected keys precede its
@@ -22,6 +22,8 @@ namespace {
 constexpr int kTopkThreads = 1024;
 constexpr int kTopkWarps = kTopkThreads / 32;
 constexpr int kTopkMaxCluster = 8;
+constexpr int kTopkBins = 2048;                         // 11-bit digits; two bins per thread
+static_assert(kTopkBins == 2 * kTopkThreads, "the bin scan gives every thread two bins");
 
 // larger float <=> larger key; -0 == +0; NaN below everything.
 __device__ __forceinline__ uint32_t score_key(float s) {
@@ -40,8 +42,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
                                                                    int n_stride_logits) {
   extern __shared__ uint32_t keys[];                    // this CTA's slice of the keys
   __shared__ float head_st[2 * kTopkMaxHeads];          // scoring mode: per head (max, 1 / sum)
-  __shared__ uint32_t hist[256];                        // this CTA's histogram (read by the whole cluster)
-  __shared__ uint32_t hist_all[256];                    // cluster totals
+  __shared__ uint32_t hist_buf[2][kTopkBins];           // this CTA's digit histograms (read by the whole cluster)
   __shared__ uint32_t warp_gt[kTopkWarps], warp_eq[kTopkWarps];
   __shared__ uint32_t slice_tot[2];                     // selected-candidate counts of this slice: above, equal
   __shared__ uint32_t sel_prefix, sel_remaining;
@@ -112,71 +113,81 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
         if (i0 + j < n_loc) keys[i0 + j] = score_key(score_finish(acc[j], num_q_heads));
     }
   }
+  hist_buf[0][2 * tid] = hist_buf[0][2 * tid + 1] = 0u;
+  hist_buf[1][2 * tid] = hist_buf[1][2 * tid + 1] = 0u;
   if (tid == 0) {
     sel_prefix = 0u;
     sel_remaining = static_cast<uint32_t>(k);
   }
+  __syncthreads();
 
-  // ---- radix select: after pass p the top 8(p+1) bits of the k-th largest key are known -------
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    if (tid < 256) hist[tid] = 0u;
-    __syncthreads();
+  // ---- radix select, three passes over digits of 11, 11 and 10 bits (most significant first) ----
+  // Pass p: every CTA histograms the digit of those of its keys that match the prefix found so far;
+  // after one cluster barrier thread t adds up bins 2t and 2t + 1 (counted from the largest digit)
+  // of all CTAs through distributed shared memory, and a block-wide scan finds the digit at which
+  // the running count from the top reaches what is left of k. The two histogram buffers alternate,
+  // so the buffer of pass p is cleared during pass p + 1, behind that pass's barrier.
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+    const uint32_t digit_mask = pass == 2 ? 0x3ffu : 0x7ffu;
+    const uint32_t hi_mask = pass == 0 ? 0u : (0xffffffffu << (pass == 1 ? 21 : 10));
+    uint32_t* hist = hist_buf[pass & 1];
     const uint32_t prefix = sel_prefix;
     const uint32_t remaining = sel_remaining;
-    const uint32_t hi_mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
     for (int base = warp * 32; base < n_loc; base += kTopkThreads) {   // warp-uniform trip count
       const int i = base + lane;
       const uint32_t key = i < n_loc ? keys[i] : 0u;
       const bool in = i < n_loc && (key & hi_mask) == prefix;
-      const uint32_t digit = (key >> shift) & 0xffu;
+      const uint32_t digit = (key >> shift) & digit_mask;
       if (pass == 0) {
-        // the leading byte (sign and most of the exponent) is heavily clustered: aggregate
-        // identical digits inside the warp before touching shared memory
+        // the leading bits (sign, exponent) are heavily clustered: aggregate identical digits
+        // inside the warp before touching shared memory
         const uint32_t active = __ballot_sync(0xffffffffu, in);
         if (in) {
           const uint32_t peers = __match_any_sync(active, digit);
           if ((__ffs(peers) - 1) == lane) atomicAdd(&hist[digit], __popc(peers));
         }
-      } else if (in) {                                  // later bytes are spread out and few keys are left
+      } else if (in) {                                  // later digits are spread out and few keys are left
         atomicAdd(&hist[digit], 1u);
       }
     }
     cluster.sync();                                     // every slice's histogram is complete
-    if (tid < 256) {
-      uint32_t t = 0;
-      for (int r = 0; r < C; ++r) t += *cluster.map_shared_rank(&hist[tid], r);
-      hist_all[tid] = t;
+    // bins in descending digit order: thread t owns digits 2047 - 2t and 2046 - 2t
+    const int d0 = kTopkBins - 1 - 2 * tid, d1 = d0 - 1;
+    uint32_t c0 = 0, c1 = 0;
+    for (int r = 0; r < C; ++r) {
+      const uint32_t* h = cluster.map_shared_rank(hist, r);
+      c0 += h[d0];
+      c1 += h[d1];
     }
-    cluster.sync();                                     // totals read: the histograms may be cleared again
-    // one warp walks the bins from the top: find the digit where the running count reaches k
-    if (warp == 0) {
-      uint32_t above = 0;                               // keys with a larger digit
-      uint32_t found_digit = 0, found_above = 0;
-      bool found = false;
-      for (int base = 224; base >= 0 && !found; base -= 32) {
-        const uint32_t cnt = hist_all[base + (31 - lane)];   // lane 0 holds the largest digit of the group
-        uint32_t incl = cnt;                            // inclusive scan, largest digit first
+    hist_buf[(pass + 1) & 1][2 * tid] = 0u;             // last read (by anyone) before the barrier above
+    hist_buf[(pass + 1) & 1][2 * tid + 1] = 0u;
+    const uint32_t local = c0 + c1;
+    uint32_t incl = local;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-          if (lane >= o) incl += t;
-        }
-        const bool hit = above + incl >= remaining;
-        const uint32_t hits = __ballot_sync(0xffffffffu, hit);
-        if (hits) {
-          const int src = __ffs(hits) - 1;
-          found_digit = base + (31 - src);
-          found_above = above + __shfl_sync(0xffffffffu, incl - cnt, src);
-          found = true;
-        } else {
-          above += __shfl_sync(0xffffffffu, incl, 31);
-        }
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_gt[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t w = warp_gt[lane];
+      uint32_t wi = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += t;
       }
-      if (lane == 0) {
-        sel_prefix = prefix | (found_digit << shift);
-        sel_remaining = remaining - found_above;
-      }
+      warp_eq[lane] = wi - w;                           // keys in the warps before this one
+    }
+    __syncthreads();
+    const uint32_t before = warp_eq[warp] + incl - local;   // keys with a larger digit than d0
+    if (before < remaining && remaining <= before + local) {   // exactly one thread
+      const bool first = before + c0 >= remaining;
+      const uint32_t found_digit = first ? d0 : d1;
+      sel_prefix = prefix | (found_digit << shift);
+      sel_remaining = remaining - (first ? before : before + c0);
     }
     __syncthreads();
   }
