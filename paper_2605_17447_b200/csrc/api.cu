@@ -253,7 +253,6 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
       if (parts > fastocr::kMaxPartsPerUnit) parts = fastocr::kMaxPartsPerUnit;
       a.grid_ctas = units * parts;
     }
-    if (const char* v = std::getenv("FASTOCR_SPARSE_GRID")) a.grid_ctas = std::atoi(v);   // EXPERIMENT
     a.active_ctas = a.grid_ctas;
   }
   a.wait_point = wait_point;

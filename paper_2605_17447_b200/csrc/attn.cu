@@ -71,11 +71,7 @@ __device__ __forceinline__ uint64_t l2_evict_first_policy() {
   return p;
 }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint64_t policy) {
-#ifdef FASTOCR_NO_EVICT_FIRST
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-#else
   asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
-#endif
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
