@@ -453,12 +453,16 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
     fastocr_status st;
     if (focal || (l == 0 && !have)) {
       // full attention + scoring + selection; the refreshed set replaces the current one.
-      // The logits workspace is written from the first block on: wait before the stream starts.
+      // The logits workspace is written from the first block on, and its last reader was the
+      // previous selection kernel. Right after that kernel the stream must wait for it; once an
+      // attention kernel lies in between, that kernel waited for the selection before it let
+      // anything else start, so this launch may stream at once, beside the draining pruned pass.
       // The selection kernel forms the scores from the logits itself (no score array, one launch
       // less) unless there are more heads than it has room for.
       const bool fused = layers[l].num_q_heads <= fastocr::kTopkMaxHeads;
       st = dense_impl(ctx, &layers[l], ql, ol, out_is_fp32, fused ? nullptr : ctx->scores, ctx->lim.max_vis_len, max_vis_len,
-                      chained ? fastocr::kWaitAfterSetup : fastocr::kWaitAtStart, s, fused);
+                      !chained ? fastocr::kWaitAtStart : (prev == kAttention ? fastocr::kWaitBeforeWrites : fastocr::kWaitAfterSetup),
+                      s, fused);
       if (st != FASTOCR_OK) return st;
       {
         ProfScope p(ctx, FASTOCR_PROF_TOPK, s);
