@@ -37,7 +37,6 @@ struct fastocr_ctx {
   // a pruned pass leaves one free (so that the next layer's launch can start beside it)
   int dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
   int sparse_ctas_per_sm = fastocr::kAttnCtasPerSm - 1;
-  int sparse_trigger_q8 = 0;
   int dense_depth = 2, sparse_depth = 3;
   unsigned long long* trace = nullptr;   // set only by debug builds
   unsigned trace_seq = 0;
@@ -127,7 +126,6 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
   a.trace = nullptr;
 #endif
   a.wait_point = fastocr::kWaitAtStart;
-  a.trigger_q8 = 0;
   a.depth = ctx->dense_depth;
   a.grid_ctas = ctx->sm_count * ctx->dense_ctas_per_sm;
   {
@@ -257,7 +255,6 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
   }
   a.wait_point = wait_point;
   a.depth = ctx->sparse_depth;
-  a.trigger_q8 = ctx->sparse_trigger_q8;   // the next layer's pruned pass sets up while this one is in mid-stream
   a.out = out;
   a.out_is_fp32 = out_is_fp32;
   {
@@ -304,8 +301,6 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   if (const char* v = std::getenv("FASTOCR_SPARSE_CTAS_PER_SM")) ctx->sparse_ctas_per_sm = std::atoi(v);   // read once here
   if (const char* v = std::getenv("FASTOCR_DENSE_DEPTH")) ctx->dense_depth = std::atoi(v);
   if (const char* v = std::getenv("FASTOCR_SPARSE_DEPTH")) ctx->sparse_depth = std::atoi(v);
-  if (const char* v = std::getenv("FASTOCR_SPARSE_TRIGGER_Q8")) ctx->sparse_trigger_q8 = std::atoi(v);
-  if (ctx->sparse_trigger_q8 < 0 || ctx->sparse_trigger_q8 > 256) ctx->sparse_trigger_q8 = 0;
   if (ctx->dense_ctas_per_sm < 1 || ctx->dense_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
   if (ctx->sparse_ctas_per_sm < 1 || ctx->sparse_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->sparse_ctas_per_sm = fastocr::kAttnCtasPerSm - 1;
   ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * fastocr::kAttnCtasPerSm +

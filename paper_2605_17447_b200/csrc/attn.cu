@@ -43,7 +43,6 @@
 
 #include <cuda_bf16.h>
 
-#include <climits>
 
 namespace fastocr {
 namespace {
@@ -196,13 +195,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   // The next kernel is let in only once this one's own early reads are known to be safe: a kernel
   // whose inputs were settled before it started says so at once, the others after their wait
   // (their successor may assume that whatever they waited for has completed).
-  // When it does so on top of that is a matter of pacing: a successor that streams the same amount
-  // of data should begin its set-up while this kernel is in mid-stream, so that one kernel's idle
-  // set-up phase falls into the other's streaming phase instead of all CTAs of the GPU setting up
-  // (memory idle) and then streaming (memory saturated) in step.
-  const bool trigger_early = a.trigger_q8 <= 0;
   if (a.wait_point == kWaitAtStart) wait_for_prior_grids();
-  if (a.wait_point != kWaitAfterSetup && trigger_early) dependents_may_launch();
+  if (a.wait_point != kWaitAfterSetup) dependents_may_launch();
 
   // ---- set-up: prefix of the units' row counts ----------------------------------------------------
   // Every thread fetches the lengths of up to kMaxUnits / kThreads units at once (one round trip to
@@ -325,10 +319,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   int seg_begin = r0;
   if (a.wait_point == kWaitAfterSetup) {               // before index-list reads and logits writes
     wait_for_prior_grids();
-    if (trigger_early) dependents_may_launch();
+    dependents_may_launch();
   }
-  // the row of this CTA's range at which it triggers (a CTA without rows triggers by exiting)
-  const int trigger_row = trigger_early ? INT_MIN : r0 + min(((r1 - r0) * min(a.trigger_q8, 256)) >> 8, r1 - r0 - 1);
 #pragma unroll 1
   while (seg_begin < r1) {
     while (prefix_s[u + 1] <= seg_begin) ++u;          // skip empty units
@@ -488,7 +480,6 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     }
 #pragma unroll 1
     for (int n = 0; n < seg_rows; ++n) {
-      if (seg_begin + n == trigger_row) dependents_may_launch();
       const int j0 = tok0 + n * kRowTokens;
       FASTOCR_TRACE_CLK(c_top);
       cp_async_wait<kWaitK>();

@@ -86,8 +86,6 @@ struct AttnLaunch {
   int32_t wait_point;         // where the kernel waits for earlier kernels: kWaitAtStart / kWaitAfterSetup / kWaitBeforeWrites
   int32_t depth;              // blocks a copy is issued ahead of its use (1..3): deeper hides more latency per warp,
                               // shallower keeps fewer requests queued when the pass saturates HBM anyway
-  int32_t trigger_q8;         // when a CTA lets the next kernel's CTAs in: 0 = as early as its wait point allows,
-                              // else after this fraction (x/256) of its own rows
   // workspace
   float* part_acc;            // [slots][8][128], slot = CTA index + unit index (unit = sequence * Hkv + KV head)
   float* part_ml;             // [slots][8][2]  (max, sum) in the log2 domain
