@@ -16,29 +16,35 @@
 // counter per unit, no spinning).
 //
 // Data path: a block's 16 K rows and 16 V rows (256 bytes each) travel HBM -> shared memory with
-// 16-byte cp.async, one full row per half-warp per instruction (so every request covers whole
-// 128-byte lines), into a per-warp ring (kStages deep; hand-off inside the warp only: one
-// __syncwarp per block). Rows are stored with their 16-byte chunks XOR-swizzled so that the
-// tensor-core fragment reads (ld.shared.v4, each lane its own chunks) are bank-conflict free.
-// Cache rows are located ahead of the copies by lanes 0-15 (one token each): first the logical
-// position (a load from the index list for selected image tokens), one block later the physical
-// row (a block-table load for paged caches), one block later the copy, so neither lookup sits on
-// the critical path. A CTA whose range covers pieces of several units handles them one after the
-// other, refilling the pipeline at each boundary.
+// 16-byte cp.async (marked evict-first in L2: cache rows are read once per layer), one full row
+// per half-warp per instruction (so every request covers whole 128-byte lines), into a per-warp
+// ring of kStages blocks (hand-off inside the warp only: __syncwarp). The K tile and the V tile of
+// a block are separate copy groups: K is waited for at the top of the block's iteration, V only
+// after the softmax, and the copies of the block kDepth ahead go out as soon as a tile's fragments
+// are in registers (K) or while the tensor cores work (V). kDepth is 3 for pruned passes (more
+// latency hidden per warp) and 2 for full-cache passes (which saturate HBM anyway and run faster
+// with fewer requests queued). Rows are stored with their 16-byte chunks XOR-swizzled by the token's
+// low three bits so that ldmatrix reads are bank-conflict free. Cache rows are located ahead of
+// the copies by lanes 0-15 (one token each): first the logical position (a load from the index
+// list for selected image tokens), one block later the physical row (a block-table load for paged
+// caches), one block later the copy, so neither lookup sits on the critical path; when a segment
+// starts, the lookups of its first blocks are issued together. A pruned pass also touches one line
+// in every 2 MiB page of its sequence's cache span at once: the address-translation misses that
+// random rows would otherwise take one by one in mid-stream are then taken in parallel. A CTA
+// whose range covers pieces of several units handles them one after the other, refilling the
+// pipeline at each boundary.
 //
 // Arithmetic: with a GQA group of 7 or 8 query heads per KV head, q.K^T and P.V are skinny matrix
 // products ([16 tokens x 128] x [128 x 8 heads]); on the fp32 CUDA cores they need more issue slots
 // than the HBM stream leaves time for, so both run on the tensor cores as warp-level
 // mma.sync.m16n8k16 (bf16 inputs, fp32 accumulation):
-//   S^T[head][token] = Q[head][d] . K^T[d][token]   (heads on M, padded to 16; 8 tokens per tile)
-//   O^T[d][head]    += V^T[d][token] . P[token][head] (16 dims per tile; 16 tokens on K)
-// The accumulator layout of S^T is exactly the B-operand layout P needs, so probabilities never
-// leave registers. bf16 products are exact in fp32; P is split into a bf16 high part and a bf16
-// remainder (two MMAs) so that the weighted sum keeps about 16 bits of P. The contraction index
-// order inside an MMA is free, which lets every fragment be a plain 16-byte row segment: K needs
-// no transposition at all, V^T is formed from pairs of rows with two byte-permutes per register.
-// The online softmax keeps a per-head running maximum that is raised only when a logit exceeds
-// it by more than 2^8, so the rescale branch is rare.
+//   S[token][head]  = K[token][d] . Q^T[d][head]      (16 tokens on M; A fragments by ldmatrix)
+//   O^T[d][head]   += V^T[d][token] . P[token][head]  (16 dims per tile; A fragments by ldmatrix.trans)
+// A lane holds the logits of two heads for two tokens; the probabilities become the B operand of
+// the second product through one movmatrix transpose per 8-token half. bf16 products are exact in
+// fp32; P is split into a bf16 high part and a bf16 remainder (two MMAs) so that the weighted sum
+// keeps about 16 bits of P. The online softmax keeps per-head running maxima that are raised only
+// when a logit exceeds them by more than 2^8, so the rescale branch is rare.
 #include "kernels.h"
 
 #include <cuda_bf16.h>
@@ -297,6 +303,24 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   const uint32_t smem_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
   const uint32_t ring_warp = smem_u32 + L::ring + warp * kStages * L::kStageBytes;
   const bool head_ok = g8 < G;
+  const int row_bytes = Hkv * kHeadDim * 2;
+  // ldmatrix row addresses inside a tile (lane l gives row l % 8 of matrix i = l / 8). K (A operand
+  // of S = K Q^T, tokens on M): matrix i = (tokens 8 (i & 1) .., chunk 2 s + (i >> 1)); V (A operand
+  // of O^T = V^T P through .trans): matrix i = (tokens 8 (i >> 1) .., chunk 2 j + (i & 1)). Steps s
+  // and s + 4 differ by 8 chunks = 128 bytes, which the swizzle (bits 0-2 of the chunk) leaves alone.
+  uint32_t k_off[4], v_off[4];
+  {
+    const int lm_r = lane & 7, lm_i = lane >> 3;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      k_off[i] = (lm_r + 8 * (lm_i & 1)) * 256 + (((2 * i + (lm_i >> 1)) ^ lm_r) << 4);
+      v_off[i] = (lm_r + 8 * (lm_i >> 1)) * 256 + (((2 * i + (lm_i & 1)) ^ lm_r) << 4);
+    }
+  }
+  // where this lane's 16-byte chunk of rows 2i + half of a tile lands (rows 2i + 8 + half: 2048 bytes further)
+  uint32_t cp_off[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) cp_off[i] = (2 * i + half) * 256 + ((c16 ^ row_swz(2 * i + half)) << 4);
   const uint64_t stream_policy = l2_evict_first_policy();
 #ifdef FASTOCR_TRACE
   if (a.trace != nullptr && lane == 0) {               // slot 2: the SM this CTA runs on
@@ -336,9 +360,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       sg = load_geom(a, b);
     }
     const int tok0 = (seg_begin - ubeg) * kRowTokens + warp * kBlockTokens;   // this warp's first token of the segment
-    const __nv_bfloat16* kptr = reinterpret_cast<const __nv_bfloat16*>(a.k) + b * seq_elems + g * kHeadDim + 8 * c16;
-    const __nv_bfloat16* vptr =
-        HAS_V ? reinterpret_cast<const __nv_bfloat16*>(a.v) + b * seq_elems + g * kHeadDim + 8 * c16 : nullptr;
+    // this lane's 16-byte chunk of cache row 0 of the unit (a row is row_bytes long)
+    const char* kptr = reinterpret_cast<const char*>(a.k) + (b * seq_elems + g * kHeadDim + 8 * c16) * 2;
+    const char* vptr = HAS_V ? reinterpret_cast<const char*>(a.v) + (b * seq_elems + g * kHeadDim + 8 * c16) * 2 : nullptr;
 
     // B fragments of Q^T for the eight 16-dim steps: head g8, dims 16 s + {2 t4, 2 t4 + 1} and 16 s + 8 + {2 t4, 2 t4 + 1}
     uint32_t qb[8][2];
@@ -361,12 +385,6 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     const bool okA = 2 * t4 < G, okB = 2 * t4 + 1 < G;
     float* logitA = (a.logits != nullptr && okA) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4) * a.n_stride : nullptr;
     float* logitB = (a.logits != nullptr && okB) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4 + 1) * a.n_stride : nullptr;
-    // ldmatrix row addresses inside a tile. K (A operand of S = K Q^T, tokens on M): matrix l / 8 =
-    // (tokens 8 (i & 1) .., chunk 2 s + (i >> 1)); V (A operand of O^T = V^T P through .trans):
-    // matrix i = (tokens 8 (i >> 1) .., chunk 2 j + (i & 1)).
-    const int lm_r = lane & 7, lm_i = lane >> 3;
-    const uint32_t k_lm = (lm_r + 8 * (lm_i & 1)) * 256, k_lm_c = lm_i >> 1;
-    const uint32_t v_lm = (lm_r + 8 * (lm_i >> 1)) * 256, v_lm_c = lm_i & 1;
 
     // Look-ahead stages, each one row behind the previous (so that no loaded value is needed in
     // the iteration that loads it): P (row n+4) logical position of token `lane` (< 16) of this
@@ -408,27 +426,23 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     // The copies of a block: its 16 K rows are one cp.async group, its 16 V rows another (K is
     // needed at the top of the block's iteration, V only after the softmax, and each tile's ring
     // slot is free again as soon as the fragments of the block that used it last are in registers).
-    auto stage_ik = [&](int r, int row) {
+    auto stage_ik = [&](int r, uint32_t dst, int row) {
       if (r < seg_rows && tok0 + r * kRowTokens < sg.n_tok) {
-        const uint32_t dst = ring_warp + (r % kStages) * L::kStageBytes;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {                  // rows 2i (lanes 0-15) and 2i + 1 (lanes 16-31)
-          const int tok = 2 * i + half;
-          const int64_t roff = __shfl_sync(0xffffffffu, row, tok) * row_elems;
-          cp_async16(dst + tok * 256 + ((c16 ^ row_swz(tok)) << 4), kptr + roff, stream_policy);
+          const int rr = __shfl_sync(0xffffffffu, row, 2 * i + half);
+          cp_async16(dst + cp_off[i & 3] + (i >> 2) * 2048, kptr + static_cast<int64_t>(rr) * row_bytes, stream_policy);
         }
       }
       cp_async_commit();
     };
-    auto stage_iv = [&](int r, int row) {
+    auto stage_iv = [&](int r, uint32_t dst, int row) {
       if (!HAS_V) return;
       if (r < seg_rows && tok0 + r * kRowTokens < sg.n_tok) {
-        const uint32_t dst = ring_warp + (r % kStages) * L::kStageBytes + L::kTileBytes;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const int tok = 2 * i + half;
-          const int64_t roff = __shfl_sync(0xffffffffu, row, tok) * row_elems;
-          cp_async16(dst + tok * 256 + ((c16 ^ row_swz(tok)) << 4), vptr + roff, stream_policy);
+          const int rr = __shfl_sync(0xffffffffu, row, 2 * i + half);
+          cp_async16(dst + L::kTileBytes + cp_off[i & 3] + (i >> 2) * 2048, vptr + static_cast<int64_t>(rr) * row_bytes, stream_policy);
         }
       }
       cp_async_commit();
@@ -470,14 +484,17 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       FASTOCR_TRACE_CYC(12);
 #pragma unroll
       for (int r = 0; r < kDepth; ++r) {
-        stage_ik(r, rowq[r]);
-        stage_iv(r, rowq[r]);
+        stage_ik(r, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
+        stage_iv(r, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
       }
       row_p = rowq[kDepth];
       pos_p = posq[kDepth + 1];
       idx_p = ixq[kDepth + 1];
       FASTOCR_TRACE_CYC(13);
     }
+    uint32_t src = ring_warp;                                          // ring slot of block n
+    uint32_t dst_ahead = ring_warp + (kDepth % kStages) * L::kStageBytes;   // ring slot of block n + kDepth
+    const uint32_t ring_end = ring_warp + kStages * L::kStageBytes;
 #pragma unroll 1
     for (int n = 0; n < seg_rows; ++n) {
       const int j0 = tok0 + n * kRowTokens;
@@ -487,7 +504,6 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       FASTOCR_TRACE_CLK(c_waited);
       FASTOCR_TRACE_ADD(trace_wait, c_waited, c_top);
       if (n == 0) { FASTOCR_TRACE_MARK(3); FASTOCR_TRACE_CYC(14); }
-      const uint32_t src = ring_warp + (n % kStages) * L::kStageBytes;
       const bool live = j0 < sg.n_tok;         // the block holds at least one attended token
       // two accumulators (even / odd 16-dim steps): dependent MMA chains of four
       float sc[4] = {0.f, 0.f, 0.f, 0.f}, sc2[4] = {0.f, 0.f, 0.f, 0.f};
@@ -496,7 +512,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 #pragma unroll
         for (int st = 0; st < 8; ++st) {
           uint32_t ka[4];
-          ldsm_x4(ka, src + k_lm + (((2 * st + k_lm_c) ^ lm_r) << 4));
+          ldsm_x4(ka, src + k_off[st & 3] + (st >> 2) * 128);
           if (st & 1) mma_bf16(sc2, ka[0], ka[1], ka[2], ka[3], qb[st][0], qb[st][1]);
           else mma_bf16(sc, ka[0], ka[1], ka[2], ka[3], qb[st][0], qb[st][1]);
         }
@@ -508,7 +524,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       // ---- look-ahead: K copies of block n + kDepth into the slot block n's K tile just left, then
       // stages R and P one and two blocks further ---------------------------------------------------
       __syncwarp();                                    // every lane has this block's K fragments
-      stage_ik(n + kDepth, row_p);
+      stage_ik(n + kDepth, dst_ahead, row_p);
       const int row_v = row_p;
       stage_r(n + kDepth + 1, pos_p, idx_p, row_p);
       stage_p(n + kDepth + 2, pos_p, idx_p);
@@ -565,12 +581,11 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           const uint32_t ph0 = movm_trans(h0), ph1 = movm_trans(h1), pl0 = movm_trans(r0w), pl1 = movm_trans(r1w);
           cp_async_wait<kWaitV>();
           __syncwarp();                                // every lane's V copies of this block have landed
-          const uint32_t vt = src + L::kTileBytes + v_lm;
           uint32_t va[8][4];                           // A fragments of V^T: dims 16 j .. + 15 x the block's 16 tokens
 #pragma unroll
-          for (int j = 0; j < 8; ++j) ldsm_x4_trans(va[j], vt + (((2 * j + v_lm_c) ^ lm_r) << 4));
+          for (int j = 0; j < 8; ++j) ldsm_x4_trans(va[j], src + L::kTileBytes + v_off[j & 3] + (j >> 2) * 128);
           __syncwarp();                                // the V tile's slot is free: copies of block n + kDepth
-          stage_iv(n + kDepth, row_v);                 // go out while the tensor cores work
+          stage_iv(n + kDepth, dst_ahead, row_v);      // go out while the tensor cores work
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             mma_bf16(o[j], va[j][0], va[j][1], va[j][2], va[j][3], ph0, ph1);
@@ -578,7 +593,11 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           }
         }
       }
-      if (HAS_V && !live) stage_iv(n + kDepth, row_v);   // keeps the group count in step (nothing to copy any more)
+      if (HAS_V && !live) stage_iv(n + kDepth, dst_ahead, row_v);   // keeps the group count in step (nothing to copy any more)
+      src += L::kStageBytes;
+      if (src == ring_end) src = ring_warp;
+      dst_ahead += L::kStageBytes;
+      if (dst_ahead == ring_end) dst_ahead = ring_warp;
       FASTOCR_TRACE_CLK(c_end);
       FASTOCR_TRACE_ADD(trace_pv, c_end, c_look);
     }
