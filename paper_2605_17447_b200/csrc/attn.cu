@@ -391,33 +391,39 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     // warp's block, a load from the index list for selected image tokens; R (row n+3) physical
     // cache row, a block-table load for paged caches; I (row n+2) the cp.async copies; C (row n)
     // the arithmetic.
-    auto stage_p = [&](int r, int& pos, bool& is_idx) {      // is_idx: pos is a raw index-list entry, checked in stage R
+    // A block is named by the list index jr of its first token (tok0 + 32 per block); it exists
+    // while jr < lim. All 32 lanes run stages P and R (lanes 16-31 mirror lanes 0-15: no divergence).
+    const int lim = min(sg.n_tok, tok0 + seg_rows * kRowTokens);
+    const int tl = lane & (kBlockTokens - 1);
+    const int vis_end = sg.vs + sg.kept_vis, text_shift = sg.N - sg.kept_vis;
+    const int32_t* idx_row = a.idx != nullptr ? a.idx + static_cast<int64_t>(b) * a.k_stride - sg.vs : nullptr;
+    const int32_t* bt_row = a.page_size > 0 ? a.block_table + static_cast<int64_t>(b) * a.max_pages : nullptr;
+    auto stage_p = [&](int jr, int& pos, bool& is_idx) {     // is_idx: pos is a raw index-list entry, checked in stage R
       is_idx = false;
-      const int jr = tok0 + r * kRowTokens;
-      if (r < seg_rows && jr < sg.n_tok && lane < kBlockTokens) {
-        const int j = min(jr + lane, sg.n_tok - 1);
+      if (jr < lim) {
+        const int j = min(jr + tl, sg.n_tok - 1);
         pos = j;
-        if (a.idx != nullptr) {                        // kept set: text before | selected image | text after
-          if (j >= sg.vs + sg.kept_vis) {
-            pos = j - sg.kept_vis + sg.N;
+        if (idx_row != nullptr) {                      // kept set: text before | selected image | text after
+          if (j >= vis_end) {
+            pos = j + text_shift;
           } else if (j >= sg.vs) {
-            pos = __ldg(a.idx + static_cast<int64_t>(b) * a.k_stride + (j - sg.vs));
+            pos = __ldg(idx_row + j);
             is_idx = true;
           }
         }
       }
     };
-    auto stage_r = [&](int r, int pos, bool is_idx, int& row) {
-      if (r < seg_rows && tok0 + r * kRowTokens < sg.n_tok && lane < kBlockTokens) {
+    auto stage_r = [&](int jr, int pos, bool is_idx, int& row) {
+      if (jr < lim) {
         if (is_idx) {
           if (pos < 0 || pos >= sg.N) {                // never read outside the image span
-            atomicAdd(a.fault_counter, 1ULL);
+            if (lane < kBlockTokens) atomicAdd(a.fault_counter, 1ULL);
             pos = pos < 0 ? 0 : sg.N - 1;
           }
           pos += sg.vs;
         }
-        if (a.page_size > 0) {
-          const int page = __ldg(a.block_table + static_cast<int64_t>(b) * a.max_pages + pos / a.page_size);
+        if (bt_row != nullptr) {
+          const int page = __ldg(bt_row + pos / a.page_size);
           pos = page * a.page_size + pos % a.page_size;
         }
         row = pos;
@@ -426,8 +432,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     // The copies of a block: its 16 K rows are one cp.async group, its 16 V rows another (K is
     // needed at the top of the block's iteration, V only after the softmax, and each tile's ring
     // slot is free again as soon as the fragments of the block that used it last are in registers).
-    auto stage_ik = [&](int r, uint32_t dst, int row) {
-      if (r < seg_rows && tok0 + r * kRowTokens < sg.n_tok) {
+    auto stage_ik = [&](int jr, uint32_t dst, int row) {
+      if (jr < lim) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {                  // rows 2i (lanes 0-15) and 2i + 1 (lanes 16-31)
           const int rr = __shfl_sync(0xffffffffu, row, 2 * i + half);
@@ -436,9 +442,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       }
       cp_async_commit();
     };
-    auto stage_iv = [&](int r, uint32_t dst, int row) {
+    auto stage_iv = [&](int jr, uint32_t dst, int row) {
       if (!HAS_V) return;
-      if (r < seg_rows && tok0 + r * kRowTokens < sg.n_tok) {
+      if (jr < lim) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int rr = __shfl_sync(0xffffffffu, row, 2 * i + half);
@@ -474,18 +480,18 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 #pragma unroll
       for (int r = 0; r < kDepth + 2; ++r) {
         posq[r] = 0;
-        stage_p(r, posq[r], ixq[r]);
+        stage_p(tok0 + r * kRowTokens, posq[r], ixq[r]);
       }
 #pragma unroll
       for (int r = 0; r < kDepth + 1; ++r) {
         rowq[r] = 0;
-        stage_r(r, posq[r], ixq[r], rowq[r]);
+        stage_r(tok0 + r * kRowTokens, posq[r], ixq[r], rowq[r]);
       }
       FASTOCR_TRACE_CYC(12);
 #pragma unroll
       for (int r = 0; r < kDepth; ++r) {
-        stage_ik(r, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
-        stage_iv(r, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
+        stage_ik(tok0 + r * kRowTokens, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
+        stage_iv(tok0 + r * kRowTokens, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
       }
       row_p = rowq[kDepth];
       pos_p = posq[kDepth + 1];
@@ -496,15 +502,14 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     uint32_t dst_ahead = ring_warp + (kDepth % kStages) * L::kStageBytes;   // ring slot of block n + kDepth
     const uint32_t ring_end = ring_warp + kStages * L::kStageBytes;
 #pragma unroll 1
-    for (int n = 0; n < seg_rows; ++n) {
-      const int j0 = tok0 + n * kRowTokens;
+    for (int j0 = tok0; j0 < tok0 + seg_rows * kRowTokens; j0 += kRowTokens) {   // j0: list index of the block's first token
       FASTOCR_TRACE_CLK(c_top);
       cp_async_wait<kWaitK>();
       __syncwarp();                                    // every lane's K copies of this block have landed
       FASTOCR_TRACE_CLK(c_waited);
       FASTOCR_TRACE_ADD(trace_wait, c_waited, c_top);
-      if (n == 0) { FASTOCR_TRACE_MARK(3); FASTOCR_TRACE_CYC(14); }
-      const bool live = j0 < sg.n_tok;         // the block holds at least one attended token
+      if (j0 == tok0) { FASTOCR_TRACE_MARK(3); FASTOCR_TRACE_CYC(14); }
+      const bool live = j0 < sg.n_tok;                 // the block holds at least one attended token
       // two accumulators (even / odd 16-dim steps): dependent MMA chains of four
       float sc[4] = {0.f, 0.f, 0.f, 0.f}, sc2[4] = {0.f, 0.f, 0.f, 0.f};
       if (live) {
@@ -524,20 +529,21 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       // ---- look-ahead: K copies of block n + kDepth into the slot block n's K tile just left, then
       // stages R and P one and two blocks further ---------------------------------------------------
       __syncwarp();                                    // every lane has this block's K fragments
-      stage_ik(n + kDepth, dst_ahead, row_p);
+      stage_ik(j0 + kDepth * kRowTokens, dst_ahead, row_p);
       const int row_v = row_p;
-      stage_r(n + kDepth + 1, pos_p, idx_p, row_p);
-      stage_p(n + kDepth + 2, pos_p, idx_p);
+      stage_r(j0 + (kDepth + 1) * kRowTokens, pos_p, idx_p, row_p);
+      stage_p(j0 + (kDepth + 2) * kRowTokens, pos_p, idx_p);
 
       FASTOCR_TRACE_CLK(c_look);
       FASTOCR_TRACE_ADD(trace_look, c_look, c_qk);
       if (live) {
         // ---- online softmax: x[0], x[1] token j0 + g8 (heads hA, hB); x[2], x[3] token j0 + 8 + g8 ------
         float x[4] = {sc[0] * scale_log2, sc[1] * scale_log2, sc[2] * scale_log2, sc[3] * scale_log2};
+        const int rem = sg.n_tok - j0 - g8;            // > 0: token j0 + g8 is attended; > 8: token j0 + 8 + g8 too
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int tok = j0 + g8 + 8 * (i >> 1);      // index in the unit's attended list
-          const bool valid = ((i & 1) ? okB : okA) && tok < sg.n_tok;
+          const bool valid = ((i & 1) ? okB : okA) && rem > 8 * (i >> 1);
           x[i] = valid ? x[i] : -INFINITY;
           float* lrow = (i & 1) ? logitB : logitA;
           if (lrow != nullptr && valid) {              // dense / scoring mode: position == list index
@@ -585,7 +591,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 #pragma unroll
           for (int j = 0; j < 8; ++j) ldsm_x4_trans(va[j], src + L::kTileBytes + v_off[j & 3] + (j >> 2) * 128);
           __syncwarp();                                // the V tile's slot is free: copies of block n + kDepth
-          stage_iv(n + kDepth, dst_ahead, row_v);      // go out while the tensor cores work
+          stage_iv(j0 + kDepth * kRowTokens, dst_ahead, row_v);   // go out while the tensor cores work
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             mma_bf16(o[j], va[j][0], va[j][1], va[j][2], va[j][3], ph0, ph1);
@@ -593,7 +599,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           }
         }
       }
-      if (HAS_V && !live) stage_iv(n + kDepth, dst_ahead, row_v);   // keeps the group count in step (nothing to copy any more)
+      if (HAS_V && !live) stage_iv(j0 + kDepth * kRowTokens, dst_ahead, row_v);   // keeps the group count in step (nothing to copy any more)
       src += L::kStageBytes;
       if (src == ring_end) src = ring_warp;
       dst_ahead += L::kStageBytes;
