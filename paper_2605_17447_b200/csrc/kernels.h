@@ -53,7 +53,9 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 // ascending order and the total divided by H; every kernel that forms scores goes through these
 // two functions, so that they all produce the same bits.
 __device__ __forceinline__ float score_add_head(float acc, float logit, float max_log2, float inv_sum) {
-  return acc + exp2f(logit - max_log2) * inv_sum;
+  float e;   // logit <= max: the weight is in (0, 1]; weights below 2^-126 count as 0
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(logit - max_log2));
+  return acc + e * inv_sum;
 }
 __device__ __forceinline__ float score_finish(float acc, int num_q_heads) { return acc / static_cast<float>(num_q_heads); }
 #endif

@@ -1,15 +1,20 @@
 // TopK of Eq. 2: exact selection of the k best-scored image tokens of every sequence.
 //
-// One thread-block cluster per sequence (1, 2, 4 or 8 CTAs, chosen so that a launch fills the GPU
-// even for small batches); CTA c of the cluster owns the contiguous slice c of the sequence's
-// scores. The scores are mapped to order-preserving 32-bit keys held in shared memory, the key of
-// the k-th largest score is found with a three-pass MSB-first radix select (digits of 11, 11 and 10
-// bits: every CTA histograms its slice, the bin totals are summed across the cluster through
-// distributed shared memory, and every CTA scans the same totals), and the result is emitted by an in-order
-// compaction: every key above the threshold, plus the first r keys equal to it, where r is what is
-// left of k. Walking the indices in ascending order gives both the "lower index wins ties" rule
-// and the ascending output order with no sort; a CTA learns how many selected keys precede its
-// slice from the other CTAs' totals.
+// Every CTA that works on a sequence holds ALL of the sequence's scores, mapped to order-preserving
+// 32-bit keys, in its own shared memory (at most 32768 keys, 128 KB) and selects on its own: the
+// key of the k-th largest score is found with a three-pass MSB-first radix select (digits of 11,
+// 11 and 10 bits; a pass is a shared-memory histogram and a block-wide scan from the top bin), and
+// the result is emitted by an in-order compaction: every key above the threshold, plus the first
+// r keys equal to it, where r is what is left of k. Walking the indices in ascending order gives
+// both the "lower index wins ties" rule and the ascending output order with no sort.
+//
+// Given a score array, one CTA per sequence does all of that. In a decode step the scores do not
+// exist yet: they are formed here from the focal layer's logits (Section 3.1.1: post-softmax
+// weight averaged over the heads), which is the expensive part (H exponentials per token), so a
+// thread-block cluster of 1, 2, 4 or 8 CTAs shares it: CTA c scores slice c of the tokens and
+// writes the keys into the shared memory of every CTA of the cluster (distributed shared memory);
+// after one cluster barrier all CTAs hold the same keys, run the same selection, and CTA c emits
+// the selected tokens of slice c. No further communication is needed.
 #include "kernels.h"
 
 #include <cooperative_groups.h>
@@ -40,11 +45,10 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
                                                                    const float* __restrict__ logits,
                                                                    const float* __restrict__ stats, int num_q_heads,
                                                                    int n_stride_logits) {
-  extern __shared__ uint32_t keys[];                    // this CTA's slice of the keys
+  extern __shared__ __align__(16) uint32_t keys[];      // all keys of the sequence
   __shared__ float head_st[2 * kTopkMaxHeads];          // scoring mode: per head (max, 1 / sum)
-  __shared__ uint32_t hist_buf[2][kTopkBins];           // this CTA's digit histograms (read by the whole cluster)
+  __shared__ uint32_t hist[kTopkBins];
   __shared__ uint32_t warp_gt[kTopkWarps], warp_eq[kTopkWarps];
-  __shared__ uint32_t slice_tot[2];                     // selected-candidate counts of this slice: above, equal
   __shared__ uint32_t sel_prefix, sel_remaining;
 
   wait_for_prior_grids();
@@ -53,29 +57,38 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   const int C = static_cast<int>(cluster.num_blocks());
   const int c = static_cast<int>(cluster.block_rank());
   const int b = blockIdx.x / C, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int N = min(vis_len[b], n_cap);                 // n_cap: what the launch sized the key slices for
+  const int N = min(vis_len[b], n_cap);                 // n_cap: what the launch sized the key array for
   int k = kreq[b];
   k = k < 0 ? 0 : (k > N ? N : k);
   k = min(k, k_stride);
   if (k == 0) return;                                   // the same decision in every CTA of the cluster
 
-  // slice [lo_i, hi_i) of the sequence, a multiple of 32 keys per CTA
+  // slice [lo_i, hi_i) of the tokens: what this CTA scores and emits; a multiple of 32 per CTA
   const int per_cta = (((N + C - 1) / C) + 31) & ~31;
   const int lo_i = min(c * per_cta, N), hi_i = min(lo_i + per_cta, N);
   const int n_loc = hi_i - lo_i;
+  // A peer's shared memory may be written only once that CTA is known to be running: every CTA
+  // signals here and checks for the others just before its first remote store.
+  if (C > 1) cluster.barrier_arrive();
+  hist[2 * tid] = hist[2 * tid + 1] = 0u;
+  if (tid == 0) {
+    sel_prefix = 0u;
+    sel_remaining = static_cast<uint32_t>(k);
+  }
   if (logits == nullptr) {
-    const float* sp = scores + static_cast<int64_t>(b) * n_stride + lo_i;
-    for (int i = tid; i < n_loc; i += kTopkThreads) keys[i] = score_key(sp[i]);
+    const float* sp = scores + static_cast<int64_t>(b) * n_stride;
+    for (int i = tid; i < N; i += kTopkThreads) keys[i] = score_key(sp[i]);
   } else {
-    // Scores formed here from the focal layer's logits (the same arithmetic as the stand-alone
-    // scoring kernel, head by head in ascending order): four tokens per thread, eight heads' loads
-    // in flight. The logits were written by the kernel just before and are read from L2.
+    // Scores of the CTA's slice (the same arithmetic as the stand-alone scoring kernel, head by
+    // head in ascending order): four tokens per thread, eight heads' loads in flight. The logits
+    // were written by the kernel just before and are read from L2.
     for (int i = tid; i < num_q_heads; i += kTopkThreads) {
       head_st[2 * i] = stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2];
       head_st[2 * i + 1] = 1.0f / stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2 + 1];
     }
     __syncthreads();
     const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + lo_i;
+    bool peers_checked = C == 1;
     const bool vec = (n_stride_logits & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;   // lo_i is a multiple of 32
     for (int i0 = tid * 4; i0 < n_loc; i0 += kTopkThreads * 4) {
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -108,36 +121,44 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
           }
         }
       }
+      uint32_t kq[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
-        if (i0 + j < n_loc) keys[i0 + j] = score_key(score_finish(acc[j], num_q_heads));
+      for (int j = 0; j < 4; ++j) kq[j] = score_key(score_finish(acc[j], num_q_heads));
+      // into every CTA's copy of the key array
+      if (!peers_checked) {
+        cluster.barrier_wait();
+        peers_checked = true;
+      }
+      for (int r = 0; r < C; ++r) {
+        uint32_t* dst = cluster.map_shared_rank(keys, r) + lo_i + i0;
+        if (i0 + 4 <= n_loc) {
+          *reinterpret_cast<uint4*>(dst) = make_uint4(kq[0], kq[1], kq[2], kq[3]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (i0 + j < n_loc) dst[j] = kq[j];
+        }
+      }
     }
-  }
-  hist_buf[0][2 * tid] = hist_buf[0][2 * tid + 1] = 0u;
-  hist_buf[1][2 * tid] = hist_buf[1][2 * tid + 1] = 0u;
-  if (tid == 0) {
-    sel_prefix = 0u;
-    sel_remaining = static_cast<uint32_t>(k);
+    if (!peers_checked) cluster.barrier_wait();         // (a thread without tokens to score)
+    if (C > 1) cluster.sync();                          // every slice has arrived in every copy
   }
   __syncthreads();
 
   // ---- radix select, three passes over digits of 11, 11 and 10 bits (most significant first) ----
-  // Pass p: every CTA histograms the digit of those of its keys that match the prefix found so far;
-  // after one cluster barrier thread t adds up bins 2t and 2t + 1 (counted from the largest digit)
-  // of all CTAs through distributed shared memory, and a block-wide scan finds the digit at which
-  // the running count from the top reaches what is left of k. The two histogram buffers alternate,
-  // so the buffer of pass p is cleared during pass p + 1, behind that pass's barrier.
+  // Pass p histograms the digit of the keys that match the prefix found so far; thread t then owns
+  // bins 2047 - 2t and 2046 - 2t, and a block-wide scan from the top bin finds the digit at which
+  // the running count reaches what is left of k.
   for (int pass = 0; pass < 3; ++pass) {
     const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
     const uint32_t digit_mask = pass == 2 ? 0x3ffu : 0x7ffu;
     const uint32_t hi_mask = pass == 0 ? 0u : (0xffffffffu << (pass == 1 ? 21 : 10));
-    uint32_t* hist = hist_buf[pass & 1];
     const uint32_t prefix = sel_prefix;
     const uint32_t remaining = sel_remaining;
-    for (int base = warp * 32; base < n_loc; base += kTopkThreads) {   // warp-uniform trip count
+    for (int base = warp * 32; base < N; base += kTopkThreads) {   // warp-uniform trip count
       const int i = base + lane;
-      const uint32_t key = i < n_loc ? keys[i] : 0u;
-      const bool in = i < n_loc && (key & hi_mask) == prefix;
+      const uint32_t key = i < N ? keys[i] : 0u;
+      const bool in = i < N && (key & hi_mask) == prefix;
       const uint32_t digit = (key >> shift) & digit_mask;
       if (pass == 0) {
         // the leading bits (sign, exponent) are heavily clustered: aggregate identical digits
@@ -151,17 +172,11 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
         atomicAdd(&hist[digit], 1u);
       }
     }
-    cluster.sync();                                     // every slice's histogram is complete
-    // bins in descending digit order: thread t owns digits 2047 - 2t and 2046 - 2t
-    const int d0 = kTopkBins - 1 - 2 * tid, d1 = d0 - 1;
-    uint32_t c0 = 0, c1 = 0;
-    for (int r = 0; r < C; ++r) {
-      const uint32_t* h = cluster.map_shared_rank(hist, r);
-      c0 += h[d0];
-      c1 += h[d1];
-    }
-    hist_buf[(pass + 1) & 1][2 * tid] = 0u;             // last read (by anyone) before the barrier above
-    hist_buf[(pass + 1) & 1][2 * tid + 1] = 0u;
+    __syncthreads();
+    const int d0 = kTopkBins - 1 - 2 * tid, d1 = d0 - 1;   // bins in descending digit order
+    const uint32_t c0 = hist[d0], c1 = hist[d1];
+    hist[d0] = 0u;                                      // ready for the next pass
+    hist[d1] = 0u;
     const uint32_t local = c0 + c1;
     uint32_t incl = local;
 #pragma unroll
@@ -194,9 +209,9 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   const uint32_t thr = sel_prefix;                      // key of the k-th largest score
   const uint32_t take_eq = sel_remaining;               // how many keys equal to thr are selected
 
-  // ---- in-order compaction --------------------------------------------------------------------
-  const int per = (n_loc + kTopkThreads - 1) / kTopkThreads;
-  const int lo = min(tid * per, n_loc), hi = min(lo + per, n_loc);
+  // ---- in-order compaction over all keys; this CTA emits the tokens of its own slice ------------
+  const int per = (N + kTopkThreads - 1) / kTopkThreads;
+  const int lo = min(tid * per, N), hi = min(lo + per, N);
   uint32_t gt = 0, eq = 0;
   for (int i = lo; i < hi; ++i) {
     const uint32_t key = keys[i];
@@ -232,37 +247,28 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
     }
     warp_gt[lane] = ai - a;                             // exclusive
     warp_eq[lane] = ei - e;
-    if (lane == 31) {
-      slice_tot[0] = ai;
-      slice_tot[1] = ei;
-    }
   }
-  cluster.sync();                                       // also orders warp_gt / warp_eq inside the CTA
+  __syncthreads();
   uint32_t gt_before = warp_gt[warp] + gt_incl - gt;
   uint32_t eq_before = warp_eq[warp] + eq_incl - eq;
-  for (int r = 0; r < c; ++r) {                         // candidates in the slices before this one
-    const uint32_t* t = cluster.map_shared_rank(slice_tot, r);
-    gt_before += t[0];
-    eq_before += t[1];
-  }
   int32_t* op = idx_out + static_cast<int64_t>(b) * k_stride;
   for (int i = lo; i < hi; ++i) {
     const uint32_t key = keys[i];
+    const bool mine = i >= lo_i && i < hi_i;
     if (key > thr) {
-      op[gt_before + min(eq_before, take_eq)] = lo_i + i;
+      if (mine) op[gt_before + min(eq_before, take_eq)] = i;
       ++gt_before;
     } else if (key == thr) {
-      if (eq_before < take_eq) op[gt_before + eq_before] = lo_i + i;
+      if (mine && eq_before < take_eq) op[gt_before + eq_before] = i;
       ++eq_before;
     }
   }
-  cluster.sync();                                       // nobody leaves while its shared memory may still be read
 }
 
 }  // namespace
 
 cudaError_t configure_topk() {
-  cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkMaxN * 4);
+  cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkMaxN * 4 + 16);
   if (e != cudaSuccess) return e;
   // same shared-memory carve-out as the attention kernel: no reconfiguration between them
   return cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
@@ -274,16 +280,18 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
                                cudaStream_t s) {
   if (batch <= 0 || max_vis_len <= 0) return cudaSuccess;
   if (logits != nullptr && (num_q_heads <= 0 || num_q_heads > kTopkMaxHeads)) return cudaErrorInvalidValue;
-  // cluster size: enough CTAs to cover the GPU for small batches, at least 1024 keys per CTA
-  int device = 0, sms = 148;
-  if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+  // Cluster size: one CTA per sequence when the scores exist; when they are formed here, enough
+  // CTAs to cover the GPU for small batches, with at least 1024 tokens to score per CTA.
   int C = 1;
-  while (C < kTopkMaxCluster && batch * C * 2 <= sms && max_vis_len / (C * 2) >= 1024) C *= 2;
-  const int per_cta = (((max_vis_len + C - 1) / C) + 31) & ~31;
+  if (logits != nullptr) {
+    int device = 0, sms = 148;
+    if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    while (C < kTopkMaxCluster && batch * C * 2 <= sms && max_vis_len / (C * 2) >= 1024) C *= 2;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(batch * C);
   cfg.blockDim = dim3(kTopkThreads);
-  cfg.dynamicSmemBytes = static_cast<size_t>(per_cta) * 4;
+  cfg.dynamicSmemBytes = (static_cast<size_t>(max_vis_len) + 31) / 32 * 32 * 4 + 16;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
