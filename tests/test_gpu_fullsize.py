@@ -3,6 +3,7 @@ heads, contiguous cache): sampled sequences are checked one by one against the o
 that hold at any size are checked on the whole batch."""
 import math
 
+import numpy as np
 import pytest
 import torch
 
@@ -20,7 +21,7 @@ def test_full_size_layer_chain_against_oracle_on_sampled_sequences():
     B, H, Hkv, N = cfg.batch, cfg.num_q_heads, cfg.num_kv_heads, cfg.vis_len[0]
     S = cfg.seq_len(0)[0] + 1
     K, V = make_kv(cfg.seed, 0, B, S, Hkv, 128, dev)
-    centres = torch.tensor([fixation_track(cfg.seed, b, 1, cfg.grid_h[b], cfg.grid_w[b], cfg.advance)[0] for b in range(B)], device=dev)
+    centres = torch.tensor(np.array([fixation_track(cfg.seed, b, 1, cfg.grid_h[b], cfg.grid_w[b], cfg.advance)[0] for b in range(B)]), device=dev)
     i32 = lambda x: torch.tensor(x, dtype=torch.int32, device=dev)
     vs = i32(cfg.vis_start)
     q = make_queries(cfg.seed, 0, 0, lambda b, pos: K[b, pos], vs.long(), centres,
@@ -51,6 +52,14 @@ def test_full_size_layer_chain_against_oracle_on_sampled_sequences():
     out_full = torch.empty_like(dense)
     fo.fastocr_sparse_decode_attn(ctx, kv, q, full, i32([N] * B), out_full)
     assert float((out_full - dense).abs().max()) <= 1e-5
+    # the decode step (scores formed inside the selection kernel, a cluster of CTAs per sequence,
+    # launches overlapping) gives the same bits as the separate calls
+    fix = torch.full((B, k), -1, dtype=torch.int32, device=dev)
+    out2 = torch.empty(2, B, H, 128, dtype=torch.float32, device=dev)
+    have = fo.fastocr_decode_step(ctx, [kv, kv], torch.stack([q, q]), out2, [True, False], kd, fix, False, N)
+    torch.cuda.synchronize()
+    assert have and torch.equal(fix, idx)
+    assert torch.equal(out2[0], dense) and torch.equal(out2[1], out)
     # sampled sequences against the oracle, element by element
     for b in (0, 17, 63):
         qc, Kc, Vc = q[b].cpu(), K[b].cpu(), V[b].cpu()

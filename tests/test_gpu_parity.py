@@ -271,6 +271,37 @@ def test_decode_step_matches_algorithm_trace(fo, ctx):
                 f_last[b] = tr.f_last
 
 
+@pytest.mark.parametrize("batch,n", [(2, 16384), (5, 4100), (1, 2048)])
+def test_decode_step_selection_equals_separate_calls(fo, batch, n):
+    """The decode step's selection kernel forms the scores itself, with a cluster of up to 8 CTAs per
+    sequence for small batches; it must select exactly what scoring + selection as separate calls do."""
+    from workloads import make_kv, normal_bf16, stream_key
+    dev = "cuda"
+    H, Hkv, T = 28, 4, 40
+    S = n + T
+    K, V = make_kv(900 + batch, 0, batch, S, Hkv, 128, dev)
+    q = (normal_bf16(stream_key(901, batch), (batch, H, 128), dev).float() * 3).to(torch.bfloat16)
+    i32 = lambda x: torch.tensor(x, dtype=torch.int32, device=dev)
+    vis = [n - 7 * b for b in range(batch)]                      # ragged image spans
+    kv = fo.KVView(K, V, i32([S - 7 * b for b in range(batch)]), i32([8] * batch), i32(vis), H, S, SCALE)
+    ks = [oracle.kept_count(v, 0.05) for v in vis]
+    kd = i32(ks)
+    c2 = fo.Context(batch, H, Hkv, S, n)
+    dense = torch.empty(batch, H, 128, dtype=torch.float32, device=dev)
+    sc = torch.zeros(batch, n, dtype=torch.float32, device=dev)
+    idx = torch.full((batch, max(ks)), -1, dtype=torch.int32, device=dev)
+    fo.fastocr_dense_decode_attn(c2, kv, q, dense, scores_out=sc)
+    fo.fastocr_select_topk(c2, sc, kv.vis_len, kd, idx, n)
+    fix = torch.full_like(idx, -1)
+    out = torch.empty(1, batch, H, 128, dtype=torch.float32, device=dev)
+    assert fo.fastocr_decode_step(c2, [kv], q[None], out, [True], kd, fix, False, n)
+    torch.cuda.synchronize()
+    assert torch.equal(fix, idx) and torch.equal(out[0], dense)
+    for b in range(batch):                                        # and both are the oracle's choice on these scores
+        assert idx[b, :ks[b]].cpu().tolist() == oracle.topk(sc[b, :vis[b]].cpu(), ks[b]).tolist()
+    c2.close()
+
+
 def test_argument_errors_are_reported_not_launched(fo, ctx):
     case = make_case(700, [(4, 64, 4)])
     kv = case.device_view()
