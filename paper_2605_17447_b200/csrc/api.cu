@@ -26,6 +26,7 @@ struct fastocr_ctx {
   int sm_count = 148;
   fastocr_limits lim{};
   int64_t cap_items = 0;        // partial slots: one per (team, sequence) pair and KV head
+  int4* plan = nullptr;         // launch plan of the decode step's pruned layers: 4 x int4 per CTA
   float* part_acc = nullptr;    // [cap_items][8][128]
   float* part_ml = nullptr;     // [cap_items][8][2]
   int32_t* counters = nullptr;  // [kMaxUnits] arrival counters of the split merge (zero between launches)
@@ -53,6 +54,8 @@ struct fastocr_ctx {
 };
 
 namespace {
+
+constexpr int kPlanCtas = 4096;   // CTAs a launch plan has room for
 
 fastocr_status fail(fastocr_ctx* ctx, fastocr_status code, const char* fmt, ...) {
   if (ctx != nullptr) {
@@ -225,11 +228,9 @@ fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
   return FASTOCR_OK;
 }
 
-// wait_point: how much of this launch may run while earlier kernels of the stream are still
-// draining (fastocr::kWait...), i.e. which of its inputs could have been written just before.
-fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, const int32_t* idx,
-                           const int32_t* k, int32_t k_stride, int32_t max_kept, void* out, int out_is_fp32,
-                           int wait_point, cudaStream_t s) {
+// launch arguments of a pruned pass (everything but the output, the wait point and the plan)
+AttnLaunch sparse_args(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, const int32_t* idx, const int32_t* k,
+                       int32_t k_stride, int32_t max_kept) {
   const int max_len = (max_kept > 0 && max_kept < kv->max_seq_len) ? max_kept : kv->max_seq_len;
   AttnLaunch a = make_launch(ctx, kv, q, true, max_len);
   a.idx = idx;
@@ -253,8 +254,19 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
     }
     a.active_ctas = a.grid_ctas;
   }
-  a.wait_point = wait_point;
   a.depth = ctx->sparse_depth;
+  return a;
+}
+
+// wait_point: how much of this launch may run while earlier kernels of the stream are still
+// draining (fastocr::kWait...), i.e. which of its inputs could have been written just before.
+// plan: NULL or a launch plan made for exactly these lengths, kept counts and plan_grid CTAs.
+fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, const int32_t* idx,
+                           const int32_t* k, int32_t k_stride, int32_t max_kept, void* out, int out_is_fp32,
+                           int wait_point, cudaStream_t s, const int4* plan = nullptr, int plan_grid = 0) {
+  AttnLaunch a = sparse_args(ctx, kv, q, idx, k, k_stride, max_kept);
+  a.wait_point = wait_point;
+  a.plan = (plan != nullptr && plan_grid == a.grid_ctas) ? plan : nullptr;
   a.out = out;
   a.out_is_fp32 = out_is_fp32;
   {
@@ -315,6 +327,7 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
       (e = cudaMalloc(&ctx->logits, bytes_logits)) != cudaSuccess || (e = cudaMalloc(&ctx->stats, bytes_stats)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->scores, bytes_scores)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->counters, fastocr::kMaxUnits * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->plan, static_cast<size_t>(kPlanCtas) * 4 * sizeof(int4))) != cudaSuccess ||
       (e = cudaMemset(ctx->counters, 0, fastocr::kMaxUnits * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->faults, sizeof(unsigned long long))) != cudaSuccess ||
       (e = cudaMemset(ctx->faults, 0, sizeof(unsigned long long))) != cudaSuccess) {
@@ -328,6 +341,7 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
 void fastocr_destroy(fastocr_ctx* ctx) {
   if (ctx == nullptr) return;
   cudaSetDevice(ctx->device);
+  cudaFree(ctx->plan);
   cudaFree(ctx->part_acc);
   cudaFree(ctx->part_ml);
   cudaFree(ctx->logits);
@@ -440,6 +454,30 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
   // dense attention kernel of this step (it wrote an output slice and the split workspace, neither
   // of which the next attention kernel reads), or the selection kernel (it wrote the index set).
   enum { kOther, kAttention, kSelection } prev = kOther;
+  // The pruned layers of a step see the same lengths and kept counts: what every CTA of theirs
+  // would work out from those (its range, its unit) is computed once, by a small kernel at the
+  // head of the step, and handed to each pruned launch as a plan. Layers whose view differs from
+  // the first pruned layer's in anything the plan depends on simply run without it.
+  const fastocr_kv_view* plan_view = nullptr;
+  int plan_grid = 0, n_pruned = 0;
+  for (int l = 0; l < num_layers; ++l) {
+    const bool pruned = !(is_focal[l] != 0 || (l == 0 && !have));
+    if (!pruned) continue;
+    if (plan_view == nullptr) plan_view = &layers[l];
+    ++n_pruned;
+  }
+  if (n_pruned >= 2 && (!ctx->prof_on || ctx->prof_runs)) {
+    AttnLaunch pa = sparse_args(ctx, plan_view, q, fixation, k, k_stride, max_kept);
+    if (pa.grid_ctas <= kPlanCtas) {
+      plan_grid = pa.grid_ctas;
+      FASTOCR_TRY_CUDA(fastocr::launch_attn_plan(pa, ctx->plan, s), "plan launch");
+    }
+  }
+  auto plan_fits = [&](const fastocr_kv_view& v) {
+    return plan_grid > 0 && v.seq_len == plan_view->seq_len && v.vis_start == plan_view->vis_start &&
+           v.vis_len == plan_view->vis_len && v.max_seq_len == plan_view->max_seq_len && v.batch == plan_view->batch &&
+           v.num_kv_heads == plan_view->num_kv_heads;
+  };
   for (int l = 0; l < num_layers; ++l) {
     const void* ql = static_cast<const char*>(q) + l * q_bytes;
     void* ol = static_cast<char*>(out) + l * o_bytes;
@@ -473,7 +511,8 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
       // queries, index set and cache were complete before), so the two may overlap; right after
       // a selection only the set-up (lengths, kept counts) may run ahead
       const int wp = !chained ? fastocr::kWaitAtStart : (prev == kAttention ? fastocr::kWaitBeforeWrites : fastocr::kWaitAfterSetup);
-      st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, wp, s);
+      st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, wp, s,
+                       plan_fits(layers[l]) ? ctx->plan : nullptr, plan_grid);
       if (st != FASTOCR_OK) return st;
       prev = kAttention;
     }

@@ -180,6 +180,12 @@ __device__ __forceinline__ unsigned long long trace_now() {
 #define FASTOCR_TRACE_ADD(acc, t1, t0) do { } while (0)
 #endif
 
+// Two ways to hand out rows (see the kernel): true = every unit cut into equal parts
+__device__ __forceinline__ bool split_rule(int units, int grid, int total_rows, int longest_unit) {
+  return units <= grid && total_rows < kLongRangeRows * grid &&
+         static_cast<int64_t>(longest_unit) * units <= static_cast<int64_t>(total_rows) + total_rows / 8;
+}
+
 // kDepth: how many blocks ahead of its use a copy is issued (1 .. kStages)
 template <int G, bool HAS_V, int kDepth>
 __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(const AttnLaunch a) {
@@ -216,25 +222,47 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   // first unit: saves that unit a second round trip to L2
   int4* geom_s = reinterpret_cast<int4*>(smem + L::ring);
   static_assert(kMaxUnits * 16 <= L::kRingBytes, "the geometry table must fit the ring");
-  {
+  // A launch plan (launch_attn_plan) hands the CTA its range, its unit and the unit's geometry
+  // in one 64-byte record: one round trip and no scan. A record marked invalid (the CTA's range
+  // would span several units) sends the CTA through the full set-up.
+  if (tid == 0) mrg_flag[3] = 0;
+  __syncthreads();
+  int4 plan0 = make_int4(0, 0, 0, 0), plan1 = plan0, plan2 = plan0, plan3 = plan0;
+  if (a.plan != nullptr) {
+    const int4* rec = a.plan + 4 * static_cast<int64_t>(blockIdx.x);
+    plan0 = __ldg(rec);
+    plan1 = __ldg(rec + 1);
+    plan2 = __ldg(rec + 2);
+    plan3 = __ldg(rec + 3);
+  }
+  const bool planned = plan0.x != 0;
+  //                  // {valid, unit, r0, r1} {ubeg, uend, split, parts} {per_cta, total, -, -} {geometry}
+  if (planned) {
+    if (tid == 0) {
+      prefix_s[plan0.y] = plan1.x;
+      prefix_s[plan0.y + 1] = plan1.y;
+      prefix_s[units] = plan2.y;
+      geom_s[plan0.y] = plan3;
+    }
+  } else {
     constexpr int kPerThread = kMaxUnits / kThreads;
-    int rows_of[kPerThread];
+    SeqGeom gq[kPerThread];                            // all loads first, so that they are in flight together
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) {
-      const int uu = i * kThreads + tid;
-      rows_of[i] = 0;
-      if (uu < units) {
-        const SeqGeom sg = load_geom(a, uu / Hkv);
-        rows_of[i] = (sg.n_tok + kRowTokens - 1) / kRowTokens;
-        geom_s[uu] = make_int4(sg.vs, sg.N, sg.kept_vis, sg.n_tok);
-      }
+      const int uu = min(i * kThreads + tid, units - 1);
+      gq[i] = load_geom(a, uu / Hkv);
     }
     int longest = 0;
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) {
       const int uu = i * kThreads + tid;
-      if (uu < units) prefix_s[uu + 1] = rows_of[i];
-      longest = max(longest, rows_of[i]);
+      if (uu < units) {
+        const int rows = (gq[i].n_tok + kRowTokens - 1) / kRowTokens;
+        geom_s[uu] = make_int4(gq[i].vs, gq[i].N, gq[i].kept_vis, gq[i].n_tok);
+        prefix_s[uu + 1] = rows;
+        longest = max(longest, rows);
+        if (rows == 0) mrg_flag[3] = 1;                // some unit has nothing to attend (rare)
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) longest = max(longest, __shfl_xor_sync(0xffffffffu, longest, o));
@@ -242,7 +270,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   }
   FASTOCR_TRACE_CYC(9);
   __syncthreads();
-  if (warp == 0) {                                     // lane l owns units [l * chunk, (l + 1) * chunk)
+  if (warp == 0 && !planned) {                         // lane l owns units [l * chunk, (l + 1) * chunk)
     const int chunk = (units + 31) >> 5;
     const int u_lo = lane * chunk, u_hi = min(units, u_lo + chunk);
     int sum = 0;
@@ -269,19 +297,22 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   __syncthreads();
   FASTOCR_TRACE_MARK(1);
   FASTOCR_TRACE_CYC(10);
-  const int total_rows = prefix_s[units], longest_unit = mrg_flag[1];
+  const int total_rows = prefix_s[units], longest_unit = planned ? 0 : mrg_flag[1];
   const int grid = min(static_cast<int>(gridDim.x), a.active_ctas);
   // Two ways to hand out rows. Short ranges over at most `grid` units of similar length: every unit
   // is cut into the same number of equal parts, one per CTA, so no CTA straddles two units (no
   // pipeline refill) and a unit that fits one CTA needs no global merge. Otherwise (ragged
   // batches, more units than CTAs, or long ranges where a few merges are negligible): all rows
   // laid end to end and cut into equal ranges.
-  const bool split_units = units <= grid && total_rows < kLongRangeRows * grid &&
-                           static_cast<int64_t>(longest_unit) * units <= static_cast<int64_t>(total_rows) + total_rows / 8;
-  const int parts = split_units ? min(grid / units, kMaxPartsPerUnit) : 1;     // CTAs per unit
-  const int per_cta = (total_rows + grid - 1) / grid;   // rows per CTA (equal-range mode)
+  const bool split_units = planned ? plan1.z != 0 : split_rule(units, grid, total_rows, longest_unit);
+  const int parts = planned ? plan1.w : (split_units ? min(grid / units, kMaxPartsPerUnit) : 1);     // CTAs per unit
+  const int per_cta = planned ? plan2.x : (total_rows + grid - 1) / grid;   // rows per CTA (equal-range mode)
   int r0 = 0, r1 = 0, first_unit = 0;
-  if (static_cast<int>(blockIdx.x) >= grid) {
+  if (planned) {
+    first_unit = plan0.y;
+    r0 = plan0.z;
+    r1 = plan0.w;
+  } else if (static_cast<int>(blockIdx.x) >= grid) {
     // a spare CTA: launched only so that the launch claims the whole shared-memory array of every SM
   } else if (split_units) {
     first_unit = blockIdx.x / parts;
@@ -332,7 +363,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 
   // ---- the CTA's range, one unit segment after the other --------------------------------------
   int u = first_unit;
-  if (!split_units && r0 < r1) {
+  if (!planned && !split_units && r0 < r1) {
     int lo = 0, hi = units;                            // largest u with prefix[u] <= r0
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
@@ -787,7 +818,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   if (blockIdx.x == 0) wait_for_prior_grids();
 
   // ---- sequences with nothing to attend get zeros (rare; kept off the main path) ---------------
-  if (blockIdx.x == 0) {
+  if (blockIdx.x == 0 && mrg_flag[3] != 0) {           // (never with a plan: it is valid only when no unit is empty)
     for (int e = 0; e < units; ++e) {
       if (prefix_s[e + 1] != prefix_s[e]) continue;
       wait_for_prior_grids();
@@ -800,6 +831,77 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           a.stats[(head0 + i) * 2 + 1] = 0.f;
         }
     }
+  }
+}
+
+// The set-up of attn_stream_kernel done once for all CTAs of a launch shape: rows per unit, their
+// prefix, the way rows are handed out, and per CTA its range, unit and the unit's geometry.
+__global__ void __launch_bounds__(kMaxUnits) attn_plan_kernel(const AttnLaunch a, int4* __restrict__ plan_out) {
+  __shared__ int prefix_s[kMaxUnits + 1];
+  __shared__ int warp_tot[kMaxUnits / 32], warp_max[kMaxUnits / 32];
+  wait_for_prior_grids();                              // the previous users of the plan are done
+  dependents_may_launch();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int Hkv = a.num_kv_heads, units = a.batch * Hkv, grid = a.grid_ctas;
+  SeqGeom sg = {0, 0, 0, 0};
+  int rows = 0;
+  if (tid < units) {
+    sg = load_geom(a, tid / Hkv);
+    rows = (sg.n_tok + kRowTokens - 1) / kRowTokens;
+  }
+  int incl = rows, longest = rows;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+    longest = max(longest, __shfl_xor_sync(0xffffffffu, longest, o));
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  if (lane == 0) warp_max[warp] = longest;
+  __syncthreads();
+  int before = 0;
+  longest = 0;
+  for (int w = 0; w < kMaxUnits / 32; ++w) {
+    if (w < warp) before += warp_tot[w];
+    longest = max(longest, warp_max[w]);
+  }
+  if (tid < units) prefix_s[tid + 1] = before + incl;
+  if (tid == 0) prefix_s[0] = 0;
+  const int any_empty = __syncthreads_or(tid < units && rows == 0);
+  const int total_rows = prefix_s[units];
+  const bool split_units = split_rule(units, grid, total_rows, longest);
+  const int parts = split_units ? min(grid / units, kMaxPartsPerUnit) : 1;
+  const int per_cta = (total_rows + grid - 1) / grid;
+  for (int c = tid; c < grid; c += blockDim.x) {
+    int r0 = 0, r1 = 0, u = 0, valid = any_empty ? 0 : 1;
+    if (split_units) {
+      u = c / parts;
+      if (u < units) {
+        const int ub = prefix_s[u], ue = prefix_s[u + 1];
+        const int per = (ue - ub + parts - 1) / parts;
+        r0 = min(ue, ub + (c - u * parts) * per);
+        r1 = min(ue, r0 + per);
+      } else {
+        u = 0;                                         // a CTA without work: an empty range of unit 0
+      }
+    } else {
+      r0 = min(total_rows, c * per_cta);
+      r1 = min(total_rows, r0 + per_cta);
+      int lo = 0, hi = units;                          // largest u with prefix[u] <= r0
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (prefix_s[mid] <= r0) lo = mid; else hi = mid;
+      }
+      u = lo;
+      if (r1 > prefix_s[u + 1]) valid = 0;             // the range spans several units
+      if (r0 >= r1) { u = 0; r0 = r1 = 0; }
+    }
+    const SeqGeom g = load_geom(a, u / Hkv);
+    int4* rec = plan_out + 4 * static_cast<int64_t>(c);
+    rec[0] = make_int4(valid, u, r0, r1);
+    rec[1] = make_int4(prefix_s[u], prefix_s[u + 1], split_units ? 1 : 0, parts);
+    rec[2] = make_int4(per_cta, total_rows, 0, 0);
+    rec[3] = make_int4(g.vs, g.N, g.kept_vis, g.n_tok);
   }
 }
 
@@ -873,6 +975,13 @@ cudaError_t configure_t() {
 }  // namespace
 
 #define FASTOCR_FOR_EACH_GROUP(X) X(1) X(2) X(4) X(7) X(8)
+
+cudaError_t launch_attn_plan(const AttnLaunch& a, int4* plan_out, cudaStream_t s) {
+  if (a.batch * a.num_kv_heads > kMaxUnits || a.grid_ctas <= 0) return cudaErrorInvalidValue;
+  const cudaError_t e = launch_pdl(attn_plan_kernel, dim3(1), dim3(kMaxUnits), 0, s, a, plan_out);
+  count_launches(1);
+  return e;
+}
 
 cudaError_t launch_attn_partial(const AttnLaunch& a, cudaStream_t s) {
   const int G = a.num_q_heads / a.num_kv_heads;

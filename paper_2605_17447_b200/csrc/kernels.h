@@ -88,6 +88,8 @@ struct AttnLaunch {
   int32_t wait_point;         // where the kernel waits for earlier kernels: kWaitAtStart / kWaitAfterSetup / kWaitBeforeWrites
   int32_t depth;              // blocks a copy is issued ahead of its use (1..3): deeper hides more latency per warp,
                               // shallower keeps fewer requests queued when the pass saturates HBM anyway
+  const int4* plan;           // NULL or one 64-byte record per CTA written by launch_attn_plan for this very launch
+                              // shape (grid, lengths, kept counts): the CTA's range and unit, ready made
   // workspace
   float* part_acc;            // [slots][8][128], slot = CTA index + unit index (unit = sequence * Hkv + KV head)
   float* part_ml;             // [slots][8][2]  (max, sum) in the log2 domain
@@ -103,6 +105,12 @@ struct AttnLaunch {
 };
 
 cudaError_t launch_attn_partial(const AttnLaunch& a, cudaStream_t s);
+
+// Work records for the CTAs of a later launch_attn_partial with the same lengths, kept counts
+// and grid (a.grid_ctas): what every CTA would otherwise work out for itself from the lengths of
+// all units. plan_out: 4 x int4 per CTA. Several launches may use one plan (the pruned layers of a
+// decode step all see the same lengths and the same kept counts).
+cudaError_t launch_attn_plan(const AttnLaunch& a, int4* plan_out, cudaStream_t s);
 
 // scores[b][i] = (1/H) sum_h 2^(logit[b][h][i] - max_h) / sum_h  for i < vis_len[b].
 cudaError_t launch_scores_finalize(const float* logits, const float* stats, const int32_t* vis_len, int32_t batch,
