@@ -212,11 +212,34 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   // ---- in-order compaction over all keys; this CTA emits the tokens of its own slice ------------
   const int per = (N + kTopkThreads - 1) / kTopkThreads;
   const int lo = min(tid * per, N), hi = min(lo + per, N);
+  // up to 8 keys per thread (N <= 8192) are kept in registers for the second walk; a full chunk of 8
+  // is fetched as two 16-byte loads (a stride of 8 words between lanes would be an 8-way bank conflict)
+  constexpr int kRegKeys = 8;
+  uint32_t kreg[kRegKeys];
+  const bool cached = per <= kRegKeys;
+  if (per == kRegKeys && hi - lo == kRegKeys) {
+    const uint4 a = *reinterpret_cast<const uint4*>(keys + lo), c4 = *reinterpret_cast<const uint4*>(keys + lo + 4);
+    kreg[0] = a.x; kreg[1] = a.y; kreg[2] = a.z; kreg[3] = a.w;
+    kreg[4] = c4.x; kreg[5] = c4.y; kreg[6] = c4.z; kreg[7] = c4.w;
+  } else if (cached) {
+#pragma unroll
+    for (int j = 0; j < kRegKeys; ++j) kreg[j] = lo + j < hi ? keys[lo + j] : 0u;
+  }
   uint32_t gt = 0, eq = 0;
-  for (int i = lo; i < hi; ++i) {
-    const uint32_t key = keys[i];
-    gt += key > thr;
-    eq += key == thr;
+  if (cached) {
+#pragma unroll
+    for (int j = 0; j < kRegKeys; ++j) {
+      if (lo + j < hi) {
+        gt += kreg[j] > thr;
+        eq += kreg[j] == thr;
+      }
+    }
+  } else {
+    for (int i = lo; i < hi; ++i) {
+      const uint32_t key = keys[i];
+      gt += key > thr;
+      eq += key == thr;
+    }
   }
   uint32_t gt_incl = gt, eq_incl = eq;
 #pragma unroll
@@ -252,8 +275,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   uint32_t gt_before = warp_gt[warp] + gt_incl - gt;
   uint32_t eq_before = warp_eq[warp] + eq_incl - eq;
   int32_t* op = idx_out + static_cast<int64_t>(b) * k_stride;
-  for (int i = lo; i < hi; ++i) {
-    const uint32_t key = keys[i];
+  auto emit = [&](int i, uint32_t key) {
     const bool mine = i >= lo_i && i < hi_i;
     if (key > thr) {
       if (mine) op[gt_before + min(eq_before, take_eq)] = i;
@@ -262,6 +284,13 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
       if (mine && eq_before < take_eq) op[gt_before + eq_before] = i;
       ++eq_before;
     }
+  };
+  if (cached) {
+#pragma unroll
+    for (int j = 0; j < kRegKeys; ++j)
+      if (lo + j < hi) emit(lo + j, kreg[j]);
+  } else {
+    for (int i = lo; i < hi; ++i) emit(i, keys[i]);
   }
 }
 
