@@ -13,7 +13,10 @@
 // CTA leaves a unit, its warps merge their running (max, sum, output) through a 4 KB shared-memory
 // buffer; a unit held by one CTA is normalised and written at once, a unit shared by several CTAs
 // goes through global partials and is merged by whichever CTA arrives last (one atomic arrival
-// counter per unit, no spinning).
+// counter per unit, no spinning). How the rows are handed out is worked out by every CTA from the
+// lengths of all units (one round trip, a scan) or, for the pruned layers of a decode step, which
+// all see the same lengths and kept counts, once per step by attn_plan_kernel: a CTA then reads a
+// 64-byte record with its range, its unit and the unit's geometry.
 //
 // Data path: a block's 16 K rows and 16 V rows (256 bytes each) travel HBM -> shared memory with
 // 16-byte cp.async (marked evict-first in L2: cache rows are read once per layer), one full row
@@ -417,11 +420,11 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     float* logitA = (a.logits != nullptr && okA) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4) * a.n_stride : nullptr;
     float* logitB = (a.logits != nullptr && okB) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4 + 1) * a.n_stride : nullptr;
 
-    // Look-ahead stages, each one row behind the previous (so that no loaded value is needed in
-    // the iteration that loads it): P (row n+4) logical position of token `lane` (< 16) of this
-    // warp's block, a load from the index list for selected image tokens; R (row n+3) physical
-    // cache row, a block-table load for paged caches; I (row n+2) the cp.async copies; C (row n)
-    // the arithmetic.
+    // Look-ahead stages, each one block behind the previous (so that no loaded value is needed in
+    // the iteration that loads it): P (block n + kDepth + 2) logical position of token `lane % 16`
+    // of this warp's block, a load from the index list for selected image tokens; R (block
+    // n + kDepth + 1) physical cache row, a block-table load for paged caches; I (block n + kDepth)
+    // the cp.async copies; C (block n) the arithmetic.
     // A block is named by the list index jr of its first token (tok0 + 32 per block); it exists
     // while jr < lim. All 32 lanes run stages P and R (lanes 16-31 mirror lanes 0-15: no divergence).
     const int lim = min(sg.n_tok, tok0 + seg_rows * kRowTokens);

@@ -8,7 +8,7 @@ namespace fastocr {
 constexpr int kHeadDim = 128;
 constexpr int kMaxGroup = 8;          // query heads per KV head handled by one CTA
 constexpr int kAttnWarps = 2;         // warps per persistent attention CTA
-constexpr int kAttnCtasPerSm = 4;     // resident CTAs per SM (shared memory); a launch uses half of them
+constexpr int kAttnCtasPerSm = 4;     // resident CTAs per SM (registers and shared memory)
 constexpr int kMaxUnits = 512;        // sequences x KV heads per launch (their row prefix lives in shared memory)
 constexpr int kMaxPartsPerUnit = 16;  // CTAs sharing one unit in split mode (bounds the last CTA's merge)
 constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
