@@ -38,7 +38,6 @@ struct fastocr_ctx {
   // a pruned pass leaves one free (so that the next layer's launch can start beside it)
   int dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
   int sparse_ctas_per_sm = fastocr::kAttnCtasPerSm - 1;
-  int dense_depth = 2, sparse_depth = 3;
   unsigned long long* trace = nullptr;   // set only by debug builds
   unsigned trace_seq = 0;
   char err[512] = {0};
@@ -129,7 +128,6 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
   a.trace = nullptr;
 #endif
   a.wait_point = fastocr::kWaitAtStart;
-  a.depth = ctx->dense_depth;
   a.grid_ctas = ctx->sm_count * ctx->dense_ctas_per_sm;
   {
     // small batches: the kernel gives every unit at most kMaxPartsPerUnit CTAs; launch no more
@@ -254,7 +252,6 @@ AttnLaunch sparse_args(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
     }
     a.active_ctas = a.grid_ctas;
   }
-  a.depth = ctx->sparse_depth;
   return a;
 }
 
@@ -311,8 +308,6 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   // one partial slot per (CTA, unit) pair that can occur: CTAs + units
   if (const char* v = std::getenv("FASTOCR_DENSE_CTAS_PER_SM")) ctx->dense_ctas_per_sm = std::atoi(v);     // tuning knobs,
   if (const char* v = std::getenv("FASTOCR_SPARSE_CTAS_PER_SM")) ctx->sparse_ctas_per_sm = std::atoi(v);   // read once here
-  if (const char* v = std::getenv("FASTOCR_DENSE_DEPTH")) ctx->dense_depth = std::atoi(v);
-  if (const char* v = std::getenv("FASTOCR_SPARSE_DEPTH")) ctx->sparse_depth = std::atoi(v);
   if (ctx->dense_ctas_per_sm < 1 || ctx->dense_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
   if (ctx->sparse_ctas_per_sm < 1 || ctx->sparse_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->sparse_ctas_per_sm = fastocr::kAttnCtasPerSm - 1;
   ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * fastocr::kAttnCtasPerSm +

@@ -129,12 +129,12 @@ __device__ __forceinline__ void store_pair(void* out, int is_fp32, int64_t index
 struct SeqGeom {
   int vs, N, kept_vis, n_tok;
 };
-__device__ __forceinline__ SeqGeom load_geom(const AttnLaunch& a, int b) {
+__device__ __forceinline__ SeqGeom load_geom(const AttnLaunch& a, int b, bool pruned) {
   SeqGeom s;
   const int S = a.seq_len[b];
   s.vs = a.vis_start[b];
   s.N = a.vis_len[b];
-  if (a.idx != nullptr) {
+  if (pruned) {
     const int kk = a.kcount[b];
     s.kept_vis = kk < 0 ? 0 : (kk > s.N ? s.N : kk);
   } else {
@@ -189,9 +189,22 @@ __device__ __forceinline__ bool split_rule(int units, int grid, int total_rows, 
          static_cast<int64_t>(longest_unit) * units <= static_cast<int64_t>(total_rows) + total_rows / 8;
 }
 
-// kDepth: how many blocks ahead of its use a copy is issued (1 .. kStages)
-template <int G, bool HAS_V, int kDepth>
+// What a launch does is fixed at compile time, so that the main loop carries no code it does not
+// run (the page-table arithmetic alone, present but skipped, cost a pruned pass 6 %):
+//   kModePruned  K = T u F: index list, K and V, no logits   (copy distance 3: more latency hidden per warp)
+//   kModeScores  full cache, K and V, logits and per-head statistics kept for the selection
+//   kModeDense   full cache, K and V
+//   kModeKeys    full cache, K only, logits and statistics (stand-alone scoring)
+// (copy distance 2 for the full-cache passes: they saturate HBM anyway and run faster with fewer
+// requests queued), each for contiguous and for paged caches.
+enum : int { kModePruned = 0, kModeScores = 1, kModeDense = 2, kModeKeys = 3 };
+
+template <int G, int MODE, bool PAGED>
 __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(const AttnLaunch a) {
+  constexpr bool HAS_V = MODE != kModeKeys;
+  constexpr bool HAS_IDX = MODE == kModePruned;
+  constexpr bool LOGITS = MODE == kModeScores || MODE == kModeKeys;
+  constexpr int kDepth = MODE == kModePruned ? 3 : 2;   // blocks a copy is issued ahead of its use (<= kStages)
   static_assert(kDepth >= 1 && kDepth <= kStages, "copy distance");
   extern __shared__ __align__(16) unsigned char smem[];
   using L = Smem<HAS_V>;
@@ -253,7 +266,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) {
       const int uu = min(i * kThreads + tid, units - 1);
-      gq[i] = load_geom(a, uu / Hkv);
+      gq[i] = load_geom(a, uu / Hkv, HAS_IDX);
     }
     int longest = 0;
 #pragma unroll
@@ -332,7 +345,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 
   const float scale_log2 = a.sm_scale * 1.4426950408889634f;
   const int64_t row_elems = static_cast<int64_t>(Hkv) * kHeadDim;
-  const int64_t seq_elems = a.page_size > 0 ? 0 : a.seq_stride_tokens * row_elems;
+  const int64_t seq_elems = PAGED ? 0 : a.seq_stride_tokens * row_elems;
   const int c16 = lane & 15, half = lane >> 4;          // copy role: chunk of a row, which row of a pair
   const uint32_t smem_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
   const uint32_t ring_warp = smem_u32 + L::ring + warp * kStages * L::kStageBytes;
@@ -391,7 +404,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       sg.vs = gq.x; sg.N = gq.y; sg.kept_vis = gq.z; sg.n_tok = gq.w;
       __syncthreads();                                 // both warps have read it: the ring may be written
     } else {
-      sg = load_geom(a, b);
+      sg = load_geom(a, b, HAS_IDX);
     }
     const int tok0 = (seg_begin - ubeg) * kRowTokens + warp * kBlockTokens;   // this warp's first token of the segment
     // this lane's 16-byte chunk of cache row 0 of the unit (a row is row_bytes long)
@@ -417,8 +430,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     float mA = -INFINITY, mB = -INFINITY;              // reference maxima (identical in the 8 lanes that share t4)
     float lA = 0.f, lB = 0.f;                          // this lane's part of the sums (tokens g8, 8 + g8 of every block)
     const bool okA = 2 * t4 < G, okB = 2 * t4 + 1 < G;
-    float* logitA = (a.logits != nullptr && okA) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4) * a.n_stride : nullptr;
-    float* logitB = (a.logits != nullptr && okB) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4 + 1) * a.n_stride : nullptr;
+    float* logitA = (LOGITS && okA) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4) * a.n_stride : nullptr;
+    float* logitB = (LOGITS && okB) ? a.logits + (static_cast<int64_t>(u) * G + 2 * t4 + 1) * a.n_stride : nullptr;
 
     // Look-ahead stages, each one block behind the previous (so that no loaded value is needed in
     // the iteration that loads it): P (block n + kDepth + 2) logical position of token `lane % 16`
@@ -430,14 +443,14 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     const int lim = min(sg.n_tok, tok0 + seg_rows * kRowTokens);
     const int tl = lane & (kBlockTokens - 1);
     const int vis_end = sg.vs + sg.kept_vis, text_shift = sg.N - sg.kept_vis;
-    const int32_t* idx_row = a.idx != nullptr ? a.idx + static_cast<int64_t>(b) * a.k_stride - sg.vs : nullptr;
-    const int32_t* bt_row = a.page_size > 0 ? a.block_table + static_cast<int64_t>(b) * a.max_pages : nullptr;
+    const int32_t* idx_row = HAS_IDX ? a.idx + static_cast<int64_t>(b) * a.k_stride - sg.vs : nullptr;
+    const int32_t* bt_row = PAGED ? a.block_table + static_cast<int64_t>(b) * a.max_pages : nullptr;
     auto stage_p = [&](int jr, int& pos, bool& is_idx) {     // is_idx: pos is a raw index-list entry, checked in stage R
       is_idx = false;
       if (jr < lim) {
         const int j = min(jr + tl, sg.n_tok - 1);
         pos = j;
-        if (idx_row != nullptr) {                      // kept set: text before | selected image | text after
+        if (HAS_IDX) {                                 // kept set: text before | selected image | text after
           if (j >= vis_end) {
             pos = j + text_shift;
           } else if (j >= sg.vs) {
@@ -456,7 +469,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           }
           pos += sg.vs;
         }
-        if (bt_row != nullptr) {
+        if (PAGED) {
           const int page = __ldg(bt_row + pos / a.page_size);
           pos = page * a.page_size + pos % a.page_size;
         }
@@ -494,7 +507,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     // sequence's cache span, and the first touch of a page by this SM costs a translation miss in
     // the middle of the stream. Touch every page of the span now, all at once (one line each, L2
     // only): lanes 0-15 of warp 0 for K, lanes 16-31 for V.
-    if (a.idx != nullptr && a.page_size == 0 && warp == 0) {
+    if (HAS_IDX && !PAGED && warp == 0) {
       const int64_t span = static_cast<int64_t>(sg.n_tok - sg.kept_vis + sg.N) * row_elems * 2;   // bytes, whole sequence
       const char* base = reinterpret_cast<const char*>(half ? static_cast<const void*>(a.v) : a.k) +
                          (b * seq_elems + g * kHeadDim) * 2;
@@ -580,7 +593,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           const bool valid = ((i & 1) ? okB : okA) && rem > 8 * (i >> 1);
           x[i] = valid ? x[i] : -INFINITY;
           float* lrow = (i & 1) ? logitB : logitA;
-          if (lrow != nullptr && valid) {              // dense / scoring mode: position == list index
+          if (LOGITS && lrow != nullptr && valid) {              // dense / scoring mode: position == list index
             const int rel = tok - sg.vs;
             if (rel >= 0 && rel < sg.N && rel < a.n_stride) lrow[rel] = x[i];
           }
@@ -797,7 +810,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 #pragma unroll
             for (int i = 0; i < 8; i += 2) store_pair(a.out, a.out_is_fp32, oi + i, num[it][i] * inv, num[it][i + 1] * inv);
           }
-          if ((e & 15) == 0 && a.stats != nullptr) {
+          if (LOGITS && (e & 15) == 0) {
             a.stats[(head0 + h) * 2 + 0] = M[it];
             a.stats[(head0 + h) * 2 + 1] = den[it];
           }
@@ -829,7 +842,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       for (int i = tid; i < G * kHeadDim / 2; i += kThreads)
         if (HAS_V) store_pair(a.out, a.out_is_fp32, head0 * kHeadDim + 2 * i, 0.f, 0.f);
       for (int i = tid; i < G; i += kThreads)
-        if (a.stats != nullptr) {
+        if (LOGITS) {
           a.stats[(head0 + i) * 2 + 0] = -INFINITY;
           a.stats[(head0 + i) * 2 + 1] = 0.f;
         }
@@ -849,7 +862,7 @@ __global__ void __launch_bounds__(kMaxUnits) attn_plan_kernel(const AttnLaunch a
   SeqGeom sg = {0, 0, 0, 0};
   int rows = 0;
   if (tid < units) {
-    sg = load_geom(a, tid / Hkv);
+    sg = load_geom(a, tid / Hkv, a.idx != nullptr);
     rows = (sg.n_tok + kRowTokens - 1) / kRowTokens;
   }
   int incl = rows, longest = rows;
@@ -899,7 +912,7 @@ __global__ void __launch_bounds__(kMaxUnits) attn_plan_kernel(const AttnLaunch a
       if (r1 > prefix_s[u + 1]) valid = 0;             // the range spans several units
       if (r0 >= r1) { u = 0; r0 = r1 = 0; }
     }
-    const SeqGeom g = load_geom(a, u / Hkv);
+    const SeqGeom g = load_geom(a, u / Hkv, a.idx != nullptr);
     int4* rec = plan_out + 4 * static_cast<int64_t>(c);
     rec[0] = make_int4(valid, u, r0, r1);
     rec[1] = make_int4(prefix_s[u], prefix_s[u + 1], split_units ? 1 : 0, parts);
@@ -959,20 +972,26 @@ __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restric
   }
 }
 
-template <int G, bool HAS_V, int DEPTH>
+template <int G, int MODE, bool PAGED>
 cudaError_t launch_partial_t(const AttnLaunch& a, cudaStream_t s) {
-  const cudaError_t e = launch_pdl(attn_stream_kernel<G, HAS_V, DEPTH>, dim3(a.grid_ctas), dim3(kThreads), Smem<HAS_V>::total, s, a);
+  const cudaError_t e = launch_pdl(attn_stream_kernel<G, MODE, PAGED>, dim3(a.grid_ctas), dim3(kThreads),
+                                   Smem<MODE != kModeKeys>::total, s, a);
   count_launches(1);
   return e;
 }
 
-template <int G, bool HAS_V, int DEPTH>
+template <int G, int MODE>
+cudaError_t launch_mode_t(const AttnLaunch& a, cudaStream_t s) {
+  return a.page_size > 0 ? launch_partial_t<G, MODE, true>(a, s) : launch_partial_t<G, MODE, false>(a, s);
+}
+
+template <int G, int MODE, bool PAGED>
 cudaError_t configure_t() {
-  cudaError_t e = cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V, DEPTH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       Smem<HAS_V>::total);
+  cudaError_t e = cudaFuncSetAttribute(attn_stream_kernel<G, MODE, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       Smem<MODE != kModeKeys>::total);
   if (e != cudaSuccess) return e;
   // all of the SM's L1/shared array as shared memory: four CTAs must fit
-  return cudaFuncSetAttribute(attn_stream_kernel<G, HAS_V, DEPTH>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+  return cudaFuncSetAttribute(attn_stream_kernel<G, MODE, PAGED>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
 }
 
 }  // namespace
@@ -988,12 +1007,18 @@ cudaError_t launch_attn_plan(const AttnLaunch& a, int4* plan_out, cudaStream_t s
 
 cudaError_t launch_attn_partial(const AttnLaunch& a, cudaStream_t s) {
   const int G = a.num_q_heads / a.num_kv_heads;
-  const bool has_v = a.v != nullptr;
+  // the mode follows from what the launch was given
+  const int mode = a.idx != nullptr ? kModePruned : (a.v == nullptr ? kModeKeys : (a.logits != nullptr ? kModeScores : kModeDense));
+  if (mode == kModeKeys && a.logits == nullptr) return cudaErrorInvalidValue;
   switch (G) {
-#define X(g)                                                                                  \
-  case g:                                                                                     \
-    if (!has_v) return launch_partial_t<g, false, 2>(a, s);                                   \
-    return a.depth >= 3 ? launch_partial_t<g, true, 3>(a, s) : launch_partial_t<g, true, 2>(a, s);
+#define X(g)                                                      \
+  case g:                                                         \
+    switch (mode) {                                               \
+      case kModePruned: return launch_mode_t<g, kModePruned>(a, s); \
+      case kModeScores: return launch_mode_t<g, kModeScores>(a, s); \
+      case kModeDense: return launch_mode_t<g, kModeDense>(a, s);   \
+      default: return launch_mode_t<g, kModeKeys>(a, s);            \
+    }
     FASTOCR_FOR_EACH_GROUP(X)
 #undef X
     default:
@@ -1007,12 +1032,13 @@ cudaError_t configure_kernels() {
   // kernels in between do not trigger a reconfiguration
   if ((e = cudaFuncSetAttribute(scores_finalize_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(image_mass_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
-#define X(g)                                                   \
-  if ((e = configure_t<g, true, 2>()) != cudaSuccess) return e;  \
-  if ((e = configure_t<g, true, 3>()) != cudaSuccess) return e;  \
-  if ((e = configure_t<g, false, 2>()) != cudaSuccess) return e;
+#define Y(g, m)                                                    \
+  if ((e = configure_t<g, m, false>()) != cudaSuccess) return e;   \
+  if ((e = configure_t<g, m, true>()) != cudaSuccess) return e;
+#define X(g) Y(g, kModePruned) Y(g, kModeScores) Y(g, kModeDense) Y(g, kModeKeys)
   FASTOCR_FOR_EACH_GROUP(X)
 #undef X
+#undef Y
   return cudaSuccess;
 }
 
@@ -1020,9 +1046,9 @@ cudaError_t configure_kernels() {
 // debug builds: resident CTAs per SM the runtime grants the 7-head attention kernel
 extern "C" int fastocr_debug_occupancy() {
   int n = -1;
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_stream_kernel<7, true, 2>, kThreads, Smem<true>::total);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_stream_kernel<7, kModeDense, false>, kThreads, Smem<true>::total);
   cudaFuncAttributes fa;
-  cudaFuncGetAttributes(&fa, attn_stream_kernel<7, true, 2>);
+  cudaFuncGetAttributes(&fa, attn_stream_kernel<7, kModeDense, false>);
   return n * 1000 + fa.numRegs;
 }
 #endif

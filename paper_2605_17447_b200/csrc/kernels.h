@@ -86,8 +86,6 @@ struct AttnLaunch {
   int32_t grid_ctas;          // CTAs launched (kAttnWarps warps each)
   int32_t active_ctas;        // CTAs that take work (<= grid_ctas); the rest exit at once
   int32_t wait_point;         // where the kernel waits for earlier kernels: kWaitAtStart / kWaitAfterSetup / kWaitBeforeWrites
-  int32_t depth;              // blocks a copy is issued ahead of its use (1..3): deeper hides more latency per warp,
-                              // shallower keeps fewer requests queued when the pass saturates HBM anyway
   const int4* plan;           // NULL or one 64-byte record per CTA written by launch_attn_plan for this very launch
                               // shape (grid, lengths, kept counts): the CTA's range and unit, ready made
   // workspace

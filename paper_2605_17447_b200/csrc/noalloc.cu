@@ -125,7 +125,6 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   a.grid_ctas = grid;
   a.active_ctas = grid;
   a.wait_point = fastocr::kWaitAtStart;
-  a.depth = 3;
   a.part_acc = reinterpret_cast<float*>(s.scratch);
   a.part_ml = reinterpret_cast<float*>(s.scratch + kAccBytes);
   a.counters = reinterpret_cast<int32_t*>(counters);
