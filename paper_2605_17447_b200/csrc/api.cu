@@ -109,6 +109,8 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
   a.block_table = kv->block_table;
   a.max_pages = kv->max_pages;
   a.page_size = kv->page_size;
+  a.page_shift = 0;
+  while ((1 << a.page_shift) < kv->page_size) ++a.page_shift;
   a.seq_len = kv->seq_len;
   a.vis_start = kv->vis_start;
   a.vis_len = kv->vis_len;

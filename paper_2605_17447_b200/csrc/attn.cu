@@ -463,15 +463,15 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     auto stage_r = [&](int jr, int pos, bool is_idx, int& row) {
       if (jr < lim) {
         if (is_idx) {
-          if (pos < 0 || pos >= sg.N) {                // never read outside the image span
+          if (__builtin_expect(static_cast<unsigned>(pos) >= static_cast<unsigned>(sg.N), 0)) {   // never read outside the image span
             if (lane < kBlockTokens) atomicAdd(a.fault_counter, 1ULL);
             pos = pos < 0 ? 0 : sg.N - 1;
           }
           pos += sg.vs;
         }
         if (PAGED) {
-          const int page = __ldg(bt_row + pos / a.page_size);
-          pos = page * a.page_size + pos % a.page_size;
+          const int page = __ldg(bt_row + (pos >> a.page_shift));   // page sizes are powers of two
+          pos = (page << a.page_shift) + (pos & (a.page_size - 1));
         }
         row = pos;
       }
@@ -599,7 +599,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           }
         }
         float mxA = fmaxf(x[0], x[2]), mxB = fmaxf(x[1], x[3]);
-        if (__any_sync(0xffffffffu, mxA > mA + kRescaleSlack || mxB > mB + kRescaleSlack)) {
+        if (__builtin_expect(__any_sync(0xffffffffu, mxA > mA + kRescaleSlack || mxB > mB + kRescaleSlack), 0)) {
 #pragma unroll
           for (int off = 4; off < 32; off <<= 1) {     // over the 8 lanes that share t4
             mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, off));

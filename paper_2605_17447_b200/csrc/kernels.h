@@ -72,7 +72,8 @@ struct AttnLaunch {
   int64_t seq_stride_tokens;
   const int32_t* block_table;
   int32_t max_pages;
-  int32_t page_size;          // 0 = contiguous
+  int32_t page_size;          // 0 = contiguous; else a power of two
+  int32_t page_shift;         // log2(page_size)
   const int32_t* seq_len;
   const int32_t* vis_start;
   const int32_t* vis_len;

@@ -111,6 +111,7 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   a.block_table = kv->block_table;
   a.max_pages = kv->max_pages;
   a.page_size = kv->page_size;
+  while ((1 << a.page_shift) < kv->page_size) ++a.page_shift;
   a.seq_len = kv->seq_len;
   a.vis_start = kv->vis_start;
   a.vis_len = kv->vis_len;
