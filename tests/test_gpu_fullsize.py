@@ -55,11 +55,11 @@ def test_full_size_layer_chain_against_oracle_on_sampled_sequences():
     # the decode step (scores formed inside the selection kernel, a cluster of CTAs per sequence,
     # launches overlapping) gives the same bits as the separate calls
     fix = torch.full((B, k), -1, dtype=torch.int32, device=dev)
-    out2 = torch.empty(2, B, H, 128, dtype=torch.float32, device=dev)
-    have = fo.fastocr_decode_step(ctx, [kv, kv], torch.stack([q, q]), out2, [True, False], kd, fix, False, N)
+    out2 = torch.empty(3, B, H, 128, dtype=torch.float32, device=dev)    # two pruned layers: they run from a launch plan
+    have = fo.fastocr_decode_step(ctx, [kv, kv, kv], torch.stack([q, q, q]), out2, [True, False, False], kd, fix, False, N)
     torch.cuda.synchronize()
     assert have and torch.equal(fix, idx)
-    assert torch.equal(out2[0], dense) and torch.equal(out2[1], out)
+    assert torch.equal(out2[0], dense) and torch.equal(out2[1], out) and torch.equal(out2[2], out)
     # sampled sequences against the oracle, element by element
     for b in (0, 17, 63):
         qc, Kc, Vc = q[b].cpu(), K[b].cpu(), V[b].cpu()

@@ -238,17 +238,27 @@ def test_fixation_window_is_selected_on_config0(fo, ctx):
     assert len(top9 & sel) == 9
 
 
-def test_decode_step_matches_algorithm_trace(fo, ctx):
-    L, spans = 5, [(6, 300, 20), (3, 170, 41)]
-    base = make_case(600, spans)
+@pytest.mark.parametrize("paged,spans", [(False, [(6, 300, 20), (3, 170, 41)]), (True, [(6, 300, 20), (3, 170, 41)]),
+                                         (False, [(5, 200, 30)] * 3), (True, [(5, 200, 30)] * 3)])
+def test_decode_step_matches_algorithm_trace(fo, ctx, paged, spans):
+    """Ragged and uniform batches (the latter get valid launch-plan records), contiguous and paged caches."""
+    L = 5
+    base = make_case(600, spans, page_size=16 if paged else 0)
     from workloads import make_kv, normal_bf16, stream_key
     layers_cpu, views = [], []
-    for l in range(L):
+    shared = None                                        # one set of length arrays for all layers, as a caller
+    for l in range(L):                                   # would have (that is what makes a launch plan usable)
         K, V = make_kv(600, l, base.B, max(base.seq_len), base.Hkv, 128)
         q = normal_bf16(stream_key(600, 55, l), (base.B, base.H, 128))
-        c = type(base)(base.B, base.H, base.Hkv, base.seq_len, base.vis_start, base.vis_len, K, V, q)
+        c = type(base)(base.B, base.H, base.Hkv, base.seq_len, base.vis_start, base.vis_len, K, V, q,
+                       base.page_size, base.block_table, base.num_pages)
         layers_cpu.append(c)
-        views.append(c.device_view())
+        v = c.device_view()
+        if shared is None:
+            shared = (v.seq_len, v.vis_start, v.vis_len)
+        v = fo.KVView(v.k, v.v, shared[0], shared[1], shared[2], base.H, max(base.seq_len), SCALE,
+                      block_table=v.block_table if paged else None)
+        views.append(v)
     q_all = torch.stack([c.q for c in layers_cpu]).cuda()
     ks = [oracle.kept_count(n, 0.1) for n in base.vis_len]
     kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
