@@ -388,6 +388,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     u = lo;
   }
   int seg_begin = r0;
+  int bad_entries = 0;                                 // index-list entries outside the image span (clamped), counted by lanes 0-15
   if (a.wait_point == kWaitAfterSetup) {               // before index-list reads and logits writes
     wait_for_prior_grids();
     dependents_may_launch();
@@ -463,11 +464,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     auto stage_r = [&](int jr, int pos, bool is_idx, int& row) {
       if (jr < lim) {
         if (is_idx) {
-          if (__builtin_expect(static_cast<unsigned>(pos) >= static_cast<unsigned>(sg.N), 0)) {   // never read outside the image span
-            if (lane < kBlockTokens) atomicAdd(a.fault_counter, 1ULL);
-            pos = pos < 0 ? 0 : sg.N - 1;
-          }
-          pos += sg.vs;
+          const int inside = min(max(pos, 0), sg.N - 1);      // never read outside the image span
+          bad_entries += inside != pos;
+          pos = inside + sg.vs;
         }
         if (PAGED) {
           const int page = __ldg(bt_row + (pos >> a.page_shift));   // page sizes are powers of two
@@ -827,6 +826,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     a.trace[(blockIdx.x * kAttnWarps + warp) * 16 + 7] = (static_cast<unsigned long long>(trace_look) << 32) | trace_pv;
   }
 #endif
+
+  if (HAS_IDX && bad_entries != 0 && lane < kBlockTokens) atomicAdd(a.fault_counter, static_cast<unsigned long long>(bad_entries));
 
   // A kernel of this library must not complete before its predecessor has (later kernels rely on
   // "my predecessor is done, hence everything before it"). CTAs that wrote only their own output
