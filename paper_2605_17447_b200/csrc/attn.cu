@@ -924,6 +924,7 @@ __global__ void __launch_bounds__(kMaxUnits) attn_plan_kernel(const AttnLaunch a
 
 constexpr int kFinalizeThreads = 256;
 
+// four tokens per thread (16-byte loads when the layout allows), eight heads' loads in flight
 __global__ void __launch_bounds__(kFinalizeThreads) scores_finalize_kernel(
     const float* __restrict__ logits, const float* __restrict__ stats, const int32_t* __restrict__ vis_len,
     int num_q_heads, int n_stride_logits, float* __restrict__ scores, int n_stride) {
@@ -931,26 +932,50 @@ __global__ void __launch_bounds__(kFinalizeThreads) scores_finalize_kernel(
   wait_for_prior_grids();
   dependents_may_launch();
   const int b = blockIdx.y;
-  const int N = vis_len[b];
+  const int N = min(min(vis_len[b], n_stride), n_stride_logits);
+  const int i0 = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (blockIdx.x * blockDim.x * 4 >= N) return;        // the whole CTA is past the end
   for (int i = threadIdx.x; i < num_q_heads; i += blockDim.x) {
     st[2 * i] = stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2];
     st[2 * i + 1] = 1.0f / stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2 + 1];
   }
   __syncthreads();
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= N || i >= n_stride || i >= n_stride_logits) return;
-  const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + i;
-  float s = 0.f;
-  int h = 0;
-  for (; h + 4 <= num_q_heads; h += 4) {               // four loads in flight; summed in head order
-    float x[4];
+  if (i0 >= N) return;
+  const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + i0;
+  const bool full = i0 + 4 <= N && (n_stride_logits & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int h0 = 0; h0 < num_q_heads; h0 += 8) {        // summed in head order
+    float4 x[8];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) x[j] = lp[static_cast<int64_t>(h + j) * n_stride_logits];
+    for (int j = 0; j < 8; ++j) {
+      x[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (h0 + j < num_q_heads) {
+        const float* src = lp + static_cast<int64_t>(h0 + j) * n_stride_logits;
+        if (full) {
+          x[j] = __ldcg(reinterpret_cast<const float4*>(src));
+        } else {
+          x[j].x = __ldcg(src);
+          if (i0 + 1 < N) x[j].y = __ldcg(src + 1);
+          if (i0 + 2 < N) x[j].z = __ldcg(src + 2);
+          if (i0 + 3 < N) x[j].w = __ldcg(src + 3);
+        }
+      }
+    }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) s = score_add_head(s, x[j], st[2 * (h + j)], st[2 * (h + j) + 1]);
+    for (int j = 0; j < 8; ++j) {
+      if (h0 + j < num_q_heads) {
+        const float m = st[2 * (h0 + j)], inv = st[2 * (h0 + j) + 1];
+        acc[0] = score_add_head(acc[0], x[j].x, m, inv);
+        acc[1] = score_add_head(acc[1], x[j].y, m, inv);
+        acc[2] = score_add_head(acc[2], x[j].z, m, inv);
+        acc[3] = score_add_head(acc[3], x[j].w, m, inv);
+      }
+    }
   }
-  for (; h < num_q_heads; ++h) s = score_add_head(s, lp[static_cast<int64_t>(h) * n_stride_logits], st[2 * h], st[2 * h + 1]);
-  scores[static_cast<int64_t>(b) * n_stride + i] = score_finish(s, num_q_heads);
+  float* out = scores + static_cast<int64_t>(b) * n_stride + i0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    if (i0 + j < N) out[j] = score_finish(acc[j], num_q_heads);
 }
 
 __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restrict__ scores, int n_stride,
@@ -1058,7 +1083,7 @@ cudaError_t launch_scores_finalize(const float* logits, const float* stats, cons
                                    int32_t num_q_heads, int32_t n_stride_logits, int32_t max_vis_len, float* scores,
                                    int32_t n_stride, cudaStream_t s) {
   if (max_vis_len <= 0) return cudaSuccess;
-  dim3 grid((max_vis_len + kFinalizeThreads - 1) / kFinalizeThreads, batch);
+  dim3 grid((max_vis_len + 4 * kFinalizeThreads - 1) / (4 * kFinalizeThreads), batch);
   const cudaError_t e = launch_pdl(scores_finalize_kernel, grid, dim3(kFinalizeThreads), num_q_heads * 2 * sizeof(float), s,
                                    logits, stats, vis_len, num_q_heads, n_stride_logits, scores, n_stride);
   count_launches(1);
