@@ -183,6 +183,34 @@ def test_sparse_tau_one_equals_dense_and_tau_zero_is_text_only(fo, ctx):
     _check_out(out, ref)
 
 
+def test_sequence_with_nothing_to_attend_gets_zeros(fo, ctx):
+    """A sequence without text tokens and with a kept count of 0 attends nothing: its outputs are
+    zeros, the others are unaffected; stand-alone and inside a decode step (whose launch plan must
+    step aside for such a batch)."""
+    case = make_case(450, spans=[(4, 200, 10), (0, 150, 0), (3, 90, 5)])
+    kv = case.device_view(poison=True)
+    q = case.q.cuda()
+    ks = [oracle.kept_count(case.vis_len[0], 0.1), 0, oracle.kept_count(case.vis_len[2], 0.1)]
+    g = torch.Generator().manual_seed(5)
+    idx = torch.zeros(case.B, max(ks), dtype=torch.int32)
+    for b in range(case.B):
+        idx[b, :ks[b]] = torch.randperm(case.vis_len[b], generator=g)[:ks[b]].sort().values.int()
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    ref = torch.stack([oracle.sparse(*case.seq(b), SCALE, case.vis_start[b], case.vis_len[b], idx[b, :ks[b]], True)
+                       if b != 1 else torch.zeros(case.H, 128) for b in range(case.B)])
+    out = torch.full((case.B, case.H, 128), 7.0, dtype=torch.float32, device="cuda")
+    fo.fastocr_sparse_decode_attn(ctx, kv, q, idx.cuda(), kd, out)
+    _check_out(out, ref)
+    assert float(out[1].abs().max()) == 0.0
+    out3 = torch.full((3, case.B, case.H, 128), 7.0, dtype=torch.float32, device="cuda")
+    fix = idx.cuda().clone()
+    assert fo.fastocr_decode_step(ctx, [kv, kv, kv], torch.stack([q, q, q]), out3, [False, False, False], kd, fix, True,
+                                  max(case.vis_len))
+    for l in range(3):
+        _check_out(out3[l], ref)
+        assert float(out3[l, 1].abs().max()) == 0.0
+
+
 def _near_tie_only(gpu_idx, ref_idx, ref_scores, k):
     """Selections may differ only in tokens whose oracle score is within 1e-5 (relative) of the
     oracle's k-th score."""
