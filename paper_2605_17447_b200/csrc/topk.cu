@@ -234,21 +234,29 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
         eq += kreg[j] == thr;
       }
     }
-  } else {
-    for (int i = lo; i < hi; ++i) {
-      const uint32_t key = keys[i];
-      gt += key > thr;
-      eq += key == thr;
+  }
+  // Longer sequences: every warp walks a contiguous region 32 keys at a time (lane = key, no bank
+  // conflicts) and counts with ballots; the counts are the same in all lanes of the warp.
+  const int per_warp = (((N + kTopkWarps - 1) / kTopkWarps) + 31) & ~31;
+  const int w_lo = min(warp * per_warp, N), w_hi = min(w_lo + per_warp, N);
+  if (!cached) {
+    for (int base = w_lo; base < w_hi; base += 32) {
+      const uint32_t key = base + lane < w_hi ? keys[base + lane] : 0u;   // 0 is below every threshold of a non-empty selection
+      const bool live = base + lane < w_hi;
+      gt += __popc(__ballot_sync(0xffffffffu, live && key > thr));
+      eq += __popc(__ballot_sync(0xffffffffu, live && key == thr));
     }
   }
   uint32_t gt_incl = gt, eq_incl = eq;
+  if (cached) {
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t a = __shfl_up_sync(0xffffffffu, gt_incl, o);
-    const uint32_t e = __shfl_up_sync(0xffffffffu, eq_incl, o);
-    if (lane >= o) {
-      gt_incl += a;
-      eq_incl += e;
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t a = __shfl_up_sync(0xffffffffu, gt_incl, o);
+      const uint32_t e = __shfl_up_sync(0xffffffffu, eq_incl, o);
+      if (lane >= o) {
+        gt_incl += a;
+        eq_incl += e;
+      }
     }
   }
   if (lane == 31) {
@@ -290,7 +298,20 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
     for (int j = 0; j < kRegKeys; ++j)
       if (lo + j < hi) emit(lo + j, kreg[j]);
   } else {
-    for (int i = lo; i < hi; ++i) emit(i, keys[i]);
+    const uint32_t below = (1u << lane) - 1u;            // lanes holding lower indices
+    uint32_t gt_run = warp_gt[warp], eq_run = warp_eq[warp];
+    for (int base = w_lo; base < w_hi; base += 32) {
+      const int i = base + lane;
+      const bool live = i < w_hi;
+      const uint32_t key = live ? keys[i] : 0u;
+      const uint32_t m_gt = __ballot_sync(0xffffffffu, live && key > thr);
+      const uint32_t m_eq = __ballot_sync(0xffffffffu, live && key == thr);
+      gt_before = gt_run + __popc(m_gt & below);
+      eq_before = eq_run + __popc(m_eq & below);
+      if (live) emit(i, key);
+      gt_run += __popc(m_gt);
+      eq_run += __popc(m_eq);
+    }
   }
 }
 
