@@ -180,15 +180,18 @@ __device__ __forceinline__ unsigned long long trace_now() {
 
 // Ways to hand out rows (see the kernel): 0 = equal ranges of all rows laid end to end; else every
 // unit is cut into this many equal parts, one CTA each. Units of similar length get as many parts as
-// the grid allows; a ragged batch of short units gets one CTA per unit (the CTAs then finish at
-// different times, but none shares a unit with another: no partial results through global memory,
-// hence no waiting for the previous kernel, and launches keep overlapping).
-constexpr int kShortUnitRows = 64;
-__device__ __forceinline__ int split_rule(int units, int grid, int total_rows, int longest_unit) {
+// the grid allows. A ragged batch of index-list units gets one CTA per unit when the units number at
+// least a fifth of the grid and none is far longer than the average: the CTAs then finish at
+// different times, but none shares a unit with another, so there are no partial results through
+// global memory, hence no waiting for the previous kernel, and the next layers' launches (two or
+// three are in flight) fill the idle slots. (Full-cache passes overlap far less and their units are
+// long: one CTA per unit left them 2.6x slower than equal ranges, so they keep the ranges.)
+constexpr int kOwnUnitMaxRows = 512;
+__device__ __forceinline__ int split_rule(int units, int grid, int total_rows, int longest_unit, bool index_list) {
   if (units > grid || total_rows >= kLongRangeRows * grid) return 0;
-  if (static_cast<int64_t>(longest_unit) * units <= static_cast<int64_t>(total_rows) + total_rows / 8)
-    return min(grid / units, kMaxPartsPerUnit);
-  return longest_unit <= kShortUnitRows ? 1 : 0;
+  const int64_t padded = static_cast<int64_t>(longest_unit) * units;
+  if (padded <= static_cast<int64_t>(total_rows) + total_rows / 8) return min(grid / units, kMaxPartsPerUnit);
+  return (index_list && 5 * units >= grid && longest_unit <= kOwnUnitMaxRows && padded <= 2 * static_cast<int64_t>(total_rows)) ? 1 : 0;
 }
 
 // What a launch does is fixed at compile time, so that the main loop carries no code it does not
@@ -322,7 +325,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   // pipeline refill) and a unit that fits one CTA needs no global merge. Otherwise (ragged
   // batches, more units than CTAs, or long ranges where a few merges are negligible): all rows
   // laid end to end and cut into equal ranges.
-  const int parts_rule = planned ? 0 : split_rule(units, grid, total_rows, longest_unit);
+  const int parts_rule = planned ? 0 : split_rule(units, grid, total_rows, longest_unit, HAS_IDX);
   const bool split_units = planned ? plan1.z != 0 : parts_rule > 0;
   const int parts = planned ? plan1.w : max(parts_rule, 1);     // CTAs per unit
   const int per_cta = planned ? plan2.x : (total_rows + grid - 1) / grid;   // rows per CTA (equal-range mode)
@@ -889,7 +892,7 @@ __global__ void __launch_bounds__(kMaxUnits) attn_plan_kernel(const AttnLaunch a
   if (tid == 0) prefix_s[0] = 0;
   const int any_empty = __syncthreads_or(tid < units && rows == 0);
   const int total_rows = prefix_s[units];
-  const int parts_rule = split_rule(units, grid, total_rows, longest);
+  const int parts_rule = split_rule(units, grid, total_rows, longest, true);
   const bool split_units = parts_rule > 0;
   const int parts = max(parts_rule, 1);
   const int per_cta = (total_rows + grid - 1) / grid;
