@@ -233,6 +233,12 @@ fastocr_status fastocr_profile_end(fastocr_ctx* ctx, double* ms_per_class, int64
 /* Number of kernels this library has launched on any context since load (for bench accounting). */
 int64_t fastocr_launch_count(void);
 
+/* Of those, the pruned-attention launches that ran one thread-block cluster per (sequence, KV head)
+ * unit, whose pieces are merged through distributed shared memory instead of global memory (chosen
+ * by the library for short passes over sequences of similar length; Eq. 2 second case either way).
+ * For tests and tuning. */
+int64_t fastocr_cluster_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -51,6 +51,7 @@ EXPORTS = {
     "fastocr_profile_begin": (C.c_int, [C.c_void_p, C.c_int32, C.c_int]),
     "fastocr_profile_end": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "fastocr_launch_count": (C.c_int64, []),
+    "fastocr_cluster_launch_count": (C.c_int64, []),
 }
 
 _lib = None

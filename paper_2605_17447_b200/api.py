@@ -155,6 +155,10 @@ def launch_count() -> int:
     return int(_lib.load().fastocr_launch_count())
 
 
+def cluster_launch_count() -> int:
+    return int(_lib.load().fastocr_cluster_launch_count())
+
+
 def fastocr_dense_decode_attn(ctx: Context, kv: KVView, q: torch.Tensor, out: torch.Tensor,
                               scores_out: Optional[torch.Tensor] = None, stream=None) -> None:
     _dev(q, torch.bfloat16, "q")

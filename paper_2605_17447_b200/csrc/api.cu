@@ -15,7 +15,9 @@
 
 namespace fastocr {
 static std::atomic<long long> g_launches{0};
+static std::atomic<long long> g_cluster_launches{0};
 void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+void count_cluster_launches(int n) { g_cluster_launches.fetch_add(n, std::memory_order_relaxed); }
 cudaError_t configure_topk();
 }  // namespace fastocr
 
@@ -35,9 +37,15 @@ struct fastocr_ctx {
   float* scores = nullptr;      // [max_batch][max_vis_len] (decode_step scratch)
   unsigned long long* faults = nullptr;
   // persistent attention CTAs per SM brought by one launch: a full cache pass takes every slot,
-  // a pruned pass leaves one free (so that the next layer's launch can start beside it)
+  // a pruned pass half of them (the next layers' launches run beside it; two per SM measured equal
+  // to or faster than three on every workload tried, by up to 28 % at 64 units)
   int dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
-  int sparse_ctas_per_sm = fastocr::kAttnCtasPerSm - 1;
+  int sparse_ctas_per_sm = 2;
+  // A pruned launch whose CTAs get at most this many rows each runs a unit's CTAs as one thread-block
+  // cluster (merge through distributed shared memory: no global partials, no wait for the previous
+  // kernel). Such launches are latency-bound and gain 5-60 %; with more rows per CTA the GPU is full,
+  // clusters are harder to place and hold their slots until the slowest CTA is done: 8-13 % slower.
+  int cluster_max_rows = 6;
   unsigned long long* trace = nullptr;   // set only by debug builds
   unsigned trace_seq = 0;
   char err[512] = {0};
@@ -139,6 +147,7 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
       a.grid_ctas = units * fastocr::kMaxPartsPerUnit;
   }
   a.active_ctas = a.grid_ctas;
+  a.cluster_ctas = 0;
   (void)max_len;
   return a;
 }
@@ -236,8 +245,8 @@ AttnLaunch sparse_args(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
   a.idx = idx;
   a.kcount = k;
   a.k_stride = k_stride;
-  // Leave a slot per SM free for the next layer's launch unless the pass is long enough (per the
-  // caller's bound on kept tokens) for the overlap not to matter: then take every slot.
+  // Leave slots on every SM free for the next layers' launches unless the pass is long enough (per
+  // the caller's bound on kept tokens) for the overlap not to matter: then take every slot.
   {
     const int64_t rows = static_cast<int64_t>(kv->batch) * kv->num_kv_heads * ((max_len + 31) / 32);
     const bool long_pass = max_kept > 0 && rows >= static_cast<int64_t>(64) * ctx->sm_count * fastocr::kAttnCtasPerSm;
@@ -251,6 +260,8 @@ AttnLaunch sparse_args(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
       if (parts > max_rows) parts = max_rows;
       if (parts > fastocr::kMaxPartsPerUnit) parts = fastocr::kMaxPartsPerUnit;
       a.grid_ctas = units * parts;
+      // (parts = what the kernel gives uniform units on this grid)
+      if ((max_rows + parts - 1) / parts <= ctx->cluster_max_rows) a.cluster_ctas = parts;
     }
     a.active_ctas = a.grid_ctas;
   }
@@ -310,8 +321,9 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   // one partial slot per (CTA, unit) pair that can occur: CTAs + units
   if (const char* v = std::getenv("FASTOCR_DENSE_CTAS_PER_SM")) ctx->dense_ctas_per_sm = std::atoi(v);     // tuning knobs,
   if (const char* v = std::getenv("FASTOCR_SPARSE_CTAS_PER_SM")) ctx->sparse_ctas_per_sm = std::atoi(v);   // read once here
+  if (const char* v = std::getenv("FASTOCR_CLUSTER_MAX_ROWS")) ctx->cluster_max_rows = std::atoi(v);
   if (ctx->dense_ctas_per_sm < 1 || ctx->dense_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
-  if (ctx->sparse_ctas_per_sm < 1 || ctx->sparse_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->sparse_ctas_per_sm = fastocr::kAttnCtasPerSm - 1;
+  if (ctx->sparse_ctas_per_sm < 1 || ctx->sparse_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->sparse_ctas_per_sm = 2;
   ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * fastocr::kAttnCtasPerSm +
                    static_cast<int64_t>(lim->max_batch) * lim->num_kv_heads + 64;
   const int64_t nvis = lim->max_vis_len > 0 ? lim->max_vis_len : 1;
@@ -596,5 +608,6 @@ void fastocr_debug_set_trace(fastocr_ctx* ctx, unsigned long long* buf) { ctx->t
 #endif
 
 int64_t fastocr_launch_count(void) { return fastocr::g_launches.load(std::memory_order_relaxed); }
+int64_t fastocr_cluster_launch_count(void) { return fastocr::g_cluster_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"

@@ -7,13 +7,15 @@
 // are divided among persistent CTAs of two warps: equal parts of every unit when the units are of
 // similar length and no more numerous than the CTAs (no CTA then straddles two units), else
 // equal ranges of all rows laid end to end. Four CTAs fit an SM; a full-cache pass brings all four,
-// a pruned pass three, so that the next layer's launch (which starts early through programmatic
-// dependent launch) can run its prologue beside it. Every CTA streams about the same number of
+// a pruned pass two, so that the next layers' launches (which start early through programmatic
+// dependent launch) can run beside it. Every CTA streams about the same number of
 // rows, pays one pipeline prologue per unit piece and exits without waiting for anyone. When a
 // CTA leaves a unit, its warps merge their running (max, sum, output) through a 4 KB shared-memory
 // buffer; a unit held by one CTA is normalised and written at once, a unit shared by several CTAs
 // goes through global partials and is merged by whichever CTA arrives last (one atomic arrival
-// counter per unit, no spinning). How the rows are handed out is worked out by every CTA from the
+// counter per unit, no spinning), or, for short pruned passes launched with one thread-block
+// cluster per unit, is merged by the cluster's first CTA out of the others' shared memory (no
+// global traffic, so no waiting for the previous kernel either). How the rows are handed out is worked out by every CTA from the
 // lengths of all units (one round trip, a scan) or, for the pruned layers of a decode step, which
 // all see the same lengths and kept counts, once per step by attn_plan_kernel: a CTA then reads a
 // 64-byte record with its range, its unit and the unit's geometry.
@@ -50,8 +52,11 @@
 // when a logit exceeds them by more than 2^8, so the rescale branch is rare.
 #include "kernels.h"
 
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
+
+namespace cg = cooperative_groups;
 
 namespace fastocr {
 namespace {
@@ -192,6 +197,13 @@ __device__ __forceinline__ int split_rule(int units, int grid, int total_rows, i
   const int64_t padded = static_cast<int64_t>(longest_unit) * units;
   if (padded <= static_cast<int64_t>(total_rows) + total_rows / 8) return min(grid / units, kMaxPartsPerUnit);
   return (index_list && 5 * units >= grid && longest_unit <= kOwnUnitMaxRows && padded <= 2 * static_cast<int64_t>(total_rows)) ? 1 : 0;
+}
+
+// A unit cut into `parts` pieces whose CTAs were launched as one thread-block cluster of that size
+// (CTA index / parts = unit, so cluster = unit) is merged inside the cluster. The answer is the same
+// in every CTA of a cluster: all derive the split from the same lengths and the same grid.
+__device__ __forceinline__ bool merges_in_cluster(bool split_units, int parts) {
+  return split_units && parts > 1 && static_cast<int>(cg::this_cluster().num_blocks()) == parts;
 }
 
 // What a launch does is fixed at compile time, so that the main loop carries no code it does not
@@ -732,7 +744,55 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       }
       const int64_t head0 = static_cast<int64_t>(u) * G;
       bool finish = true;
-      if (c_lo != c_hi) {                              // the unit is shared with other CTAs
+      if (HAS_IDX && merges_in_cluster(split_units, parts)) {
+        // The unit's CTAs are one thread-block cluster: CTA 0 of the cluster folds the others'
+        // merge buffers into its own through distributed shared memory. Nothing goes through
+        // global memory, so nobody waits for the previous kernel. Every CTA of the cluster passes
+        // the same two barriers, here or (a CTA without rows) after the loop.
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();                                // every CTA's merged state is in its buffer
+        finish = cluster.block_rank() == 0;
+        if (finish) {
+          const int peers = c_hi - c_lo;               // CTAs 1 .. peers of the cluster hold rows
+#pragma unroll 1
+          for (int c0 = 1; c0 <= peers; c0 += kMergeRound) {
+            float pm[kItems][kMergeRound], pl[kItems][kMergeRound];
+            float4 x0[kItems][kMergeRound], x1[kItems][kMergeRound];
+#pragma unroll
+            for (int r = 0; r < kMergeRound; ++r) {    // a short tail re-reads the last peer (ignored below)
+              const float* peer_m = cluster.map_shared_rank(mrg_m, min(c0 + r, peers));
+#pragma unroll
+              for (int it = 0; it < kItems; ++it) {
+                const int e = it * kThreads + tid, h = e >> 4, d8 = (e & 15) * 8;
+                pm[it][r] = peer_m[h];
+                pl[it][r] = peer_m[8 + h];
+                x0[it][r] = x1[it][r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (HAS_V) {
+                  const float4* srcp = reinterpret_cast<const float4*>(peer_m + 16 + h * kMergePitch + d8);
+                  x0[it][r] = srcp[0];
+                  x1[it][r] = srcp[1];
+                }
+              }
+            }
+#pragma unroll
+            for (int it = 0; it < kItems; ++it) {
+#pragma unroll
+              for (int r = 0; r < kMergeRound; ++r) {
+                if (c0 + r > peers || pm[it][r] == -INFINITY) continue;
+                const float Mn = fmaxf(M[it], pm[it][r]);
+                const float so = (M[it] == -INFINITY) ? 0.f : exp2f(M[it] - Mn), sn = exp2f(pm[it][r] - Mn);
+                num[it][0] = num[it][0] * so + x0[it][r].x * sn; num[it][1] = num[it][1] * so + x0[it][r].y * sn;
+                num[it][2] = num[it][2] * so + x0[it][r].z * sn; num[it][3] = num[it][3] * so + x0[it][r].w * sn;
+                num[it][4] = num[it][4] * so + x1[it][r].x * sn; num[it][5] = num[it][5] * so + x1[it][r].y * sn;
+                num[it][6] = num[it][6] * so + x1[it][r].z * sn; num[it][7] = num[it][7] * so + x1[it][r].w * sn;
+                den[it] = den[it] * so + pl[it][r] * sn;
+                M[it] = Mn;
+              }
+            }
+          }
+        }
+        cluster.sync();                                // no CTA leaves while its buffer may still be read
+      } else if (c_lo != c_hi) {                       // the unit is shared with other CTAs
         wait_for_prior_grids();                        // the split workspace may still be in use by the previous kernel
         const int64_t slot = static_cast<int64_t>(blockIdx.x) + u;
 #pragma unroll
@@ -824,6 +884,11 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     }
     seg_begin += seg_rows;
     ++u;
+  }
+  if (HAS_IDX && r0 >= r1 && merges_in_cluster(split_units, parts)) {
+    cg::cluster_group cluster = cg::this_cluster();    // a CTA without rows: the two barriers of the cluster merge
+    cluster.sync();
+    cluster.sync();
   }
   FASTOCR_TRACE_MARK(5);
 #ifdef FASTOCR_TRACE
@@ -1005,11 +1070,39 @@ __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restric
   }
 }
 
+// Cluster sizes (2 .. kMaxPartsPerUnit) the device can schedule for a pruned-pass instance, asked once
+// in configure_t; a size it cannot schedule falls back to the merge through global memory.
+template <int G, bool PAGED>
+bool* cluster_ok_table() {
+  static bool ok[kMaxPartsPerUnit + 1] = {};
+  return ok;
+}
+
 template <int G, int MODE, bool PAGED>
 cudaError_t launch_partial_t(const AttnLaunch& a, cudaStream_t s) {
-  const cudaError_t e = launch_pdl(attn_stream_kernel<G, MODE, PAGED>, dim3(a.grid_ctas), dim3(kThreads),
-                                   Smem<MODE != kModeKeys>::total, s, a);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.grid_ctas);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = Smem<MODE != kModeKeys>::total;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (MODE == kModePruned) {
+    const int c = a.cluster_ctas;
+    if (c >= 2 && c <= kMaxPartsPerUnit && a.grid_ctas % c == 0 && cluster_ok_table<G, PAGED>()[c]) {
+      attr[1].id = cudaLaunchAttributeClusterDimension;
+      attr[1].val.clusterDim.x = c;
+      attr[1].val.clusterDim.y = 1;
+      attr[1].val.clusterDim.z = 1;
+      cfg.numAttrs = 2;
+    }
+  }
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, attn_stream_kernel<G, MODE, PAGED>, a);
   count_launches(1);
+  if (cfg.numAttrs == 2) count_cluster_launches(1);
   return e;
 }
 
@@ -1024,7 +1117,32 @@ cudaError_t configure_t() {
                                        Smem<MODE != kModeKeys>::total);
   if (e != cudaSuccess) return e;
   // all of the SM's L1/shared array as shared memory: four CTAs must fit
-  return cudaFuncSetAttribute(attn_stream_kernel<G, MODE, PAGED>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+  e = cudaFuncSetAttribute(attn_stream_kernel<G, MODE, PAGED>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+  if (e != cudaSuccess) return e;
+  if (MODE == kModePruned) {
+    // clusters of more than 8 CTAs need the kernel's consent; which sizes the device can place is asked, not assumed
+    const bool big = cudaFuncSetAttribute(attn_stream_kernel<G, MODE, PAGED>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+    bool* ok = cluster_ok_table<G, PAGED>();
+    for (int c = 2; c <= kMaxPartsPerUnit; ++c) {
+      ok[c] = false;
+      if (c > 8 && !big) continue;
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(c);
+      cfg.blockDim = dim3(kThreads);
+      cfg.dynamicSmemBytes = Smem<true>::total;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = c;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, attn_stream_kernel<G, MODE, PAGED>, &cfg) == cudaSuccess && n > 0) ok[c] = true;
+    }
+    (void)cudaGetLastError();                          // a refused size is an answer, not an error
+  }
+  return cudaSuccess;
 }
 
 }  // namespace

@@ -86,6 +86,8 @@ struct AttnLaunch {
   int32_t k_stride;
   int32_t grid_ctas;          // CTAs launched (kAttnWarps warps each)
   int32_t active_ctas;        // CTAs that take work (<= grid_ctas); the rest exit at once
+  int32_t cluster_ctas;       // pruned passes: CTAs per unit when the grid is units x this many (launched as clusters
+                              // of that size so that a unit's pieces merge through distributed shared memory); else 0
   int32_t wait_point;         // where the kernel waits for earlier kernels: kWaitAtStart / kWaitAfterSetup / kWaitBeforeWrites
   const int4* plan;           // NULL or one 64-byte record per CTA written by launch_attn_plan for this very launch
                               // shape (grid, lengths, kept counts): the CTA's range and unit, ready made
@@ -130,5 +132,6 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
 cudaError_t configure_kernels();   // one-time cudaFuncSetAttribute calls (current device)
 
 void count_launches(int n);
+void count_cluster_launches(int n);   // of those, pruned passes launched as one thread-block cluster per unit
 
 }  // namespace fastocr

@@ -165,6 +165,48 @@ def test_sparse_matches_oracle(fo, ctx, shape, paged):
     _check_out(out, ref)
 
 
+# Short pruned passes over sequences of similar length run one thread-block cluster per unit and
+# merge a unit's pieces through distributed shared memory: cluster sizes up to 16, a shorter
+# sequence whose units leave CTAs of their cluster without rows, the 8-head group, paged caches.
+CLUSTER_CASES = [
+    dict(spans=[(16, 4000, 48)], k=[200]),                          # 264 tokens: 9 rows, 9 CTAs per unit
+    dict(spans=[(10, 3000, 22), (10, 2500, 22)], k=[224, 192]),     # 8 and 7 rows on clusters of 8: one idle CTA each
+    dict(spans=[(30, 6000, 40)], k=[440], H=64, Hkv=8),             # 510 tokens: 16 rows, clusters of 16
+    dict(spans=[(5, 900, 5), (6, 880, 5), (5, 910, 4), (4, 905, 6)], k=[90, 88, 91, 90]),   # 4 rows: clusters of 4
+]
+
+
+@pytest.mark.parametrize("case_no", range(len(CLUSTER_CASES)))
+@pytest.mark.parametrize("paged", [False, True])
+def test_sparse_cluster_merge_matches_oracle(fo, ctx, case_no, paged):
+    spec = dict(CLUSTER_CASES[case_no])
+    ks = spec.pop("k")
+    case = make_case(350 + case_no, page_size=16 if paged else 0, **spec)
+    kv = case.device_view(poison=True)
+    g = torch.Generator().manual_seed(case_no)
+    idx = torch.zeros(case.B, max(ks), dtype=torch.int32)
+    for b in range(case.B):
+        idx[b, :ks[b]] = torch.randperm(case.vis_len[b], generator=g)[:ks[b]].sort().values.int()
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    max_kept = max(k + s - n for k, s, n in zip(ks, case.seq_len, case.vis_len))
+    ref = torch.stack([oracle.sparse(*case.seq(b), SCALE, case.vis_start[b], case.vis_len[b], idx[b, :ks[b]], True)
+                       for b in range(case.B)])
+    q = case.q.cuda()
+    out = torch.full((case.B, case.H, 128), 7.0, dtype=torch.float32, device="cuda")
+    before = fo.cluster_launch_count()
+    fo.fastocr_sparse_decode_attn(ctx, kv, q, idx.cuda(), kd, out, max_kept=max_kept)
+    assert fo.cluster_launch_count() == before + 1       # the path under test is the one that ran
+    _check_out(out, ref)
+    # the same inside a decode step (launch plan in use), three pruned layers on last step's set
+    out3 = torch.full((3, case.B, case.H, 128), 7.0, dtype=torch.float32, device="cuda")
+    before = fo.cluster_launch_count()
+    assert fo.fastocr_decode_step(ctx, [kv, kv, kv], torch.stack([q, q, q]), out3, [False, False, False], kd,
+                                  idx.cuda().clone(), True, max(case.vis_len), max_kept=max_kept)
+    assert fo.cluster_launch_count() == before + 3
+    for l in range(3):
+        assert torch.equal(out3[l], out)
+
+
 def test_sparse_tau_one_equals_dense_and_tau_zero_is_text_only(fo, ctx):
     case = make_case(401, spans=[(16, 600, 40), (4, 333, 9)])
     kv = case.device_view()
