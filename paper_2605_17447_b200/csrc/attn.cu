@@ -78,11 +78,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
 // Cache rows are read once per layer: they go through L2 marked evict-first, so that streaming a
 // gigabyte of them does not push out what is read again soon (the logits of a focal layer, the
 // index list, the queries).
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
+__device__ __forceinline__ uint64_t l2_evict_first_policy() { return l2_policy_evict_first(); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint64_t policy) {
   asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
 }
@@ -387,6 +383,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 #pragma unroll
   for (int i = 0; i < 4; ++i) cp_off[i] = (2 * i + half) * 256 + ((c16 ^ row_swz(2 * i + half)) << 4);
   const uint64_t stream_policy = l2_evict_first_policy();
+  const uint64_t keep_policy = LOGITS ? l2_policy_evict_last() : 0;   // logits: read back by the next kernel
 #ifdef FASTOCR_TRACE
   if (a.trace != nullptr && lane == 0) {               // slot 2: the SM this CTA runs on
     unsigned smid;
@@ -612,7 +609,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           float* lrow = (i & 1) ? logitB : logitA;
           if (LOGITS && lrow != nullptr && valid) {              // dense / scoring mode: position == list index
             const int rel = tok - sg.vs;
-            if (rel >= 0 && rel < sg.N && rel < a.n_stride) lrow[rel] = x[i];
+            if (rel >= 0 && rel < sg.N && rel < a.n_stride) store_logit(lrow + rel, x[i], keep_policy);
           }
         }
         float mxA = fmaxf(x[0], x[2]), mxB = fmaxf(x[1], x[3]);
@@ -1016,6 +1013,7 @@ __global__ void __launch_bounds__(kFinalizeThreads) scores_finalize_kernel(
   const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + i0;
   const bool full = i0 + 4 <= N && (n_stride_logits & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  const uint64_t once = l2_policy_evict_first();
   for (int h0 = 0; h0 < num_q_heads; h0 += 8) {        // summed in head order
     float4 x[8];
 #pragma unroll
@@ -1024,12 +1022,12 @@ __global__ void __launch_bounds__(kFinalizeThreads) scores_finalize_kernel(
       if (h0 + j < num_q_heads) {
         const float* src = lp + static_cast<int64_t>(h0 + j) * n_stride_logits;
         if (full) {
-          x[j] = __ldcg(reinterpret_cast<const float4*>(src));
+          x[j] = load_logit4(src, once);
         } else {
-          x[j].x = __ldcg(src);
-          if (i0 + 1 < N) x[j].y = __ldcg(src + 1);
-          if (i0 + 2 < N) x[j].z = __ldcg(src + 2);
-          if (i0 + 3 < N) x[j].w = __ldcg(src + 3);
+          x[j].x = load_logit(src, once);
+          if (i0 + 1 < N) x[j].y = load_logit(src + 1, once);
+          if (i0 + 2 < N) x[j].z = load_logit(src + 2, once);
+          if (i0 + 3 < N) x[j].w = load_logit(src + 3, once);
         }
       }
     }

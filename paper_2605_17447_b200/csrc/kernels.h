@@ -58,6 +58,34 @@ __device__ __forceinline__ float score_add_head(float acc, float logit, float ma
   return acc + e * inv_sum;
 }
 __device__ __forceinline__ float score_finish(float acc, int num_q_heads) { return acc / static_cast<float>(num_q_heads); }
+
+// The logits of a focal layer are written with an L2 evict-last policy (they are read back within
+// microseconds, while a gigabyte of cache rows streams past) and read with evict-first, so that
+// they stop occupying L2 once the scores are formed.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void store_logit(float* dst, float x, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(dst), "f"(x), "l"(policy) : "memory");
+}
+__device__ __forceinline__ float load_logit(const float* src, uint64_t policy) {
+  float x;
+  asm volatile("ld.global.cg.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(x) : "l"(src), "l"(policy));
+  return x;
+}
+__device__ __forceinline__ float4 load_logit4(const float* src, uint64_t policy) {
+  float4 v;
+  asm volatile("ld.global.cg.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(src), "l"(policy));
+  return v;
+}
 #endif
 
 // AttnLaunch::wait_point

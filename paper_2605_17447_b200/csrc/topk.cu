@@ -89,6 +89,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
     __syncthreads();
     const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + lo_i;
     bool peers_checked = C == 1;
+    const uint64_t once = l2_policy_evict_first();
     const bool vec = (n_stride_logits & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;   // lo_i is a multiple of 32
     for (int i0 = tid * 4; i0 < n_loc; i0 += kTopkThreads * 4) {
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -101,12 +102,12 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
           if (h0 + j < num_q_heads) {
             const float* src = lp + static_cast<int64_t>(h0 + j) * n_stride_logits + i0;
             if (full) {
-              x[j] = __ldcg(reinterpret_cast<const float4*>(src));
+              x[j] = load_logit4(src, once);
             } else {
-              x[j].x = __ldcg(src);
-              if (i0 + 1 < n_loc) x[j].y = __ldcg(src + 1);
-              if (i0 + 2 < n_loc) x[j].z = __ldcg(src + 2);
-              if (i0 + 3 < n_loc) x[j].w = __ldcg(src + 3);
+              x[j].x = load_logit(src, once);
+              if (i0 + 1 < n_loc) x[j].y = load_logit(src + 1, once);
+              if (i0 + 2 < n_loc) x[j].z = load_logit(src + 2, once);
+              if (i0 + 3 < n_loc) x[j].w = load_logit(src + 3, once);
             }
           }
         }
