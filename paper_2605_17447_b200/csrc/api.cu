@@ -143,11 +143,14 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
     // small batches: the kernel gives every unit at most kMaxPartsPerUnit CTAs; launch no more
     const int units = kv->batch * kv->num_kv_heads;
     const int64_t rows = static_cast<int64_t>(units) * ((max_len + 31) / 32);
-    if (units * fastocr::kMaxPartsPerUnit < a.grid_ctas && rows < static_cast<int64_t>(128) * a.grid_ctas)
+    a.cluster_ctas = 0;
+    if (units * fastocr::kMaxPartsPerUnit < a.grid_ctas && rows < static_cast<int64_t>(128) * a.grid_ctas) {
       a.grid_ctas = units * fastocr::kMaxPartsPerUnit;
+      // the GPU is far from full: one cluster per unit, pieces merged through distributed shared memory
+      if (ctx->cluster_max_rows > 0) a.cluster_ctas = fastocr::kMaxPartsPerUnit;
+    }
   }
   a.active_ctas = a.grid_ctas;
-  a.cluster_ctas = 0;
   (void)max_len;
   return a;
 }

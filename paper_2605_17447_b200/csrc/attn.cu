@@ -741,7 +741,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       }
       const int64_t head0 = static_cast<int64_t>(u) * G;
       bool finish = true;
-      if (HAS_IDX && merges_in_cluster(split_units, parts)) {
+      if (merges_in_cluster(split_units, parts)) {
         // The unit's CTAs are one thread-block cluster: CTA 0 of the cluster folds the others'
         // merge buffers into its own through distributed shared memory. Nothing goes through
         // global memory, so nobody waits for the previous kernel. Every CTA of the cluster passes
@@ -882,7 +882,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     seg_begin += seg_rows;
     ++u;
   }
-  if (HAS_IDX && r0 >= r1 && merges_in_cluster(split_units, parts)) {
+  if (r0 >= r1 && merges_in_cluster(split_units, parts)) {
     cg::cluster_group cluster = cg::this_cluster();    // a CTA without rows: the two barriers of the cluster merge
     cluster.sync();
     cluster.sync();
@@ -1068,9 +1068,9 @@ __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restric
   }
 }
 
-// Cluster sizes (2 .. kMaxPartsPerUnit) the device can schedule for a pruned-pass instance, asked once
+// Cluster sizes (2 .. kMaxPartsPerUnit) the device can schedule for a kernel instance, asked once
 // in configure_t; a size it cannot schedule falls back to the merge through global memory.
-template <int G, bool PAGED>
+template <int G, int MODE, bool PAGED>
 bool* cluster_ok_table() {
   static bool ok[kMaxPartsPerUnit + 1] = {};
   return ok;
@@ -1088,9 +1088,9 @@ cudaError_t launch_partial_t(const AttnLaunch& a, cudaStream_t s) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (MODE == kModePruned) {
+  {
     const int c = a.cluster_ctas;
-    if (c >= 2 && c <= kMaxPartsPerUnit && a.grid_ctas % c == 0 && cluster_ok_table<G, PAGED>()[c]) {
+    if (c >= 2 && c <= kMaxPartsPerUnit && a.grid_ctas % c == 0 && cluster_ok_table<G, MODE, PAGED>()[c]) {
       attr[1].id = cudaLaunchAttributeClusterDimension;
       attr[1].val.clusterDim.x = c;
       attr[1].val.clusterDim.y = 1;
@@ -1117,17 +1117,17 @@ cudaError_t configure_t() {
   // all of the SM's L1/shared array as shared memory: four CTAs must fit
   e = cudaFuncSetAttribute(attn_stream_kernel<G, MODE, PAGED>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
   if (e != cudaSuccess) return e;
-  if (MODE == kModePruned) {
+  {
     // clusters of more than 8 CTAs need the kernel's consent; which sizes the device can place is asked, not assumed
     const bool big = cudaFuncSetAttribute(attn_stream_kernel<G, MODE, PAGED>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
-    bool* ok = cluster_ok_table<G, PAGED>();
+    bool* ok = cluster_ok_table<G, MODE, PAGED>();
     for (int c = 2; c <= kMaxPartsPerUnit; ++c) {
       ok[c] = false;
       if (c > 8 && !big) continue;
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3(c);
       cfg.blockDim = dim3(kThreads);
-      cfg.dynamicSmemBytes = Smem<true>::total;
+      cfg.dynamicSmemBytes = Smem<MODE != kModeKeys>::total;
       cudaLaunchAttribute attr[1];
       attr[0].id = cudaLaunchAttributeClusterDimension;
       attr[0].val.clusterDim.x = c;

@@ -64,7 +64,11 @@ def test_dense_and_fused_scores_match_oracle(fo, ctx, shape, paged):
     out = torch.empty(case.B, case.H, 128, dtype=torch.float32, device="cuda")
     nmax = max(max(case.vis_len), 1)
     sc = torch.full((case.B, nmax + 3), -7.0, dtype=torch.float32, device="cuda")
+    before = fo.cluster_launch_count()
     fo.fastocr_dense_decode_attn(ctx, kv, q, out, scores_out=sc)
+    # these batches are small: each (sequence, KV head) unit is one cluster of 16 CTAs, and the uniform
+    # ones merge inside it (several with units of fewer than 16 rows: CTAs without work in the cluster)
+    assert fo.cluster_launch_count() == before + 1
     _check_out(out, _oracle_dense(case))
     # fp32-accumulating oracle too (the stated reference)
     err32 = (out.cpu() - _oracle_dense(case, acc64=False)).abs()
