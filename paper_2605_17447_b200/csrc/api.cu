@@ -46,6 +46,8 @@ struct fastocr_ctx {
   // kernel). Such launches are latency-bound and gain 5-60 %; with more rows per CTA the GPU is full,
   // clusters are harder to place and hold their slots until the slowest CTA is done: 8-13 % slower.
   int cluster_max_rows = 6;
+  bool l2_persist_set = false;      // FASTOCR_L2_PERSIST_MB changed the context's persisting-L2 limit: put it back
+  size_t l2_persist_before = 0;
   unsigned long long* trace = nullptr;   // set only by debug builds
   unsigned trace_seq = 0;
   char err[512] = {0};
@@ -325,6 +327,18 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   if (const char* v = std::getenv("FASTOCR_DENSE_CTAS_PER_SM")) ctx->dense_ctas_per_sm = std::atoi(v);     // tuning knobs,
   if (const char* v = std::getenv("FASTOCR_SPARSE_CTAS_PER_SM")) ctx->sparse_ctas_per_sm = std::atoi(v);   // read once here
   if (const char* v = std::getenv("FASTOCR_CLUSTER_MAX_ROWS")) ctx->cluster_max_rows = std::atoi(v);
+  if (const char* v = std::getenv("FASTOCR_L2_PERSIST_MB")) {
+    // Experiment, off by default: an L2 set-aside for evict-last lines (the logits of a focal layer).
+    // It is a limit of this process's CUDA context and takes that much L2 away from everything else.
+    int max_persist = 0;
+    cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, device);
+    size_t want = static_cast<size_t>(std::atoi(v) > 0 ? std::atoi(v) : 0) << 20;
+    if (want > static_cast<size_t>(max_persist)) want = static_cast<size_t>(max_persist);
+    if (cudaDeviceGetLimit(&ctx->l2_persist_before, cudaLimitPersistingL2CacheSize) == cudaSuccess &&
+        cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) == cudaSuccess)
+      ctx->l2_persist_set = true;
+    (void)cudaGetLastError();
+  }
   if (ctx->dense_ctas_per_sm < 1 || ctx->dense_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
   if (ctx->sparse_ctas_per_sm < 1 || ctx->sparse_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->sparse_ctas_per_sm = 2;
   ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * fastocr::kAttnCtasPerSm +
@@ -361,6 +375,7 @@ void fastocr_destroy(fastocr_ctx* ctx) {
   cudaFree(ctx->scores);
   cudaFree(ctx->counters);
   cudaFree(ctx->faults);
+  if (ctx->l2_persist_set) cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, ctx->l2_persist_before);
   delete ctx;
 }
 
