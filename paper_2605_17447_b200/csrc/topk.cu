@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
                                                                    int32_t* __restrict__ idx_out, int k_stride, int n_cap,
                                                                    const float* __restrict__ logits,
                                                                    const float* __restrict__ stats, int num_q_heads,
-                                                                   int n_stride_logits) {
+                                                                   int n_stride_logits, int drop_logits) {
   extern __shared__ __align__(16) uint32_t keys[];      // all keys of the sequence
   __shared__ float head_st[2 * kTopkMaxHeads];          // scoring mode: per head (max, 1 / sum)
   __shared__ uint32_t hist[kTopkBins];
@@ -168,6 +168,18 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
       }
       if (!peers_checked) cluster.barrier_wait();       // (a thread without tokens to score)
       if (C > 1) cluster.sync();                        // every slice has arrived in every copy
+    }
+    __syncthreads();                                    // every load of this CTA's slice has returned
+    if (drop_logits) {
+      // The logits are dead now: their lines are dropped from L2 instead of being written back to
+      // HBM later, in the middle of the pruned layers' streams (59 MB per focal layer at B = 64,
+      // N = 8192). The launch sets the flag only when rows start on 128-byte boundaries; slices
+      // are multiples of 32 tokens, so every line here belongs to this CTA alone.
+      const int lines = (n_loc + 31) >> 5;
+      for (int e = tid; e < num_q_heads * lines; e += kTopkThreads) {
+        const int h = e / lines, l = e - h * lines;
+        asm volatile("discard.global.L2 [%0], 128;" ::"l"(lp + static_cast<int64_t>(h) * n_stride_logits + 32 * l) : "memory");
+      }
     }
   }
   __syncthreads();
@@ -365,6 +377,8 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
     if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
     while (C < kTopkMaxCluster && batch * C * 2 <= sms && max_vis_len / (C * 2) >= 1024) C *= 2;
   }
+  // whole 128-byte lines per (head, 32 tokens): the kernel may drop them from L2 once read
+  const int drop = logits != nullptr && (reinterpret_cast<uintptr_t>(logits) & 127) == 0 && (n_stride_logits & 31) == 0 ? 1 : 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(batch * C);
   cfg.blockDim = dim3(kTopkThreads);
@@ -381,7 +395,7 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
   cfg.numAttrs = 2;
   const cudaError_t e = cudaLaunchKernelEx(&cfg, select_topk_kernel, scores, n_stride, vis_len, k, idx_out, k_stride,
                                            static_cast<int>(max_vis_len), logits, stats, static_cast<int>(num_q_heads),
-                                           static_cast<int>(n_stride_logits));
+                                           static_cast<int>(n_stride_logits), drop);
   count_launches(1);
   return e;
 }
