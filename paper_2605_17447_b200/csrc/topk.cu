@@ -377,8 +377,11 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
     if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
     while (C < kTopkMaxCluster && batch * C * 2 <= sms && max_vis_len / (C * 2) >= 1024) C *= 2;
   }
-  // whole 128-byte lines per (head, 32 tokens): the kernel may drop them from L2 once read
-  const int drop = logits != nullptr && (reinterpret_cast<uintptr_t>(logits) & 127) == 0 && (n_stride_logits & 31) == 0 ? 1 : 0;
+  // Whole 128-byte lines per (head, 32 tokens): the kernel may drop them from L2 once read. Worth its
+  // 2-3 us only when the logits are a load on L2 (tens of MB); small ones are simply overwritten in
+  // place by the next focal layer.
+  const bool big = static_cast<int64_t>(batch) * num_q_heads * max_vis_len * 4 >= (static_cast<int64_t>(8) << 20);
+  const int drop = logits != nullptr && big && (reinterpret_cast<uintptr_t>(logits) & 127) == 0 && (n_stride_logits & 31) == 0 ? 1 : 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(batch * C);
   cfg.blockDim = dim3(kTopkThreads);
