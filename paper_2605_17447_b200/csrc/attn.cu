@@ -13,9 +13,9 @@
 // CTA leaves a unit, its warps merge their running (max, sum, output) through a 4 KB shared-memory
 // buffer; a unit held by one CTA is normalised and written at once, a unit shared by several CTAs
 // goes through global partials and is merged by whichever CTA arrives last (one atomic arrival
-// counter per unit, no spinning), or, for short pruned passes launched with one thread-block
-// cluster per unit, is merged by the cluster's first CTA out of the others' shared memory (no
-// global traffic, so no waiting for the previous kernel either). How the rows are handed out is worked out by every CTA from the
+// counter per unit, no spinning), or, for passes launched with one thread-block cluster per unit
+// (short pruned passes, full-cache passes of small batches), is merged by the cluster's first CTA
+// out of the others' shared memory (no global traffic, so no waiting for the previous kernel either). How the rows are handed out is worked out by every CTA from the
 // lengths of all units (one round trip, a scan) or, for the pruned layers of a decode step, which
 // all see the same lengths and kept counts, once per step by attn_plan_kernel: a CTA then reads a
 // 64-byte record with its range, its unit and the unit's geometry.

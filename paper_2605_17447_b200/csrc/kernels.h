@@ -114,8 +114,8 @@ struct AttnLaunch {
   int32_t k_stride;
   int32_t grid_ctas;          // CTAs launched (kAttnWarps warps each)
   int32_t active_ctas;        // CTAs that take work (<= grid_ctas); the rest exit at once
-  int32_t cluster_ctas;       // pruned passes: CTAs per unit when the grid is units x this many (launched as clusters
-                              // of that size so that a unit's pieces merge through distributed shared memory); else 0
+  int32_t cluster_ctas;       // CTAs per unit when the grid is units x this many and the launch should run one cluster
+                              // of that size per unit (a unit's pieces then merge through distributed shared memory); else 0
   int32_t wait_point;         // where the kernel waits for earlier kernels: kWaitAtStart / kWaitAfterSetup / kWaitBeforeWrites
   const int4* plan;           // NULL or one 64-byte record per CTA written by launch_attn_plan for this very launch
                               // shape (grid, lengths, kept counts): the CTA's range and unit, ready made
