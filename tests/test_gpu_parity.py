@@ -211,6 +211,39 @@ def test_sparse_cluster_merge_matches_oracle(fo, ctx, case_no, paged):
         assert torch.equal(out3[l], out)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_sparse_random_batches_match_oracle(fo, ctx, seed):
+    """Seeded random batches (1-8 sequences, similar or very different lengths, any kept fraction, paged
+    or not, with and without the caller's bound on kept tokens): whichever way the kernel hands out
+    the rows (equal parts, one CTA per unit, equal ranges; merged in clusters or through global
+    memory), the result is the oracle's."""
+    g = torch.Generator().manual_seed(1000 + seed)
+    ri = lambda lo, hi: int(torch.randint(lo, hi + 1, (1,), generator=g))
+    B = ri(1, 8)
+    similar = seed % 2 == 0
+    n0 = ri(64, 3000)
+    spans = []
+    for _ in range(B):
+        n = max(1, n0 + ri(-n0 // 20, n0 // 20)) if similar else ri(1, 3000)
+        spans.append((ri(0, 40), n, ri(0, 120)))
+    tau = [0.02, 0.05, 0.1, 0.3, 0.6, 1.0][seed % 6]
+    heads = dict(H=64, Hkv=8) if seed % 4 == 3 else {}
+    case = make_case(1100 + seed, spans=spans, page_size=16 if seed % 3 == 0 else 0, **heads)
+    kv = case.device_view(poison=True)
+    ks = [oracle.kept_count(n, tau) for n in case.vis_len]
+    idx = torch.zeros(case.B, max(max(ks), 1), dtype=torch.int32)
+    for b in range(case.B):
+        idx[b, :ks[b]] = torch.randperm(case.vis_len[b], generator=g)[:ks[b]].sort().values.int()
+    attended = [k + s - n for k, s, n in zip(ks, case.seq_len, case.vis_len)]
+    ref = torch.stack([oracle.sparse(*case.seq(b), SCALE, case.vis_start[b], case.vis_len[b], idx[b, :ks[b]], True)
+                       if attended[b] > 0 else torch.zeros(case.H, 128) for b in range(case.B)])
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    for max_kept in (max(attended), 0):
+        out = torch.full((case.B, case.H, 128), 7.0, dtype=torch.float32, device="cuda")
+        fo.fastocr_sparse_decode_attn(ctx, kv, case.q.cuda(), idx.cuda(), kd, out, max_kept=max_kept)
+        _check_out(out, ref)
+
+
 def test_sparse_tau_one_equals_dense_and_tau_zero_is_text_only(fo, ctx):
     case = make_case(401, spans=[(16, 600, 40), (4, 333, 9)])
     kv = case.device_view()
