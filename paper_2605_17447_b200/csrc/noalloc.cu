@@ -94,7 +94,14 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   fastocr_status st = setup_current_device(device);
   if (st != FASTOCR_OK) return st;
   const DeviceSetup& s = g_setup[device];
-  const int grid = 3 * s.sm_count;
+  // two persistent CTAs per SM (the next launch runs beside them), no idle ones: when every unit
+  // gets the same number of CTAs, a grid that is a multiple of the unit count has none left over
+  int grid = 2 * s.sm_count;
+  if (units <= grid) {
+    int parts = grid / static_cast<int>(units);
+    if (parts > fastocr::kMaxPartsPerUnit) parts = fastocr::kMaxPartsPerUnit;
+    grid = static_cast<int>(units) * parts;
+  }
   if (units + grid > kNoallocMaxSlots) return fail(FASTOCR_ERR_WORKSPACE, "this GPU has more SMs than the built-in scratch was sized for");
 
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
