@@ -19,6 +19,8 @@
 
 #include <cooperative_groups.h>
 
+#include <mutex>
+
 namespace cg = cooperative_groups;
 
 namespace fastocr {
@@ -356,6 +358,36 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
 
 }  // namespace
 
+// Clusters of C CTAs with `smem` bytes of dynamic shared memory the device can hold at once; the
+// answers are remembered (a handful of distinct shapes per process).
+static int max_active_clusters(int C, size_t smem) {
+  struct Memo { int c; size_t smem; int n; };
+  static Memo memo[16];
+  static int used = 0;
+  static std::mutex lock;
+  std::lock_guard<std::mutex> hold(lock);
+  for (int i = 0; i < used; ++i)
+    if (memo[i].c == C && memo[i].smem == smem) return memo[i].n;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(C);
+  cfg.blockDim = dim3(kTopkThreads);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, select_topk_kernel, &cfg) != cudaSuccess) {
+    (void)cudaGetLastError();
+    n = 0;
+  }
+  if (used < 16) memo[used++] = Memo{C, smem, n};
+  return n;
+}
+
 cudaError_t configure_topk() {
   cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkMaxN * 4 + 16);
   if (e != cudaSuccess) return e;
@@ -376,6 +408,10 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
     int device = 0, sms = 148;
     if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
     while (C < kTopkMaxCluster && batch * C * 2 <= sms && max_vis_len / (C * 2) >= 1024) C *= 2;
+    // all clusters must be resident at once (a second wave doubles the kernel's time): the device says
+    // how many clusters of this size and shared-memory footprint it can hold (15 of 8 CTAs on a B200)
+    const size_t smem = (static_cast<size_t>(max_vis_len) + 31) / 32 * 32 * 4 + 16;
+    while (C > 1 && max_active_clusters(C, smem) < batch) C /= 2;
   }
   // Whole 128-byte lines per (head, 32 tokens): the kernel may drop them from L2 once read. Worth its
   // 2-3 us only when the logits are a load on L2 (tens of MB); small ones are simply overwritten in
