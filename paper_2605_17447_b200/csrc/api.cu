@@ -148,8 +148,10 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
     a.cluster_ctas = 0;
     if (units * fastocr::kMaxPartsPerUnit < a.grid_ctas && rows < static_cast<int64_t>(128) * a.grid_ctas) {
       a.grid_ctas = units * fastocr::kMaxPartsPerUnit;
-      // the GPU is far from full: one cluster per unit, pieces merged through distributed shared memory
-      if (ctx->cluster_max_rows > 0) a.cluster_ctas = fastocr::kMaxPartsPerUnit;
+      // A launch that leaves most SMs empty anyway (a single sequence): one cluster per unit, pieces
+      // merged through distributed shared memory. From two sequences on, placing clusters of 16 costs a
+      // full-cache pass more than the merge saves (batch 8: 57.6 against 37.3 us).
+      if (ctx->cluster_max_rows > 0 && 2 * a.grid_ctas <= ctx->sm_count) a.cluster_ctas = fastocr::kMaxPartsPerUnit;
     }
   }
   a.active_ctas = a.grid_ctas;

@@ -66,9 +66,10 @@ def test_dense_and_fused_scores_match_oracle(fo, ctx, shape, paged):
     sc = torch.full((case.B, nmax + 3), -7.0, dtype=torch.float32, device="cuda")
     before = fo.cluster_launch_count()
     fo.fastocr_dense_decode_attn(ctx, kv, q, out, scores_out=sc)
-    # these batches are small: each (sequence, KV head) unit is one cluster of 16 CTAs, and the uniform
-    # ones merge inside it (several with units of fewer than 16 rows: CTAs without work in the cluster)
-    assert fo.cluster_launch_count() == before + 1
+    # a single sequence leaves most SMs empty anyway: each (sequence, KV head) unit is then one cluster of
+    # 16 CTAs and merges inside it (some units have fewer than 16 rows: CTAs without work in the cluster)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert fo.cluster_launch_count() == before + (1 if 2 * 16 * case.B * case.Hkv <= sms else 0)
     _check_out(out, _oracle_dense(case))
     # fp32-accumulating oracle too (the stated reference)
     err32 = (out.cpu() - _oracle_dense(case, acc64=False)).abs()
