@@ -389,10 +389,12 @@ def test_decode_step_matches_algorithm_trace(fo, ctx, paged, spans):
                 f_last[b] = tr.f_last
 
 
-@pytest.mark.parametrize("batch,n", [(2, 16384), (5, 4100), (1, 2048)])
+@pytest.mark.parametrize("batch,n", [(2, 16384), (5, 4100), (1, 2048), (1, 32768), (3, 32768), (20, 16384)])
 def test_decode_step_selection_equals_separate_calls(fo, batch, n):
     """The decode step's selection kernel forms the scores itself, with a cluster of up to 8 CTAs per
-    sequence for small batches; it must select exactly what scoring + selection as separate calls do."""
+    sequence for small batches; it must select exactly what scoring + selection as separate calls do.
+    (The last three shapes take the variant that splits the selection itself over the cluster:
+    32768 keys on clusters of 8, 16384 keys on clusters of 4.)"""
     from workloads import make_kv, normal_bf16, stream_key
     dev = "cuda"
     H, Hkv, T = 28, 4, 40
