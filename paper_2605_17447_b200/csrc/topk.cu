@@ -42,6 +42,103 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Scores of tokens [lo_i, lo_i + n_loc) of sequence b from a focal layer's logits and per-head
+// (max, sum) (Section 3.1.1; the same arithmetic as the stand-alone scoring kernel, head by head in
+// ascending order), turned into keys and handed to put1(j, key) / put4(j0, keys[4], count) with j
+// relative to lo_i; ready() is called once by every thread, all together, before the first put (the
+// place for a barrier that the puts depend on). The logits were written by the kernel just before
+// and are read from L2; with `drop_logits` their lines are dropped from L2 afterwards. Every thread
+// of the CTA must call this (barriers inside); per_cta is the slice length of the launch (the same
+// for every thread).
+template <typename Ready, typename Put1, typename Put4>
+__device__ __forceinline__ void score_slice(const float* __restrict__ logits, const float* __restrict__ stats, float* head_st,
+                                            int b, int num_q_heads, int n_stride_logits, int lo_i, int n_loc, int per_cta,
+                                            int drop_logits, Ready ready, Put1 put1, Put4 put4) {
+  const int tid = threadIdx.x;
+  const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + lo_i;
+  const uint64_t once = l2_policy_evict_first();
+  auto fetch_stats = [&]() {
+    for (int i = tid; i < num_q_heads; i += kTopkThreads) {
+      head_st[2 * i] = stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2];
+      head_st[2 * i + 1] = 1.0f / stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2 + 1];
+    }
+    __syncthreads();
+  };
+  if (per_cta <= kTopkThreads) {
+    // Few tokens per CTA (small batches, where the kernel is a chain of latencies): one token per
+    // thread, up to 32 heads' logits in flight at once, issued before the statistics are fetched.
+    const bool live = tid < n_loc;
+    float acc = 0.f;
+    for (int h0 = 0; h0 < num_q_heads; h0 += 32) {
+      float x[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        x[j] = (live && h0 + j < num_q_heads) ? load_logit(lp + static_cast<int64_t>(h0 + j) * n_stride_logits + tid, once) : 0.f;
+      if (h0 == 0) {
+        fetch_stats();
+        ready();
+      }
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (h0 + j < num_q_heads) acc = score_add_head(acc, x[j], head_st[2 * (h0 + j)], head_st[2 * (h0 + j) + 1]);
+    }
+    if (live) put1(tid, score_key(score_finish(acc, num_q_heads)));
+  } else {
+    // four tokens per thread, eight heads' loads in flight
+    fetch_stats();
+    ready();
+    const bool vec = (n_stride_logits & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;   // lo_i is a multiple of 32
+    for (int i0 = tid * 4; i0 < n_loc; i0 += kTopkThreads * 4) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      const bool full = vec && i0 + 4 <= n_loc;
+      for (int h0 = 0; h0 < num_q_heads; h0 += 8) {
+        float4 x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          x[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (h0 + j < num_q_heads) {
+            const float* src = lp + static_cast<int64_t>(h0 + j) * n_stride_logits + i0;
+            if (full) {
+              x[j] = load_logit4(src, once);
+            } else {
+              x[j].x = load_logit(src, once);
+              if (i0 + 1 < n_loc) x[j].y = load_logit(src + 1, once);
+              if (i0 + 2 < n_loc) x[j].z = load_logit(src + 2, once);
+              if (i0 + 3 < n_loc) x[j].w = load_logit(src + 3, once);
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (h0 + j < num_q_heads) {
+            const float m = head_st[2 * (h0 + j)], inv = head_st[2 * (h0 + j) + 1];
+            acc[0] = score_add_head(acc[0], x[j].x, m, inv);
+            acc[1] = score_add_head(acc[1], x[j].y, m, inv);
+            acc[2] = score_add_head(acc[2], x[j].z, m, inv);
+            acc[3] = score_add_head(acc[3], x[j].w, m, inv);
+          }
+        }
+      }
+      uint32_t kq[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) kq[j] = score_key(score_finish(acc[j], num_q_heads));
+      put4(i0, kq, min(4, n_loc - i0));
+    }
+  }
+  __syncthreads();                                      // every load of this CTA's slice has returned
+  if (drop_logits) {
+    // The logits are dead now: their lines are dropped from L2 instead of being written back to
+    // HBM later, in the middle of the pruned layers' streams (59 MB per focal layer at B = 64,
+    // N = 8192). The launch sets the flag only when rows start on 128-byte boundaries; slices
+    // are multiples of 32 tokens, so every line here belongs to this CTA alone.
+    const int lines = (n_loc + 31) >> 5;
+    for (int e = tid; e < num_q_heads * lines; e += kTopkThreads) {
+      const int h = e / lines, l = e - h * lines;
+      asm volatile("discard.global.L2 [%0], 128;" ::"l"(lp + static_cast<int64_t>(h) * n_stride_logits + 32 * l) : "memory");
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* __restrict__ scores, int n_stride,
                                                                    const int32_t* __restrict__ vis_len,
                                                                    const int32_t* __restrict__ kreq,
@@ -83,108 +180,26 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
     const float* sp = scores + static_cast<int64_t>(b) * n_stride;
     for (int i = tid; i < N; i += kTopkThreads) keys[i] = score_key(sp[i]);
   } else {
-    // Scores of the CTA's slice (the same arithmetic as the stand-alone scoring kernel, head by
-    // head in ascending order). The logits were written by the kernel just before and are read
-    // from L2.
-    const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + lo_i;
-    const uint64_t once = l2_policy_evict_first();
-    auto fetch_stats = [&]() {
-      for (int i = tid; i < num_q_heads; i += kTopkThreads) {
-        head_st[2 * i] = stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2];
-        head_st[2 * i + 1] = 1.0f / stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2 + 1];
-      }
-      __syncthreads();
+    // The CTA scores its slice and writes the keys into every CTA's copy of the key array
+    // (distributed shared memory). Before the first remote store all threads, together, make sure
+    // that the peers are running (the second half of the barrier begun above).
+    auto all_copies = [&](int j, uint32_t key) {
+      for (int r = 0; r < C; ++r) cluster.map_shared_rank(keys, r)[lo_i + j] = key;
     };
-    if (per_cta <= kTopkThreads) {
-      // Few tokens per CTA (small batches, where the kernel is a chain of latencies): one token per
-      // thread, up to 32 heads' logits in flight at once, issued before the statistics are fetched.
-      const bool live = tid < n_loc;
-      float acc = 0.f;
-      for (int h0 = 0; h0 < num_q_heads; h0 += 32) {
-        float x[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          x[j] = (live && h0 + j < num_q_heads) ? load_logit(lp + static_cast<int64_t>(h0 + j) * n_stride_logits + tid, once) : 0.f;
-        if (h0 == 0) fetch_stats();
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (h0 + j < num_q_heads) acc = score_add_head(acc, x[j], head_st[2 * (h0 + j)], head_st[2 * (h0 + j) + 1]);
-      }
-      const uint32_t key = score_key(score_finish(acc, num_q_heads));
-      if (C > 1) cluster.barrier_wait();                // the peers are running: their copies may be written
-      if (live)
-        for (int r = 0; r < C; ++r) cluster.map_shared_rank(keys, r)[lo_i + tid] = key;
-      if (C > 1) cluster.sync();                        // every slice has arrived in every copy
-    } else {
-      // four tokens per thread, eight heads' loads in flight
-      fetch_stats();
-      bool peers_checked = C == 1;
-      const bool vec = (n_stride_logits & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;   // lo_i is a multiple of 32
-      for (int i0 = tid * 4; i0 < n_loc; i0 += kTopkThreads * 4) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        const bool full = vec && i0 + 4 <= n_loc;
-        for (int h0 = 0; h0 < num_q_heads; h0 += 8) {
-          float4 x[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            x[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (h0 + j < num_q_heads) {
-              const float* src = lp + static_cast<int64_t>(h0 + j) * n_stride_logits + i0;
-              if (full) {
-                x[j] = load_logit4(src, once);
-              } else {
-                x[j].x = load_logit(src, once);
-                if (i0 + 1 < n_loc) x[j].y = load_logit(src + 1, once);
-                if (i0 + 2 < n_loc) x[j].z = load_logit(src + 2, once);
-                if (i0 + 3 < n_loc) x[j].w = load_logit(src + 3, once);
-              }
-            }
-          }
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            if (h0 + j < num_q_heads) {
-              const float m = head_st[2 * (h0 + j)], inv = head_st[2 * (h0 + j) + 1];
-              acc[0] = score_add_head(acc[0], x[j].x, m, inv);
-              acc[1] = score_add_head(acc[1], x[j].y, m, inv);
-              acc[2] = score_add_head(acc[2], x[j].z, m, inv);
-              acc[3] = score_add_head(acc[3], x[j].w, m, inv);
-            }
-          }
-        }
-        uint32_t kq[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) kq[j] = score_key(score_finish(acc[j], num_q_heads));
-        // into every CTA's copy of the key array
-        if (!peers_checked) {
-          cluster.barrier_wait();
-          peers_checked = true;
-        }
-        for (int r = 0; r < C; ++r) {
-          uint32_t* dst = cluster.map_shared_rank(keys, r) + lo_i + i0;
-          if (i0 + 4 <= n_loc) {
-            *reinterpret_cast<uint4*>(dst) = make_uint4(kq[0], kq[1], kq[2], kq[3]);
-          } else {
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (i0 + j < n_loc) dst[j] = kq[j];
-          }
-        }
-      }
-      if (!peers_checked) cluster.barrier_wait();       // (a thread without tokens to score)
-      if (C > 1) cluster.sync();                        // every slice has arrived in every copy
-    }
-    __syncthreads();                                    // every load of this CTA's slice has returned
-    if (drop_logits) {
-      // The logits are dead now: their lines are dropped from L2 instead of being written back to
-      // HBM later, in the middle of the pruned layers' streams (59 MB per focal layer at B = 64,
-      // N = 8192). The launch sets the flag only when rows start on 128-byte boundaries; slices
-      // are multiples of 32 tokens, so every line here belongs to this CTA alone.
-      const int lines = (n_loc + 31) >> 5;
-      for (int e = tid; e < num_q_heads * lines; e += kTopkThreads) {
-        const int h = e / lines, l = e - h * lines;
-        asm volatile("discard.global.L2 [%0], 128;" ::"l"(lp + static_cast<int64_t>(h) * n_stride_logits + 32 * l) : "memory");
-      }
-    }
+    score_slice(logits, stats, head_st, b, num_q_heads, n_stride_logits, lo_i, n_loc, per_cta, drop_logits,
+                [&]() {
+                  if (C > 1) cluster.barrier_wait();
+                },
+                all_copies,
+                [&](int j0, const uint32_t* kq, int count) {
+                  if (count == 4) {
+                    for (int r = 0; r < C; ++r)
+                      *reinterpret_cast<uint4*>(cluster.map_shared_rank(keys, r) + lo_i + j0) = make_uint4(kq[0], kq[1], kq[2], kq[3]);
+                  } else {
+                    for (int t = 0; t < count; ++t) all_copies(j0 + t, kq[t]);
+                  }
+                });
+    if (C > 1) cluster.sync();                          // every slice has arrived in every copy
   }
   __syncthreads();
 
@@ -404,93 +419,16 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_split_kernel(const f
     const float* sp = scores + static_cast<int64_t>(b) * n_stride + lo_i;
     for (int i = tid; i < n_loc; i += kTopkThreads) keys[i] = score_key(sp[i]);
   } else {
-    // Scores of the CTA's slice (the same arithmetic as the stand-alone scoring kernel, head by
-    // head in ascending order). The logits were written by the kernel just before and are read
-    // from L2.
-    const float* lp = logits + static_cast<int64_t>(b) * num_q_heads * n_stride_logits + lo_i;
-    const uint64_t once = l2_policy_evict_first();
-    auto fetch_stats = [&]() {
-      for (int i = tid; i < num_q_heads; i += kTopkThreads) {
-        head_st[2 * i] = stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2];
-        head_st[2 * i + 1] = 1.0f / stats[(static_cast<int64_t>(b) * num_q_heads + i) * 2 + 1];
-      }
-      __syncthreads();
-    };
-    if (per_cta <= kTopkThreads) {
-      // Few tokens per CTA (small batches, where the kernel is a chain of latencies): one token per
-      // thread, up to 32 heads' logits in flight at once, issued before the statistics are fetched.
-      const bool live = tid < n_loc;
-      float acc = 0.f;
-      for (int h0 = 0; h0 < num_q_heads; h0 += 32) {
-        float x[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          x[j] = (live && h0 + j < num_q_heads) ? load_logit(lp + static_cast<int64_t>(h0 + j) * n_stride_logits + tid, once) : 0.f;
-        if (h0 == 0) fetch_stats();
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (h0 + j < num_q_heads) acc = score_add_head(acc, x[j], head_st[2 * (h0 + j)], head_st[2 * (h0 + j) + 1]);
-      }
-      if (live) keys[tid] = score_key(score_finish(acc, num_q_heads));
-    } else {
-      // four tokens per thread, eight heads' loads in flight
-      fetch_stats();
-      const bool vec = (n_stride_logits & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;   // lo_i is a multiple of 32
-      for (int i0 = tid * 4; i0 < n_loc; i0 += kTopkThreads * 4) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        const bool full = vec && i0 + 4 <= n_loc;
-        for (int h0 = 0; h0 < num_q_heads; h0 += 8) {
-          float4 x[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            x[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (h0 + j < num_q_heads) {
-              const float* src = lp + static_cast<int64_t>(h0 + j) * n_stride_logits + i0;
-              if (full) {
-                x[j] = load_logit4(src, once);
-              } else {
-                x[j].x = load_logit(src, once);
-                if (i0 + 1 < n_loc) x[j].y = load_logit(src + 1, once);
-                if (i0 + 2 < n_loc) x[j].z = load_logit(src + 2, once);
-                if (i0 + 3 < n_loc) x[j].w = load_logit(src + 3, once);
-              }
-            }
-          }
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            if (h0 + j < num_q_heads) {
-              const float m = head_st[2 * (h0 + j)], inv = head_st[2 * (h0 + j) + 1];
-              acc[0] = score_add_head(acc[0], x[j].x, m, inv);
-              acc[1] = score_add_head(acc[1], x[j].y, m, inv);
-              acc[2] = score_add_head(acc[2], x[j].z, m, inv);
-              acc[3] = score_add_head(acc[3], x[j].w, m, inv);
-            }
-          }
-        }
-        uint32_t kq[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) kq[j] = score_key(score_finish(acc[j], num_q_heads));
-        if (i0 + 4 <= n_loc) {
-          *reinterpret_cast<uint4*>(keys + i0) = make_uint4(kq[0], kq[1], kq[2], kq[3]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            if (i0 + j < n_loc) keys[i0 + j] = kq[j];
-        }
-      }
-    }
-    __syncthreads();                                    // every load of this CTA's slice has returned
-    if (drop_logits) {
-      // The logits are dead now: their lines are dropped from L2 instead of being written back to
-      // HBM later, in the middle of the pruned layers' streams (59 MB per focal layer at B = 64,
-      // N = 8192). The launch sets the flag only when rows start on 128-byte boundaries; slices
-      // are multiples of 32 tokens, so every line here belongs to this CTA alone.
-      const int lines = (n_loc + 31) >> 5;
-      for (int e = tid; e < num_q_heads * lines; e += kTopkThreads) {
-        const int h = e / lines, l = e - h * lines;
-        asm volatile("discard.global.L2 [%0], 128;" ::"l"(lp + static_cast<int64_t>(h) * n_stride_logits + 32 * l) : "memory");
-      }
-    }
+    score_slice(logits, stats, head_st, b, num_q_heads, n_stride_logits, lo_i, n_loc, per_cta, drop_logits,
+                []() {},
+                [&](int j, uint32_t key) { keys[j] = key; },
+                [&](int j0, const uint32_t* kq, int count) {
+                  if (count == 4) {
+                    *reinterpret_cast<uint4*>(keys + j0) = make_uint4(kq[0], kq[1], kq[2], kq[3]);
+                  } else {
+                    for (int t = 0; t < count; ++t) keys[j0 + t] = kq[t];
+                  }
+                });
   }
   __syncthreads();
 
