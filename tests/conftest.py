@@ -19,6 +19,12 @@ def pytest_collection_modifyitems(config, items):
     except Exception:  # pragma: no cover
         has_gpu = False
     if has_gpu:
+        # a GPU test that does not end is a bug to be reported, not waited for (pytest-timeout, if installed,
+        # ends the process; every test here finishes in seconds)
+        if config.pluginmanager.hasplugin("timeout"):
+            for item in items:
+                if "gpu" in item.keywords and item.get_closest_marker("timeout") is None:
+                    item.add_marker(pytest.mark.timeout(300))
         return
     skip = pytest.mark.skip(reason="no CUDA device")
     for item in items:
