@@ -27,9 +27,16 @@
  *   - Return value: FASTOCR_OK or an error code; on error nothing was launched
  *     and fastocr_last_error(ctx) describes the problem. Argument checks are
  *     host-side only; the contents of device arrays (lengths, indices, page
- *     ids) cannot be validated without a synchronisation: indices outside
- *     [0, vis_len) are clamped on the device and counted in a status word
- *     readable with fastocr_device_faults.
+ *     ids) cannot be validated without a synchronisation. The kernels force
+ *     them into what the host did check, so that nothing outside the caller's
+ *     buffers is addressed: seq_len[b] into [0, max_seq_len], the image span
+ *     into the sequence, index-list entries into [0, vis_len), block-table
+ *     entries into [0, num_pages) when num_pages is given. Every value that
+ *     had to be changed is counted in a status word readable with
+ *     fastocr_device_faults (the affected sequence's result is then
+ *     meaningless; all other sequences are unaffected). Kept counts above
+ *     vis_len[b] or above the index list's row length k_stride are clamped
+ *     silently (documented behaviour, not a fault).
  *   - head_dim must be 128 and num_q_heads / num_kv_heads (the GQA group size)
  *     one of 1, 2, 4, 7, 8; query head h reads KV head h / group size.
  */
@@ -79,6 +86,9 @@ typedef struct fastocr_kv_view {
   int64_t seq_stride_tokens;  /* contiguous only: tokens between consecutive sequences           */
   const int32_t* block_table; /* paged only: device [B][max_pages], physical page of each logical page */
   int32_t max_pages;          /* paged only: row length of block_table                           */
+  int32_t num_pages;          /* paged only: pages in the k / v pools; block-table entries outside
+                                 [0, num_pages) are clamped on the device and counted as faults.
+                                 0 = not given: entries are used as they are                        */
   const int32_t* seq_len;     /* device [B]: S_b, number of cached tokens                        */
   const int32_t* vis_start;   /* device [B]: first image position                                */
   const int32_t* vis_len;     /* device [B]: N_b, number of image tokens                         */
@@ -191,7 +201,8 @@ double fastocr_attn_flops(double batch, double layers, double hidden, double seq
  * on every GPU that loads it, held until the process exits) instead of a context's workspace.
  *   - Limit: batch * num_kv_heads <= FASTOCR_NOALLOC_MAX_UNITS, else FASTOCR_ERR_WORKSPACE.
  *   - The first call on each device resolves the array's device address and sets kernel
- *     attributes (no allocation); make that first call outside any stream capture.
+ *     attributes (no allocation); make that first call outside any stream capture. First calls
+ *     from several host threads are serialised by the library.
  *   - All calls on a device share the one array, which keeps the previous call's contents (the
  *     entry point re-zeroes the counters it needs on `stream` before launching). Two calls that
  *     may overlap on the GPU (different streams without ordering) race on it: serialise them.
@@ -204,6 +215,11 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
                                                   const int32_t* k, int32_t k_stride, void* out, int out_is_fp32,
                                                   void* stream);
 const char* fastocr_noalloc_last_error(void);
+/* Counterpart of fastocr_device_faults for the allocation-free entry point (the paper has no
+ * counterpart): synchronises the current device and returns how many device-side lengths, index-list
+ * or block-table entries its kernels have had to force into range on this device since the last
+ * call; clears the count. Not for the hot path. Negative on CUDA error. */
+int64_t fastocr_noalloc_device_faults(void);
 
 /*
  * Optional per-kernel timing (the paper has no counterpart; measurement aid). Between

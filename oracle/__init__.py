@@ -5,7 +5,7 @@ the product package. The arithmetic lives in fastocr_oracle.cpp (plain C++); thi
 a ctypes wrapper plus the step schedule of Algorithm 1 written over those primitives.
 """
 from .binding import (  # noqa: F401
-    dense, probs, scores, topk, sparse, masked_dense, kept_count, focal_layers, attn_flops,
+    dense, probs, scores, topk, sparse, masked_dense, kept_count, focal_layers, attn_flops, attn_flops_pruned,
     set_threads, num_threads,
 )
-from .schedule import decode_step, StepTrace, profile_focal_layers  # noqa: F401
+from .schedule import decode_step, warmup_step, StepTrace, profile_focal_layers  # noqa: F401

@@ -29,6 +29,8 @@ _lib.fastocr_oracle_kept_count.argtypes = [C.c_int, C.c_double]
 _lib.fastocr_oracle_focal_layers.argtypes = [_f64p, C.c_int, C.c_double, C.c_int, _i32p]
 _lib.fastocr_oracle_attn_flops.argtypes = [C.c_double] * 4
 _lib.fastocr_oracle_attn_flops.restype = C.c_double
+_lib.fastocr_oracle_attn_flops_pruned.argtypes = [C.c_double] * 6
+_lib.fastocr_oracle_attn_flops_pruned.restype = C.c_double
 
 
 def set_threads(n: int) -> None:
@@ -122,3 +124,7 @@ def focal_layers(mean_ratio, rho: float, gap: int):
 
 def attn_flops(b, l, h, s) -> float:
     return float(_lib.fastocr_oracle_attn_flops(float(b), float(l), float(h), float(s)))
+
+
+def attn_flops_pruned(b, l, h, s, full_layers, s_kept) -> float:
+    return float(_lib.fastocr_oracle_attn_flops_pruned(float(b), float(l), float(h), float(s), float(full_layers), float(s_kept)))

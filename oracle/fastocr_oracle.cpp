@@ -256,4 +256,14 @@ int fastocr_oracle_focal_layers(const double* mean_ratio, int L, double rho, int
 // Appendix B: self-attention FLOPs of one decode step, b * l * (8 h^2 + 4 h s).
 double fastocr_oracle_attn_flops(double b, double l, double h, double s) { return b * l * (8.0 * h * h + 4.0 * h * s); }
 
+// The same count for a pruned step (how Tables 1 and 2 arrive at the method's "FLOPs (G)"):
+// the projection term 8 h^2 is paid by every layer; `full_layers` of the l layers attend the whole
+// sequence s, the others attend s_kept tokens. The tables' values are reproduced with
+// s_kept = tau * s (the representative sequence counted as image tokens throughout).
+double fastocr_oracle_attn_flops_pruned(double b, double l, double h, double s, double full_layers, double s_kept) {
+  const double full = full_layers * (8.0 * h * h + 4.0 * h * s);
+  const double pruned = (l - full_layers) * (8.0 * h * h + 4.0 * h * s_kept);
+  return b * (full + pruned);
+}
+
 }  // extern "C"

@@ -15,7 +15,7 @@ class KVViewStruct(C.Structure):
         ("page_size", C.c_int32), ("max_seq_len", C.c_int32),
         ("k", C.c_void_p), ("v", C.c_void_p),
         ("seq_stride_tokens", C.c_int64),
-        ("block_table", C.c_void_p), ("max_pages", C.c_int32),
+        ("block_table", C.c_void_p), ("max_pages", C.c_int32), ("num_pages", C.c_int32),
         ("seq_len", C.c_void_p), ("vis_start", C.c_void_p), ("vis_len", C.c_void_p),
         ("sm_scale", C.c_float),
     ]
@@ -48,6 +48,7 @@ EXPORTS = {
     "fastocr_sparse_decode_attn_noalloc": (C.c_int, [C.POINTER(KVViewStruct), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                                      C.c_void_p, C.c_int, C.c_void_p]),
     "fastocr_noalloc_last_error": (C.c_char_p, []),
+    "fastocr_noalloc_device_faults": (C.c_int64, []),
     "fastocr_profile_begin": (C.c_int, [C.c_void_p, C.c_int32, C.c_int]),
     "fastocr_profile_end": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "fastocr_launch_count": (C.c_int64, []),

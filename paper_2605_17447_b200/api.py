@@ -55,6 +55,7 @@ class KVView:
     max_seq_len: int
     sm_scale: float
     block_table: Optional[torch.Tensor] = None   # int32 CUDA [B][max_pages] when paged
+    num_pages: int = -1            # paged: pages in the pools (block-table entries are clamped to it); -1: k.shape[0]
 
     def struct(self) -> _lib.KVViewStruct:
         _dev(self.k, torch.bfloat16, "k")
@@ -75,6 +76,7 @@ class KVView:
             s.page_size = int(self.k.shape[1])
             s.block_table = self.block_table.data_ptr()
             s.max_pages = int(self.block_table.shape[1])
+            s.num_pages = int(self.k.shape[0]) if self.num_pages < 0 else int(self.num_pages)
             s.seq_stride_tokens = 0
         else:
             s.page_size = 0

@@ -95,6 +95,7 @@ fastocr_status check_view(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
     return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "page_size %d is not 0 or a power of two", kv->page_size);
   if (kv->page_size > 0) {
     if (kv->block_table == nullptr || kv->max_pages <= 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "paged view without block_table");
+    if (kv->num_pages < 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "num_pages must not be negative");
     if (static_cast<int64_t>(kv->max_pages) * kv->page_size < kv->max_seq_len)
       return fail(ctx, FASTOCR_ERR_INVALID_ARG, "max_pages * page_size < max_seq_len");
   } else if (kv->seq_stride_tokens < kv->max_seq_len) {
@@ -118,6 +119,8 @@ AttnLaunch make_launch(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
   a.seq_stride_tokens = kv->seq_stride_tokens;
   a.block_table = kv->block_table;
   a.max_pages = kv->max_pages;
+  a.num_pages = kv->page_size > 0 ? kv->num_pages : 0;
+  a.max_seq_len = kv->max_seq_len;
   a.page_size = kv->page_size;
   a.page_shift = 0;
   while ((1 << a.page_shift) < kv->page_size) ++a.page_shift;

@@ -123,21 +123,34 @@ __device__ __forceinline__ void store_pair(void* out, int is_fp32, int64_t index
 
 // number of attended tokens of sequence b and the pieces needed to enumerate them
 struct SeqGeom {
-  int vs, N, kept_vis, n_tok;
+  int vs, N, kept_vis, n_tok;                           // n_tok < 0: the sequence takes no part in this launch
 };
-__device__ __forceinline__ SeqGeom load_geom(const AttnLaunch& a, int b, bool pruned) {
+// The lengths come from device memory and cannot be checked by the host without a synchronisation:
+// they are forced into what the host did check (0 <= seq_len <= max_seq_len, the image span inside
+// the sequence, the kept count inside the span and inside the index list's row), so that no cache
+// row, block-table entry or index-list entry outside the caller's buffers is ever addressed. `bad`
+// counts the lengths that had to be changed (a kept count above the span or the row length is
+// documented behaviour, not a fault).
+__device__ __forceinline__ SeqGeom load_geom(const AttnLaunch& a, int b, bool pruned, int& bad) {
   SeqGeom s;
-  const int S = a.seq_len[b];
-  s.vs = a.vis_start[b];
-  s.N = a.vis_len[b];
+  const int S_in = a.seq_len[b], vs_in = a.vis_start[b], N_in = a.vis_len[b];
+  const int S = min(max(S_in, 0), a.max_seq_len);
+  s.vs = min(max(vs_in, 0), S);
+  s.N = min(max(N_in, 0), S - s.vs);
+  bad += (S != S_in) + (s.vs != vs_in) + (s.N != N_in);
   if (pruned) {
     const int kk = a.kcount[b];
-    s.kept_vis = kk < 0 ? 0 : (kk > s.N ? s.N : kk);
+    s.kept_vis = min(max(kk, 0), min(s.N, a.k_stride));
   } else {
     s.kept_vis = s.N;
   }
-  s.n_tok = max(S - s.N + s.kept_vis, 0);
+  s.n_tok = S - s.N + s.kept_vis;
+  if (a.seq_mask != nullptr && a.seq_mask[b] != a.mask_want) s.n_tok = -1;
   return s;
+}
+__device__ __forceinline__ SeqGeom load_geom(const AttnLaunch& a, int b, bool pruned) {
+  int ignored = 0;
+  return load_geom(a, b, pruned, ignored);
 }
 
 // chunk swizzle of a staged row (16 chunks of 16 bytes): the eight rows of an ldmatrix 8x8 matrix
@@ -256,6 +269,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   // would span several units) sends the CTA through the full set-up.
   if (tid == 0) mrg_flag[3] = 0;
   __syncthreads();
+  int bad_lengths = 0;                                 // CTA 0: device-side lengths outside what the host checked
   int4 plan0 = make_int4(0, 0, 0, 0), plan1 = plan0, plan2 = plan0, plan3 = plan0;
   if (a.plan != nullptr) {
     const int4* rec = a.plan + 4 * static_cast<int64_t>(blockIdx.x);
@@ -279,7 +293,10 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) {
       const int uu = min(i * kThreads + tid, units - 1);
-      gq[i] = load_geom(a, uu / Hkv, HAS_IDX);
+      int bad = 0;
+      gq[i] = load_geom(a, uu / Hkv, HAS_IDX, bad);
+      // lengths that had to be forced into range: counted once per launch and sequence
+      if (blockIdx.x == 0 && i * kThreads + tid < units && uu % Hkv == 0) bad_lengths += bad;
     }
     int longest = 0;
 #pragma unroll
@@ -290,7 +307,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
         geom_s[uu] = make_int4(gq[i].vs, gq[i].N, gq[i].kept_vis, gq[i].n_tok);
         prefix_s[uu + 1] = rows;
         longest = max(longest, rows);
-        if (rows == 0) mrg_flag[3] = 1;                // some unit has nothing to attend (rare)
+        if (gq[i].n_tok == 0) mrg_flag[3] = 1;         // some unit has nothing to attend (rare)
       }
     }
 #pragma unroll
@@ -484,7 +501,12 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           pos = inside + sg.vs;
         }
         if (PAGED) {
-          const int page = __ldg(bt_row + (pos >> a.page_shift));   // page sizes are powers of two
+          int page = __ldg(bt_row + (pos >> a.page_shift));         // page sizes are powers of two
+          if (a.num_pages > 0) {                                    // never read outside the pool
+            const int inside = min(max(page, 0), a.num_pages - 1);
+            bad_entries += inside != page;
+            page = inside;
+          }
           pos = (page << a.page_shift) + (pos & (a.page_size - 1));
         }
         row = pos;
@@ -895,7 +917,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   }
 #endif
 
-  if (HAS_IDX && bad_entries != 0 && lane < kBlockTokens) atomicAdd(a.fault_counter, static_cast<unsigned long long>(bad_entries));
+  if ((HAS_IDX || PAGED) && bad_entries != 0 && lane < kBlockTokens) atomicAdd(a.fault_counter, static_cast<unsigned long long>(bad_entries));
+  if (bad_lengths != 0) atomicAdd(a.fault_counter, static_cast<unsigned long long>(bad_lengths));
 
   // A kernel of this library must not complete before its predecessor has (later kernels rely on
   // "my predecessor is done, hence everything before it"). CTAs that wrote only their own output
@@ -906,6 +929,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   if (blockIdx.x == 0 && mrg_flag[3] != 0) {           // (never with a plan: it is valid only when no unit is empty)
     for (int e = 0; e < units; ++e) {
       if (prefix_s[e + 1] != prefix_s[e]) continue;
+      if (load_geom(a, e / Hkv, HAS_IDX).n_tok != 0) continue;   // not part of this launch: left alone
       wait_for_prior_grids();
       const int64_t head0 = static_cast<int64_t>(e) * G;
       for (int i = tid; i < G * kHeadDim / 2; i += kThreads)
@@ -931,8 +955,10 @@ __global__ void __launch_bounds__(kMaxUnits) attn_plan_kernel(const AttnLaunch a
   SeqGeom sg = {0, 0, 0, 0};
   int rows = 0;
   if (tid < units) {
-    sg = load_geom(a, tid / Hkv, a.idx != nullptr);
+    int bad = 0;
+    sg = load_geom(a, tid / Hkv, a.idx != nullptr, bad);
     rows = (sg.n_tok + kRowTokens - 1) / kRowTokens;
+    if (bad != 0 && tid % Hkv == 0) atomicAdd(a.fault_counter, static_cast<unsigned long long>(bad));
   }
   int incl = rows, longest = rows;
 #pragma unroll
@@ -1053,7 +1079,7 @@ __global__ void __launch_bounds__(1024) image_mass_kernel(const float* __restric
   __shared__ float red[32];
   wait_for_prior_grids();
   dependents_may_launch();
-  const int b = blockIdx.x, N = vis_len[b];
+  const int b = blockIdx.x, N = min(vis_len[b], n_stride);
   float s = 0.f;
   for (int i = threadIdx.x; i < N; i += blockDim.x) s += scores[static_cast<int64_t>(b) * n_stride + i];
 #pragma unroll

@@ -100,11 +100,15 @@ struct AttnLaunch {
   int64_t seq_stride_tokens;
   const int32_t* block_table;
   int32_t max_pages;
+  int32_t num_pages;          // paged: pages in the pool (block-table entries are clamped to it); 0 = unknown, no check
   int32_t page_size;          // 0 = contiguous; else a power of two
   int32_t page_shift;         // log2(page_size)
+  int32_t max_seq_len;        // host bound on seq_len[b] (what the strides / the block table were checked against)
   const int32_t* seq_len;
   const int32_t* vis_start;
   const int32_t* vis_len;
+  const uint8_t* seq_mask;    // nullptr, or [B]: only sequences with seq_mask[b] == mask_want take part in this launch
+  int32_t mask_want;          //   (the others are neither read nor written: per-sequence focal layer sets)
   int32_t batch, num_q_heads, num_kv_heads;
   float sm_scale;
   const void* q;
@@ -150,12 +154,14 @@ cudaError_t launch_scores_finalize(const float* logits, const float* stats, cons
 cudaError_t launch_image_mass(const float* scores, int32_t n_stride, const int32_t* vis_len, int32_t batch,
                               float* mass, cudaStream_t s);
 
+// seq_mask: nullptr, or [B]; only sequences with seq_mask[b] == mask_want are selected for (the other rows of
+// idx_out are left as they are).
 // Scores come either from `scores` ([B][n_stride]) or, when `logits` is not NULL, are formed on the fly
 // from the attention kernel's logits ([B][H][n_stride_logits]) and per-head (max, sum) statistics.
 cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int32_t* vis_len, const int32_t* k,
                                int32_t batch, int32_t max_vis_len, int32_t* idx_out, int32_t k_stride,
                                const float* logits, const float* stats, int32_t num_q_heads, int32_t n_stride_logits,
-                               cudaStream_t s);
+                               cudaStream_t s, const uint8_t* seq_mask = nullptr, int32_t mask_want = 0);
 
 cudaError_t configure_kernels();   // one-time cudaFuncSetAttribute calls (current device)
 

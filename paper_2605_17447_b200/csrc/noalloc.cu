@@ -9,13 +9,15 @@
 // The price is a hard size limit and the loss of isolation between calls (see the header).
 #include "../../include/fastocr.h"
 
+#include <cmath>
 #include <cstdio>
+#include <mutex>
 
 #include "kernels.h"
 
 namespace {
 
-constexpr int kNoallocMaxSlots = FASTOCR_NOALLOC_MAX_UNITS + 3 * 160;   // units + persistent CTAs (3 per SM, <= 160 SMs)
+constexpr int kNoallocMaxSlots = FASTOCR_NOALLOC_MAX_UNITS + 3 * 160;   // units + persistent CTAs (the launch brings 2 per SM; room for 3 on up to 160 SMs)
 constexpr size_t kAccBytes = static_cast<size_t>(kNoallocMaxSlots) * fastocr::kMaxGroup * fastocr::kHeadDim * sizeof(float);
 constexpr size_t kMlBytes = static_cast<size_t>(kNoallocMaxSlots) * fastocr::kMaxGroup * 2 * sizeof(float);
 constexpr size_t kCounterBytes = static_cast<size_t>(FASTOCR_NOALLOC_MAX_UNITS) * sizeof(int32_t);
@@ -30,7 +32,9 @@ struct DeviceSetup {
   unsigned char* scratch = nullptr;   // device address of g_noalloc_scratch on this device
   int sm_count = 0;
 };
-DeviceSetup g_setup[64];
+constexpr int kMaxDevices = 64;
+DeviceSetup g_setup[kMaxDevices];
+std::mutex g_setup_lock;              // first calls from several host threads: one of them sets a device up, the others wait
 thread_local char g_error[256] = "";
 
 fastocr_status fail(fastocr_status code, const char* msg) {
@@ -41,6 +45,7 @@ fastocr_status fail(fastocr_status code, const char* msg) {
 // Once per device, with that device current: resolve the array's device address (in host code the
 // symbol is only a stand-in, not an address a kernel could use) and set the kernels' attributes.
 fastocr_status setup_current_device(int device) {
+  std::lock_guard<std::mutex> hold(g_setup_lock);     // also orders the fields below for every later caller
   DeviceSetup& s = g_setup[device];
   if (s.ready) return FASTOCR_OK;
   void* ptr = nullptr;
@@ -62,6 +67,23 @@ extern "C" {
 
 const char* fastocr_noalloc_last_error(void) { return g_error; }
 
+int64_t fastocr_noalloc_device_faults(void) {
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return -1;
+  unsigned char* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> hold(g_setup_lock);
+    if (!g_setup[device].ready) return 0;              // no call has run on this device yet
+    scratch = g_setup[device].scratch;
+  }
+  unsigned long long v = 0;
+  unsigned char* word = scratch + kAccBytes + kMlBytes + kCounterBytes;
+  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+  if (cudaMemcpy(&v, word, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  if (cudaMemset(word, 0, sizeof v) != cudaSuccess) return -1;
+  return static_cast<int64_t>(v);
+}
+
 fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, const void* q, const int32_t* idx,
                                                   const int32_t* k, int32_t k_stride, void* out, int out_is_fp32,
                                                   void* stream) {
@@ -80,7 +102,8 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   if (kv->page_size > 0 && (kv->block_table == nullptr || static_cast<int64_t>(kv->max_pages) * kv->page_size < kv->max_seq_len))
     return fail(FASTOCR_ERR_INVALID_ARG, "paged view needs a block_table covering max_seq_len");
   if (kv->page_size == 0 && kv->seq_stride_tokens < kv->max_seq_len) return fail(FASTOCR_ERR_INVALID_ARG, "seq_stride_tokens < max_seq_len");
-  if (!(kv->sm_scale > 0.f)) return fail(FASTOCR_ERR_INVALID_ARG, "sm_scale must be positive");
+  if (!(kv->sm_scale > 0.f) || !std::isfinite(kv->sm_scale)) return fail(FASTOCR_ERR_INVALID_ARG, "sm_scale must be positive and finite");
+  if (kv->page_size > 0 && kv->num_pages < 0) return fail(FASTOCR_ERR_INVALID_ARG, "num_pages must not be negative");
   const int64_t units = static_cast<int64_t>(kv->batch) * kv->num_kv_heads;
   if (units > FASTOCR_NOALLOC_MAX_UNITS) {
     snprintf(g_error, sizeof g_error, "batch x num_kv_heads = %lld exceeds the built-in scratch (limit %d); use a context",
@@ -90,7 +113,7 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   int device = 0;
   cudaError_t e = cudaGetDevice(&device);
   if (e != cudaSuccess) return fail(FASTOCR_ERR_CUDA, cudaGetErrorString(e));
-  if (device < 0 || device >= 64) return fail(FASTOCR_ERR_UNSUPPORTED, "device ordinal above 63");
+  if (device < 0 || device >= kMaxDevices) return fail(FASTOCR_ERR_UNSUPPORTED, "device ordinal above 63");
   fastocr_status st = setup_current_device(device);
   if (st != FASTOCR_OK) return st;
   const DeviceSetup& s = g_setup[device];
@@ -105,10 +128,11 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   if (units + grid > kNoallocMaxSlots) return fail(FASTOCR_ERR_WORKSPACE, "this GPU has more SMs than the built-in scratch was sized for");
 
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  // The arrival counters and the fault word must start at zero; partial slots are written before
-  // they are read. (The array keeps whatever the previous call left.)
+  // The arrival counters must start at zero; partial slots are written before they are read.
+  // (The array keeps whatever the previous call left; the fault word is meant to: it adds up until
+  // fastocr_noalloc_device_faults reads and clears it. A module's __device__ arrays start as zeros.)
   unsigned char* counters = s.scratch + kAccBytes + kMlBytes;
-  if ((e = cudaMemsetAsync(counters, 0, kCounterBytes + kFaultBytes, cs)) != cudaSuccess)
+  if ((e = cudaMemsetAsync(counters, 0, kCounterBytes, cs)) != cudaSuccess)
     return fail(FASTOCR_ERR_CUDA, cudaGetErrorString(e));
 
   fastocr::AttnLaunch a{};
@@ -117,6 +141,8 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   a.seq_stride_tokens = kv->seq_stride_tokens;
   a.block_table = kv->block_table;
   a.max_pages = kv->max_pages;
+  a.num_pages = kv->page_size > 0 ? kv->num_pages : 0;
+  a.max_seq_len = kv->max_seq_len;
   a.page_size = kv->page_size;
   while ((1 << a.page_shift) < kv->page_size) ++a.page_shift;
   a.seq_len = kv->seq_len;

@@ -145,7 +145,8 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
                                                                    int32_t* __restrict__ idx_out, int k_stride, int n_cap,
                                                                    const float* __restrict__ logits,
                                                                    const float* __restrict__ stats, int num_q_heads,
-                                                                   int n_stride_logits, int drop_logits) {
+                                                                   int n_stride_logits, int drop_logits,
+                                                                   const uint8_t* __restrict__ seq_mask, int mask_want) {
   extern __shared__ __align__(16) uint32_t keys[];      // all keys of the sequence
   __shared__ float head_st[2 * kTopkMaxHeads];          // scoring mode: per head (max, 1 / sum)
   __shared__ uint32_t hist[kTopkBins];
@@ -158,10 +159,11 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   const int C = static_cast<int>(cluster.num_blocks());
   const int c = static_cast<int>(cluster.block_rank());
   const int b = blockIdx.x / C, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int N = min(vis_len[b], n_cap);                 // n_cap: what the launch sized the key array for
+  const int N = max(min(vis_len[b], n_cap), 0);         // n_cap: what the launch sized the key array for
   int k = kreq[b];
   k = k < 0 ? 0 : (k > N ? N : k);
   k = min(k, k_stride);
+  if (seq_mask != nullptr && seq_mask[b] != mask_want) k = 0;   // this sequence's set is not refreshed by this launch
   if (k == 0) return;                                   // the same decision in every CTA of the cluster
 
   // slice [lo_i, hi_i) of the tokens: what this CTA scores and emits; a multiple of 32 per CTA
@@ -385,7 +387,8 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_split_kernel(const f
                                                                    int32_t* __restrict__ idx_out, int k_stride, int n_cap,
                                                                    const float* __restrict__ logits,
                                                                    const float* __restrict__ stats, int num_q_heads,
-                                                                   int n_stride_logits, int drop_logits) {
+                                                                   int n_stride_logits, int drop_logits,
+                                                                   const uint8_t* __restrict__ seq_mask, int mask_want) {
   extern __shared__ __align__(16) uint32_t keys[];      // keys of the CTA's slice (key of token lo_i + j at j)
   __shared__ float head_st[2 * kTopkMaxHeads];          // scoring mode: per head (max, 1 / sum)
   __shared__ uint32_t hist[2][kTopkBins];               // per pass, alternating: the peers read one while the other refills
@@ -399,10 +402,11 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_split_kernel(const f
   const int C = static_cast<int>(cluster.num_blocks());
   const int c = static_cast<int>(cluster.block_rank());
   const int b = blockIdx.x / C, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int N = min(vis_len[b], n_cap);                 // n_cap: what the launch sized the key arrays for
+  const int N = max(min(vis_len[b], n_cap), 0);         // n_cap: what the launch sized the key arrays for
   int k = kreq[b];
   k = k < 0 ? 0 : (k > N ? N : k);
   k = min(k, k_stride);
+  if (seq_mask != nullptr && seq_mask[b] != mask_want) k = 0;   // this sequence's set is not refreshed by this launch
   if (k == 0) return;                                   // the same decision in every CTA of the cluster
 
   // slice [lo_i, hi_i) of the tokens: what this CTA scores, histograms and emits; a multiple of 32 per CTA
@@ -670,7 +674,7 @@ cudaError_t configure_topk() {
 cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int32_t* vis_len, const int32_t* k,
                                int32_t batch, int32_t max_vis_len, int32_t* idx_out, int32_t k_stride,
                                const float* logits, const float* stats, int32_t num_q_heads, int32_t n_stride_logits,
-                               cudaStream_t s) {
+                               cudaStream_t s, const uint8_t* seq_mask, int32_t mask_want) {
   if (batch <= 0 || max_vis_len <= 0) return cudaSuccess;
   if (logits != nullptr && (num_q_heads <= 0 || num_q_heads > kTopkMaxHeads)) return cudaErrorInvalidValue;
   // Cluster size: one CTA per sequence when the scores exist; when they are formed here, enough
@@ -715,11 +719,11 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
     cfg.dynamicSmemBytes = ((static_cast<size_t>(max_vis_len) + C - 1) / C + 31) / 32 * 32 * 4 + 16;   // one slice's keys
     e = cudaLaunchKernelEx(&cfg, select_topk_split_kernel, scores, n_stride, vis_len, k, idx_out, k_stride,
                            static_cast<int>(max_vis_len), logits, stats, static_cast<int>(num_q_heads),
-                           static_cast<int>(n_stride_logits), drop);
+                           static_cast<int>(n_stride_logits), drop, seq_mask, static_cast<int>(mask_want));
   } else {
     e = cudaLaunchKernelEx(&cfg, select_topk_kernel, scores, n_stride, vis_len, k, idx_out, k_stride,
                            static_cast<int>(max_vis_len), logits, stats, static_cast<int>(num_q_heads),
-                           static_cast<int>(n_stride_logits), drop);
+                           static_cast<int>(n_stride_logits), drop, seq_mask, static_cast<int>(mask_want));
   }
   count_launches(1);
   return e;

@@ -18,6 +18,17 @@ def test_attention_flops_reproduce_printed_values():
         assert abs(got - row["printed"]) < 0.006, row["cite"]
 
 
+def test_pruned_flops_reproduce_printed_values():
+    for row in GOLD["attn_flops_pruned_G"]["rows"]:
+        got = oracle.attn_flops_pruned(row["b"], row["l"], row["h"], row["s"], row["full_layers"], row["tau"] * row["s"]) / 1e9
+        assert abs(got - row["printed"]) < row["tol"], (row["cite"], got)
+    # special cases: every layer full = the vanilla count; no layer full, nothing kept = projections only
+    assert oracle.attn_flops_pruned(8, 36, 2048, 4096, 36, 0) == oracle.attn_flops(8, 36, 2048, 4096)
+    assert oracle.attn_flops_pruned(2, 10, 64, 999, 0, 0) == 2 * 10 * 8 * 64 * 64
+    # a dropped projection term on the pruned layers, or tau*s swapped for s, would miss the printed values by > 1 G
+    assert abs(oracle.attn_flops_pruned(8, 36, 2048, 4096, 4, 4096) / 1e9 - 19.33) < 0.006
+
+
 def test_kept_count_is_a_ceiling():
     assert oracle.kept_count(1024, 0.05) == 52          # 51.2 -> 52 (a floor would give 51)
     assert [oracle.kept_count(n, 0.05) for n in (4096, 8192, 16384, 32768)] == [205, 410, 820, 1639]
@@ -103,3 +114,40 @@ def test_schedule_layer0_focal_and_no_focal_layers():
     assert t.mode == ["focal", "pruned", "pruned"] and torch.equal(t.f_last, t.selected[0])
     t = oracle.decode_step(lay, [], prev, vs, N, tau, SCALE)            # C empty with a set: pure reuse
     assert t.mode == ["pruned"] * 3 and torch.equal(t.f_last, prev)
+
+
+def test_schedule_union_of_the_steps_selections():
+    # L=5, C={1,3}: layer 0 borrows last step's set; layer 1 selects F1 (replaces the borrowed set);
+    # layer 2 attends T u F1; layer 3 selects F3; layer 4 attends T u (F1 u F3) in the union variant
+    # and T u F3 in Algorithm 1 itself; in both, F3 alone is carried to the next step.
+    vs, N, tau = 5, 60, 0.1
+    lay = _layers(7, 5, 70)
+    prev = torch.tensor([0, 1, 2, 3, 4, 59], dtype=torch.int32)
+    plain = oracle.decode_step(lay, [1, 3], prev, vs, N, tau, SCALE)
+    uni = oracle.decode_step(lay, [1, 3], prev, vs, N, tau, SCALE, union_sets=True)
+    assert uni.mode == plain.mode == ["pruned", "focal", "pruned", "focal", "pruned"]
+    f1, f3 = plain.selected[1], plain.selected[3]
+    assert torch.equal(uni.selected[1], f1) and torch.equal(uni.selected[3], f3)      # selections do not depend on the variant
+    assert torch.equal(uni.used_set[0], prev) and torch.equal(uni.used_set[2], f1)
+    both = sorted(set(f1.tolist()) | set(f3.tolist()))
+    assert uni.used_set[4].tolist() == both and len(both) > len(f3)                    # the sets differ on this input
+    assert torch.equal(plain.used_set[4], f3)
+    assert torch.equal(uni.outputs[4], oracle.sparse(*lay[4], SCALE, vs, N, torch.tensor(both, dtype=torch.int32)))
+    assert not torch.equal(uni.outputs[4], plain.outputs[4])
+    for l in range(4):
+        assert torch.equal(uni.outputs[l], plain.outputs[l])
+    assert torch.equal(uni.f_last, f3) and torch.equal(plain.f_last, f3)
+    # the fallback's selection at layer 0 counts as the step's first
+    u2 = oracle.decode_step(lay, [3], None, vs, N, tau, SCALE, union_sets=True)
+    assert u2.used_set[4].tolist() == sorted(set(u2.selected[0].tolist()) | set(u2.selected[3].tolist()))
+
+
+def test_warmup_step_is_dense_everywhere_and_records_eq1():
+    vs, N = 4, 40
+    lay = _layers(9, 3, 50)
+    outs, ratios = oracle.warmup_step(lay, vs, N, SCALE)
+    for l in range(3):
+        assert torch.equal(outs[l], oracle.dense(*lay[l], SCALE))
+        p = oracle.probs(lay[l][0], lay[l][1], SCALE, True).double().mean(dim=0)     # head-averaged weights over the cache
+        img, txt = p[vs:vs + N].sum(), p[:vs].sum() + p[vs + N:].sum()
+        assert abs(ratios[l] - float(img / (img + txt))) < 1e-6 and 0 < ratios[l] < 1   # Eq. 1 written out
