@@ -118,9 +118,13 @@ int32_t fastocr_kept_count(int32_t n_vis, double tau);
  *   scores_out NULL, or device fp32 [B][n_stride]: additionally receives the head-averaged image
  *              attention of fastocr_focal_scores from the same pass over K (entries
  *              [vis_len[b], n_stride) are left untouched); n_stride >= max vis_len.
+ *   image_mass_out NULL, or device fp32 [B]: Eq. 1's image-attention ratio r of this layer (the sum
+ *              of those scores over the image span), from the same pass; what a warm-up step records
+ *              (Section 3.1.1). May be asked for without scores_out.
  */
 fastocr_status fastocr_dense_decode_attn(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, void* out,
-                                         int out_is_fp32, float* scores_out, int32_t n_stride, void* stream);
+                                         int out_is_fp32, float* scores_out, int32_t n_stride, float* image_mass_out,
+                                         void* stream);
 
 /*
  * Focal scores: for image token i of sequence b, the attention weight from the current query to
@@ -180,6 +184,44 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
                                    int32_t max_vis_len, int32_t max_kept, int* has_fixation_out, void* stream);
 
 /*
+ * The same step with options (NULL options = fastocr_decode_step):
+ *   is_focal_seq / is_focal_seq_dev  per-sequence focal layer sets (Section 3.1.1 and Appendix E: C is
+ *       profiled per sample): the matrix [L][B] of memberships, once in host memory (the library
+ *       decides the launches from it) and once in device memory (the kernels read a layer's row to
+ *       tell which sequences take part in a launch); both or neither. It replaces is_focal, which
+ *       may then be NULL. A layer that is focal for some sequences only runs as a pruned pass over
+ *       the others followed by a full pass and a selection over those. The caller uploads the device
+ *       copy once, C being frozen after warm-up.
+ *   union_sets  a variant, not Algorithm 1: the kept image set after a focal layer is the union of the
+ *       sets selected so far in this step (Section 3.1.1 calls the union over the focal layers the
+ *       aggregated focal token set); the first selection of a step replaces what was borrowed from
+ *       the previous step. `fixation` still receives every focal layer's own selection, so that what
+ *       is carried to the next step is the deepest focal layer's set as in Algorithm 1. The union
+ *       lives in the context's workspace; max_kept must bound text + union size.
+ */
+typedef struct fastocr_step_options {
+  const uint8_t* is_focal_seq;     /* host uint8 [L][B], or NULL   */
+  const uint8_t* is_focal_seq_dev; /* device uint8 [L][B], or NULL */
+  int32_t union_sets;              /* 0 = Algorithm 1              */
+} fastocr_step_options;
+fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
+                                      const void* q, void* out, int out_is_fp32, const uint8_t* is_focal,
+                                      const int32_t* k, int32_t* fixation, int32_t k_stride, int has_fixation,
+                                      int32_t max_vis_len, int32_t max_kept, int* has_fixation_out,
+                                      const fastocr_step_options* options, void* stream);
+
+/*
+ * One warm-up step (Algorithm 1, profiling block; Section 3.1.1): nothing is pruned, every layer
+ * attends the full cache, and Eq. 1's image-attention ratio is recorded for every layer and
+ * sequence from the same pass over K that produces the layer's output.
+ *   layers, q, out as in fastocr_decode_step
+ *   ratio_out device fp32 [L][B]: r of layer l and sequence b at this step; the caller averages
+ *             the w steps' records per sequence and hands the means to fastocr_focal_layers
+ */
+fastocr_status fastocr_warmup_step(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers, const void* q,
+                                   void* out, int out_is_fp32, float* ratio_out, void* stream);
+
+/*
  * Focal Layer Selection (Section 3.1.1; Algorithm 1, profiling block), host-only: rank layers by
  * mean image-attention ratio (descending; equal ratios: lower layer first) and accept greedily
  * while fewer than floor(rho*L) are chosen and the candidate is more than `gap` layers from every
@@ -191,6 +233,10 @@ int32_t fastocr_focal_layers(const double* mean_ratio, int32_t num_layers, doubl
 
 /* Appendix B: self-attention FLOPs of one decode step, b*l*(8h^2 + 4hs). Host-only. */
 double fastocr_attn_flops(double batch, double layers, double hidden, double seq_len);
+/* The same count for a pruned step, as Tables 1 and 2 print it for the method: every layer pays the
+ * projections, `full_layers` of them attend seq_len tokens, the others kept_len tokens. Host-only. */
+double fastocr_attn_flops_pruned(double batch, double layers, double hidden, double seq_len, double full_layers,
+                                 double kept_len);
 
 /*
  * Pruned decode attention without a context and without any allocation (the paper has no

@@ -21,6 +21,10 @@ class KVViewStruct(C.Structure):
     ]
 
 
+class StepOptionsStruct(C.Structure):
+    _fields_ = [("is_focal_seq", C.c_void_p), ("is_focal_seq_dev", C.c_void_p), ("union_sets", C.c_int32)]
+
+
 class LimitsStruct(C.Structure):
     _fields_ = [("max_batch", C.c_int32), ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
                 ("max_seq_len", C.c_int32), ("max_vis_len", C.c_int32)]
@@ -33,7 +37,7 @@ EXPORTS = {
     "fastocr_device_faults": (C.c_int64, [C.c_void_p]),
     "fastocr_kept_count": (C.c_int32, [C.c_int32, C.c_double]),
     "fastocr_dense_decode_attn": (C.c_int, [C.c_void_p, C.POINTER(KVViewStruct), C.c_void_p, C.c_void_p, C.c_int,
-                                            C.c_void_p, C.c_int32, C.c_void_p]),
+                                            C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "fastocr_focal_scores": (C.c_int, [C.c_void_p, C.POINTER(KVViewStruct), C.c_void_p, C.c_void_p, C.c_int32,
                                        C.c_void_p, C.c_void_p]),
     "fastocr_select_topk": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
@@ -43,8 +47,14 @@ EXPORTS = {
     "fastocr_decode_step": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(KVViewStruct), C.c_void_p, C.c_void_p, C.c_int,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int, C.c_int32, C.c_int32,
                                       C.POINTER(C.c_int), C.c_void_p]),
+    "fastocr_decode_step_ex": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(KVViewStruct), C.c_void_p, C.c_void_p, C.c_int,
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int, C.c_int32, C.c_int32,
+                                         C.POINTER(C.c_int), C.POINTER(StepOptionsStruct), C.c_void_p]),
+    "fastocr_warmup_step": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(KVViewStruct), C.c_void_p, C.c_void_p, C.c_int,
+                                      C.c_void_p, C.c_void_p]),
     "fastocr_focal_layers": (C.c_int32, [C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_void_p]),
     "fastocr_attn_flops": (C.c_double, [C.c_double] * 4),
+    "fastocr_attn_flops_pruned": (C.c_double, [C.c_double] * 6),
     "fastocr_sparse_decode_attn_noalloc": (C.c_int, [C.POINTER(KVViewStruct), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                                      C.c_void_p, C.c_int, C.c_void_p]),
     "fastocr_noalloc_last_error": (C.c_char_p, []),

@@ -153,6 +153,11 @@ def attn_flops(batch, layers, hidden, seq_len) -> float:
     return float(_lib.load().fastocr_attn_flops(float(batch), float(layers), float(hidden), float(seq_len)))
 
 
+def attn_flops_pruned(batch, layers, hidden, seq_len, full_layers, kept_len) -> float:
+    return float(_lib.load().fastocr_attn_flops_pruned(float(batch), float(layers), float(hidden), float(seq_len),
+                                                       float(full_layers), float(kept_len)))
+
+
 def launch_count() -> int:
     return int(_lib.load().fastocr_launch_count())
 
@@ -162,14 +167,17 @@ def cluster_launch_count() -> int:
 
 
 def fastocr_dense_decode_attn(ctx: Context, kv: KVView, q: torch.Tensor, out: torch.Tensor,
-                              scores_out: Optional[torch.Tensor] = None, stream=None) -> None:
+                              scores_out: Optional[torch.Tensor] = None, image_mass_out: Optional[torch.Tensor] = None,
+                              stream=None) -> None:
     _dev(q, torch.bfloat16, "q")
     st = kv.struct()
     n_stride = int(scores_out.shape[-1]) if scores_out is not None else 0
     if scores_out is not None:
         _dev(scores_out, torch.float32, "scores_out")
+    if image_mass_out is not None:
+        _dev(image_mass_out, torch.float32, "image_mass_out")
     ctx.check(ctx._lib.fastocr_dense_decode_attn(ctx._h, C.byref(st), _ptr(q), _ptr(out), int(out.dtype == torch.float32),
-                                                 _ptr(scores_out), n_stride, _stream(stream)))
+                                                 _ptr(scores_out), n_stride, _ptr(image_mass_out), _stream(stream)))
 
 
 def fastocr_focal_scores(ctx: Context, kv: KVView, q: torch.Tensor, scores_out: torch.Tensor,
@@ -218,45 +226,75 @@ def fastocr_sparse_decode_attn_noalloc(kv: KVView, q: torch.Tensor, idx: torch.T
         raise FastOCRError(rc, lib.fastocr_noalloc_last_error().decode())
 
 
+class _StepArgs:
+    """Marshalled arguments of fastocr_decode_step_ex that do not change between steps."""
+
+    def __init__(self, layers: Sequence[KVView], is_focal, k: torch.Tensor, fixation: torch.Tensor, max_vis_len: int,
+                 max_kept: int, union_sets: bool):
+        self.L = len(layers)
+        self.keep = (list(layers), k, fixation)
+        self.arr = (_lib.KVViewStruct * self.L)(*[kv.struct() for kv in layers])
+        focal = np.ascontiguousarray(np.asarray(is_focal, dtype=np.uint8))
+        self.opt = _lib.StepOptionsStruct(None, None, int(bool(union_sets)))
+        self.focal = focal
+        self.focal_ptr = focal.ctypes.data
+        if focal.ndim == 2:                       # per-sequence focal layer sets [L][B]: host copy + device copy
+            if focal.shape != (self.L, int(k.numel())):
+                raise ValueError("per-sequence focal sets must be [layers][batch]")
+            self.focal_dev = torch.from_numpy(focal).to(k.device)
+            self.opt.is_focal_seq = focal.ctypes.data
+            self.opt.is_focal_seq_dev = self.focal_dev.data_ptr()
+            self.focal_ptr = None
+        elif focal.shape != (self.L,):
+            raise ValueError("is_focal must have one entry per layer")
+        self.k = _ptr(_dev(k, torch.int32, "k"))
+        self.fix = _ptr(_dev(fixation, torch.int32, "fixation"))
+        self.k_stride = int(fixation.shape[-1])
+        self.max_vis, self.max_kept = int(max_vis_len), int(max_kept)
+        self.have = C.c_int(0)
+
+    def run(self, ctx: Context, q: torch.Tensor, out: torch.Tensor, has_fixation: bool, stream=None) -> bool:
+        ctx.check(ctx._lib.fastocr_decode_step_ex(ctx._h, self.L, self.arr, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()),
+                                                  int(out.dtype == torch.float32), self.focal_ptr, self.k, self.fix,
+                                                  self.k_stride, int(bool(has_fixation)), self.max_vis, self.max_kept,
+                                                  C.byref(self.have), C.byref(self.opt), _stream(stream)))
+        return bool(self.have.value)
+
+
+def noalloc_device_faults() -> int:
+    """Values the allocation-free entry point's kernels have had to force into range on the current device."""
+    return int(_lib.load().fastocr_noalloc_device_faults())
+
+
 def fastocr_decode_step(ctx: Context, layers: Sequence[KVView], q: torch.Tensor, out: torch.Tensor,
-                        is_focal: Sequence[bool], k: torch.Tensor, fixation: torch.Tensor, has_fixation: bool,
-                        max_vis_len: int, max_kept: int = 0, stream=None) -> bool:
-    """q/out: [L][B][H][128]. Returns whether `fixation` is valid after the step."""
+                        is_focal, k: torch.Tensor, fixation: torch.Tensor, has_fixation: bool,
+                        max_vis_len: int, max_kept: int = 0, union_sets: bool = False, stream=None) -> bool:
+    """q/out: [L][B][H][128]. is_focal: [L] (one focal layer set for the batch) or [L][B] (per-sequence
+    sets). Returns whether `fixation` is valid after the step."""
     _dev(q, torch.bfloat16, "q")
-    _dev(k, torch.int32, "k")
-    _dev(fixation, torch.int32, "fixation")
+    return _StepArgs(layers, is_focal, k, fixation, max_vis_len, max_kept, union_sets).run(ctx, q, out, has_fixation, stream)
+
+
+def fastocr_warmup_step(ctx: Context, layers: Sequence[KVView], q: torch.Tensor, out: torch.Tensor,
+                        ratio_out: torch.Tensor, stream=None) -> None:
+    """One warm-up step: every layer dense, Eq. 1's ratio of layer l and sequence b into ratio_out[l][b]."""
+    _dev(q, torch.bfloat16, "q")
+    _dev(ratio_out, torch.float32, "ratio_out")
     L = len(layers)
     arr = (_lib.KVViewStruct * L)(*[kv.struct() for kv in layers])
-    focal = np.ascontiguousarray(np.asarray(is_focal, dtype=np.uint8))
-    have = C.c_int(0)
-    ctx.check(ctx._lib.fastocr_decode_step(ctx._h, L, arr, _ptr(q), _ptr(out), int(out.dtype == torch.float32),
-                                           focal.ctypes.data, _ptr(k), _ptr(fixation), int(fixation.shape[-1]),
-                                           int(bool(has_fixation)), int(max_vis_len), int(max_kept), C.byref(have),
-                                           _stream(stream)))
-    return bool(have.value)
+    ctx.check(ctx._lib.fastocr_warmup_step(ctx._h, L, arr, _ptr(q), _ptr(out), int(out.dtype == torch.float32),
+                                           _ptr(ratio_out), _stream(stream)))
 
 
 class StepPlan:
     """fastocr_decode_step with everything that does not change between steps marshalled once
     (the per-step Python cost is then a single foreign call)."""
 
-    def __init__(self, ctx: Context, layers: Sequence[KVView], is_focal: Sequence[bool], k: torch.Tensor,
-                 fixation: torch.Tensor, max_vis_len: int, max_kept: int = 0):
+    def __init__(self, ctx: Context, layers: Sequence[KVView], is_focal, k: torch.Tensor,
+                 fixation: torch.Tensor, max_vis_len: int, max_kept: int = 0, union_sets: bool = False):
         self.ctx = ctx
         self.L = len(layers)
-        self._keep = (list(layers), k, fixation)
-        self._arr = (_lib.KVViewStruct * self.L)(*[kv.struct() for kv in layers])
-        self._focal = np.ascontiguousarray(np.asarray(is_focal, dtype=np.uint8))
-        self._k = _ptr(_dev(k, torch.int32, "k"))
-        self._fix = _ptr(_dev(fixation, torch.int32, "fixation"))
-        self._k_stride = int(fixation.shape[-1])
-        self._max_vis, self._max_kept = int(max_vis_len), int(max_kept)
-        self._have = C.c_int(0)
+        self._args = _StepArgs(layers, is_focal, k, fixation, max_vis_len, max_kept, union_sets)
 
     def run(self, q: torch.Tensor, out: torch.Tensor, has_fixation: bool, stream=None) -> bool:
-        c = self.ctx
-        c.check(c._lib.fastocr_decode_step(c._h, self.L, self._arr, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()),
-                                           int(out.dtype == torch.float32), self._focal.ctypes.data, self._k, self._fix,
-                                           self._k_stride, int(bool(has_fixation)), self._max_vis, self._max_kept,
-                                           C.byref(self._have), _stream(stream)))
-        return bool(self._have.value)
+        return self._args.run(self.ctx, q, out, has_fixation, stream)

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfastocr.so")
-SOURCES = ["api.cu", "attn.cu", "topk.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "attn.cu", "topk.cu", "sets.cu", "noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 
@@ -31,12 +31,12 @@ def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str |
     tag = "" if out is None else "." + os.path.basename(out).replace(".so", "")
     if verbose:
         flags += ["-Xptxas", "-v"]
-    objs = []
-    for src in SOURCES:
-        obj = os.path.join(CSRC, src.replace(".cu", tag + ".o"))
-        subprocess.check_call([nvcc, *flags, "-c", os.path.join(CSRC, src), "-o", obj])
-        objs.append(obj)
-    subprocess.check_call([nvcc, "-shared", "-o", lib, *objs, "-lcudart"])
+    objs = [os.path.join(CSRC, src.replace(".cu", tag + ".o")) for src in SOURCES]
+    procs = [subprocess.Popen([nvcc, *flags, "-c", os.path.join(CSRC, src), "-o", obj]) for src, obj in zip(SOURCES, objs)]
+    failed = [src for src, p in zip(SOURCES, procs) if p.wait() != 0]      # the files compile side by side
+    if failed:
+        raise subprocess.CalledProcessError(1, f"nvcc -c {' '.join(failed)}")
+    subprocess.check_call([nvcc, "-shared", "-o", lib, *objs, "-lcudart", "-ldl"])
     return lib
 
 

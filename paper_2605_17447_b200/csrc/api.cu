@@ -11,6 +11,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "kernels.h"
 
 namespace fastocr {
@@ -35,6 +37,8 @@ struct fastocr_ctx {
   float* logits = nullptr;      // [max_batch][H][max_vis_len]
   float* stats = nullptr;       // [max_batch][H][2]
   float* scores = nullptr;      // [max_batch][max_vis_len] (decode_step scratch)
+  int32_t* uni_idx = nullptr;   // [2][max_batch][max_vis_len]: kept image sets of the union variant (current / next)
+  int32_t* uni_cnt = nullptr;   // [2][max_batch]
   unsigned long long* faults = nullptr;
   // persistent attention CTAs per SM brought by one launch: a full cache pass takes every slot,
   // a pruned pass half of them (the next layers' launches run beside it; two per SM measured equal
@@ -218,12 +222,19 @@ struct ProfScope {
     if (e_ != cudaSuccess) return cuda_fail(ctx, e_, what);  \
   } while (0)
 
+// One NVTX range per entry point (visible in a timeline when a tool is attached, free otherwise).
+struct NvtxScope {
+  explicit NvtxScope(const char* name) { nvtxRangePushA(name); }
+  ~NvtxScope() { nvtxRangePop(); }
+};
+
 // dense pass (+ optional fused scoring) without re-validating the view
 // scores_out == NULL with logits_only: logits and per-head statistics are left in the context's
 // workspace for a consumer that forms the scores itself (the selection kernel)
 fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, void* out, int out_is_fp32,
                           float* scores_out, int32_t n_stride, int32_t max_vis, int wait_point, cudaStream_t s,
-                          bool logits_only = false) {
+                          bool logits_only = false, float* image_mass_out = nullptr, const uint8_t* seq_mask = nullptr,
+                          int mask_want = 0) {
   AttnLaunch a = make_launch(ctx, kv, q, /*with_v=*/out != nullptr, kv->max_seq_len);
   const bool want_scores = scores_out != nullptr || logits_only;
   if (want_scores) {
@@ -234,6 +245,8 @@ fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
   a.out_is_fp32 = out_is_fp32;
   a.wait_point = wait_point;
   a.stats = want_scores ? ctx->stats : nullptr;
+  a.seq_mask = seq_mask;
+  a.mask_want = mask_want;
   {
     ProfScope p(ctx, out != nullptr ? FASTOCR_PROF_ATTN_DENSE : FASTOCR_PROF_ATTN_KEYS, s);
     FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
@@ -243,6 +256,10 @@ fastocr_status dense_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
     FASTOCR_TRY_CUDA(fastocr::launch_scores_finalize(ctx->logits, ctx->stats, kv->vis_len, kv->batch, kv->num_q_heads,
                                                      ctx->lim.max_vis_len, max_vis, scores_out, n_stride, s),
                      "score finalisation launch");
+    if (image_mass_out != nullptr) {
+      ProfScope pm(ctx, FASTOCR_PROF_MASS, s);
+      FASTOCR_TRY_CUDA(fastocr::launch_image_mass(scores_out, n_stride, kv->vis_len, kv->batch, image_mass_out, s), "image mass launch");
+    }
   }
   return FASTOCR_OK;
 }
@@ -283,9 +300,12 @@ AttnLaunch sparse_args(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* 
 // plan: NULL or a launch plan made for exactly these lengths, kept counts and plan_grid CTAs.
 fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, const int32_t* idx,
                            const int32_t* k, int32_t k_stride, int32_t max_kept, void* out, int out_is_fp32,
-                           int wait_point, cudaStream_t s, const int4* plan = nullptr, int plan_grid = 0) {
+                           int wait_point, cudaStream_t s, const int4* plan = nullptr, int plan_grid = 0,
+                           const uint8_t* seq_mask = nullptr, int mask_want = 0) {
   AttnLaunch a = sparse_args(ctx, kv, q, idx, k, k_stride, max_kept);
   a.wait_point = wait_point;
+  a.seq_mask = seq_mask;
+  a.mask_want = mask_want;
   a.plan = (plan != nullptr && plan_grid == a.grid_ctas) ? plan : nullptr;
   a.out = out;
   a.out_is_fp32 = out_is_fp32;
@@ -357,6 +377,8 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   if ((e = cudaMalloc(&ctx->part_acc, bytes_acc)) != cudaSuccess || (e = cudaMalloc(&ctx->part_ml, bytes_ml)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->logits, bytes_logits)) != cudaSuccess || (e = cudaMalloc(&ctx->stats, bytes_stats)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->scores, bytes_scores)) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->uni_idx, 2 * static_cast<size_t>(lim->max_batch) * nvis * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->uni_cnt, 2 * static_cast<size_t>(lim->max_batch) * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->counters, fastocr::kMaxUnits * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->plan, static_cast<size_t>(kPlanCtas) * 4 * sizeof(int4))) != cudaSuccess ||
       (e = cudaMemset(ctx->counters, 0, fastocr::kMaxUnits * sizeof(int32_t))) != cudaSuccess ||
@@ -378,6 +400,8 @@ void fastocr_destroy(fastocr_ctx* ctx) {
   cudaFree(ctx->logits);
   cudaFree(ctx->stats);
   cudaFree(ctx->scores);
+  cudaFree(ctx->uni_idx);
+  cudaFree(ctx->uni_cnt);
   cudaFree(ctx->counters);
   cudaFree(ctx->faults);
   if (ctx->l2_persist_set) cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, ctx->l2_persist_before);
@@ -404,34 +428,36 @@ int32_t fastocr_kept_count(int32_t n_vis, double tau) {
 }
 
 fastocr_status fastocr_dense_decode_attn(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, void* out,
-                                         int out_is_fp32, float* scores_out, int32_t n_stride, void* stream) {
+                                         int out_is_fp32, float* scores_out, int32_t n_stride, float* image_mass_out,
+                                         void* stream) {
+  NvtxScope range("fastocr_dense_decode_attn");
   fastocr_status st = check_view(ctx, kv, q, true);
   if (st != FASTOCR_OK) return st;
   if (out == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL out");
   int32_t max_vis = 0;
+  if (scores_out == nullptr && image_mass_out != nullptr) {      // Eq. 1's ratio alone: the scores go to the context's scratch
+    scores_out = ctx->scores;
+    n_stride = ctx->lim.max_vis_len;
+  }
   if (scores_out != nullptr) {
+    if (ctx->lim.max_vis_len <= 0) return fail(ctx, FASTOCR_ERR_WORKSPACE, "context was created with max_vis_len = 0");
     if ((st = check_scores_args(ctx, kv, scores_out, n_stride)) != FASTOCR_OK) return st;
     max_vis = n_stride < ctx->lim.max_vis_len ? n_stride : ctx->lim.max_vis_len;
-    if (ctx->lim.max_vis_len <= 0) return fail(ctx, FASTOCR_ERR_WORKSPACE, "context was created with max_vis_len = 0");
   }
-  return dense_impl(ctx, kv, q, out, out_is_fp32, scores_out, n_stride, max_vis, fastocr::kWaitAtStart, static_cast<cudaStream_t>(stream));
+  return dense_impl(ctx, kv, q, out, out_is_fp32, scores_out, n_stride, max_vis, fastocr::kWaitAtStart,
+                    static_cast<cudaStream_t>(stream), false, image_mass_out);
 }
 
 fastocr_status fastocr_focal_scores(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, float* scores_out,
                                     int32_t n_stride, float* image_mass_out, void* stream) {
+  NvtxScope range("fastocr_focal_scores");
   fastocr_status st = check_view(ctx, kv, q, false);
   if (st != FASTOCR_OK) return st;
   if ((st = check_scores_args(ctx, kv, scores_out, n_stride)) != FASTOCR_OK) return st;
   if (ctx->lim.max_vis_len <= 0) return fail(ctx, FASTOCR_ERR_WORKSPACE, "context was created with max_vis_len = 0");
   const int32_t max_vis = n_stride < ctx->lim.max_vis_len ? n_stride : ctx->lim.max_vis_len;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  st = dense_impl(ctx, kv, q, nullptr, 0, scores_out, n_stride, max_vis, fastocr::kWaitAtStart, s);
-  if (st != FASTOCR_OK) return st;
-  if (image_mass_out != nullptr) {
-    ProfScope p(ctx, FASTOCR_PROF_MASS, s);
-    FASTOCR_TRY_CUDA(fastocr::launch_image_mass(scores_out, n_stride, kv->vis_len, kv->batch, image_mass_out, s), "image mass launch");
-  }
-  return FASTOCR_OK;
+  return dense_impl(ctx, kv, q, nullptr, 0, scores_out, n_stride, max_vis, fastocr::kWaitAtStart,
+                    static_cast<cudaStream_t>(stream), false, image_mass_out);
 }
 
 fastocr_status fastocr_select_topk(fastocr_ctx* ctx, const float* scores, int32_t n_stride, const int32_t* vis_len,
@@ -444,6 +470,7 @@ fastocr_status fastocr_select_topk(fastocr_ctx* ctx, const float* scores, int32_
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "need batch, n_stride, k_stride > 0 and 0 < max_vis_len <= n_stride");
   if (max_vis_len > fastocr::kTopkMaxN)
     return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "max_vis_len %d exceeds %d", max_vis_len, fastocr::kTopkMaxN);
+  NvtxScope range("fastocr_select_topk");
   ProfScope p(ctx, FASTOCR_PROF_TOPK, static_cast<cudaStream_t>(stream));
   FASTOCR_TRY_CUDA(fastocr::launch_select_topk(scores, n_stride, vis_len, k, batch, max_vis_len, idx_out, k_stride,
                                                nullptr, nullptr, 0, 0, static_cast<cudaStream_t>(stream)),
@@ -458,17 +485,24 @@ fastocr_status fastocr_sparse_decode_attn(fastocr_ctx* ctx, const fastocr_kv_vie
   if (st != FASTOCR_OK) return st;
   if (idx == nullptr || k == nullptr || out == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL idx, k or out");
   if (k_stride <= 0 || max_kept < 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "k_stride must be positive, max_kept non-negative");
+  NvtxScope range("fastocr_sparse_decode_attn");
   return sparse_impl(ctx, kv, q, idx, k, k_stride, max_kept, out, out_is_fp32, fastocr::kWaitAtStart, static_cast<cudaStream_t>(stream));
 }
 
-fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
-                                   const void* q, void* out, int out_is_fp32, const uint8_t* is_focal,
-                                   const int32_t* k, int32_t* fixation, int32_t k_stride, int has_fixation,
-                                   int32_t max_vis_len, int32_t max_kept, int* has_fixation_out, void* stream) {
+fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
+                                      const void* q, void* out, int out_is_fp32, const uint8_t* is_focal,
+                                      const int32_t* k, int32_t* fixation, int32_t k_stride, int has_fixation,
+                                      int32_t max_vis_len, int32_t max_kept, int* has_fixation_out,
+                                      const fastocr_step_options* opt, void* stream) {
   if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
-  if (num_layers <= 0 || layers == nullptr || q == nullptr || out == nullptr || is_focal == nullptr || k == nullptr ||
-      fixation == nullptr)
+  const uint8_t* focal_seq = opt != nullptr ? opt->is_focal_seq : nullptr;           // host [L][B]
+  const uint8_t* focal_seq_dev = opt != nullptr ? opt->is_focal_seq_dev : nullptr;   // the same on the device
+  const bool unite = opt != nullptr && opt->union_sets != 0;
+  if (num_layers <= 0 || layers == nullptr || q == nullptr || out == nullptr || (is_focal == nullptr && focal_seq == nullptr) ||
+      k == nullptr || fixation == nullptr)
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL pointer or num_layers <= 0");
+  if ((focal_seq == nullptr) != (focal_seq_dev == nullptr))
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "per-sequence focal sets need both the host and the device copy of the matrix");
   if (k_stride <= 0 || max_vis_len <= 0 || max_vis_len > ctx->lim.max_vis_len)
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "k_stride / max_vis_len out of range (context max_vis_len %d)", ctx->lim.max_vis_len);
   for (int l = 0; l < num_layers; ++l) {
@@ -478,27 +512,55 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
         layers[l].num_kv_heads != layers[0].num_kv_heads)
       return fail(ctx, FASTOCR_ERR_INVALID_ARG, "layer %d has a different batch / head geometry", l);
   }
+  NvtxScope range("fastocr_decode_step");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int64_t per_layer = static_cast<int64_t>(layers[0].batch) * layers[0].num_q_heads * fastocr::kHeadDim;
+  const int B = layers[0].batch;
+  const int64_t per_layer = static_cast<int64_t>(B) * layers[0].num_q_heads * fastocr::kHeadDim;
   const size_t q_bytes = per_layer * 2, o_bytes = per_layer * (out_is_fp32 ? 4 : 2);
   bool have = has_fixation != 0;
+  // How many sequences treat layer l as a focal layer: all or none with one focal set for the batch;
+  // anything in between with per-sequence sets (Section 3.1.1 profiles C per sample). Layer 0 without
+  // a set from the previous step is the fallback: every sequence attends the full cache and selects.
+  auto focal_count = [&](int l) {
+    if (l == 0 && !have) return B;
+    if (focal_seq == nullptr) return is_focal[l] != 0 ? B : 0;
+    int n = 0;
+    for (int b = 0; b < B; ++b) n += focal_seq[static_cast<size_t>(l) * B + b] != 0;
+    return n;
+  };
   // What the launch issued just before the next one was: nothing of this step yet, a pruned or
   // dense attention kernel of this step (it wrote an output slice and the split workspace, neither
-  // of which the next attention kernel reads), or the selection kernel (it wrote the index set).
+  // of which the next attention kernel reads), the selection kernel (it wrote the index set), or
+  // the union kernel (it wrote an index set and its counts, on which even the set-up depends).
   enum { kOther, kAttention, kSelection } prev = kOther;
+  const bool overlap = !ctx->prof_on || ctx->prof_runs;
+  // The kept image set the pruned layers read: Algorithm 1's `fixation` itself, or, in the union
+  // variant, one of two buffers of the context that the union kernel fills in turn.
+  const int32_t U = ctx->lim.max_vis_len;
+  int cur = 0;
+  auto uni_idx = [&](int i) { return ctx->uni_idx + static_cast<size_t>(i) * ctx->lim.max_batch * U; };
+  auto uni_cnt = [&](int i) { return ctx->uni_cnt + static_cast<size_t>(i) * ctx->lim.max_batch; };
+  if (unite && have) {      // what the previous step left is the kept set until this step's first selection
+    FASTOCR_TRY_CUDA(fastocr::launch_union_sets(nullptr, nullptr, U, fixation, k, k_stride, layers[0].vis_len, max_vis_len, B,
+                                                uni_idx(0), uni_cnt(0), nullptr, 0, 1, 0, s), "kept-set launch");
+  }
   // The pruned layers of a step see the same lengths and kept counts: what every CTA of theirs
   // would work out from those (its range, its unit) is computed once, by a small kernel at the
   // head of the step, and handed to each pruned launch as a plan. Layers whose view differs from
-  // the first pruned layer's in anything the plan depends on simply run without it.
+  // the first pruned layer's in anything the plan depends on simply run without it, and so do
+  // layers that only part of the batch attends pruned, and the union variant (its counts change).
   const fastocr_kv_view* plan_view = nullptr;
   int plan_grid = 0, n_pruned = 0;
-  for (int l = 0; l < num_layers; ++l) {
-    const bool pruned = !(is_focal[l] != 0 || (l == 0 && !have));
-    if (!pruned) continue;
-    if (plan_view == nullptr) plan_view = &layers[l];
-    ++n_pruned;
+  {
+    const bool have0 = have;
+    for (int l = 0; l < num_layers; ++l) {
+      if (focal_count(l) != 0) { have = true; continue; }
+      if (plan_view == nullptr) plan_view = &layers[l];
+      ++n_pruned;
+    }
+    have = have0;
   }
-  if (n_pruned >= 2 && (!ctx->prof_on || ctx->prof_runs)) {
+  if (n_pruned >= 2 && overlap && !unite) {
     AttnLaunch pa = sparse_args(ctx, plan_view, q, fixation, k, k_stride, max_kept);
     if (pa.grid_ctas <= kPlanCtas) {
       plan_grid = pa.grid_ctas;
@@ -510,46 +572,101 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
            v.vis_len == plan_view->vis_len && v.max_seq_len == plan_view->max_seq_len && v.batch == plan_view->batch &&
            v.num_kv_heads == plan_view->num_kv_heads;
   };
+  bool selected_this_step = false, fallback_ran = false;
   for (int l = 0; l < num_layers; ++l) {
     const void* ql = static_cast<const char*>(q) + l * q_bytes;
     void* ol = static_cast<char*>(out) + l * o_bytes;
-    const bool focal = is_focal[l] != 0;
-    const bool chained = prev != kOther && (!ctx->prof_on || ctx->prof_runs);
+    const int n_focal = focal_count(l);
+    const bool fallback = l == 0 && !have;
+    const bool mixed = n_focal != 0 && n_focal != B;
+    const uint8_t* mask = mixed ? focal_seq_dev + static_cast<size_t>(l) * B : nullptr;
     fastocr_status st;
-    if (focal || (l == 0 && !have)) {
-      // full attention + scoring + selection; the refreshed set replaces the current one.
+    if (n_focal != B) {
+      // A pruned layer that follows another attention layer reads nothing the latter wrote (its
+      // queries, index set and cache were complete before), so the two may overlap; right after
+      // a selection only the set-up (lengths, kept counts) may run ahead; after the union kernel
+      // (new counts) nothing may.
+      const bool chained = prev != kOther && overlap;
+      const int wp = !chained ? fastocr::kWaitAtStart : (prev == kAttention ? fastocr::kWaitBeforeWrites : fastocr::kWaitAfterSetup);
+      st = sparse_impl(ctx, &layers[l], ql, unite ? uni_idx(cur) : fixation, unite ? uni_cnt(cur) : k, unite ? U : k_stride,
+                       max_kept, ol, out_is_fp32, wp, s, (!mixed && plan_fits(layers[l])) ? ctx->plan : nullptr, plan_grid, mask, 0);
+      if (st != FASTOCR_OK) return st;
+      prev = kAttention;
+    }
+    if (n_focal != 0) {
+      // Full attention + scoring + selection; the refreshed set replaces the current one.
       // The logits workspace is written from the first block on, and its last reader was the
       // previous selection kernel. Right after that kernel the stream must wait for it; once an
       // attention kernel lies in between, that kernel waited for the selection before it let
       // anything else start, so this launch may stream at once, beside the draining pruned pass.
       // The selection kernel forms the scores from the logits itself (no score array, one launch
       // less) unless there are more heads than it has room for.
+      const bool chained = prev != kOther && overlap;
       const bool fused = layers[l].num_q_heads <= fastocr::kTopkMaxHeads;
       st = dense_impl(ctx, &layers[l], ql, ol, out_is_fp32, fused ? nullptr : ctx->scores, ctx->lim.max_vis_len, max_vis_len,
                       !chained ? fastocr::kWaitAtStart : (prev == kAttention ? fastocr::kWaitBeforeWrites : fastocr::kWaitAfterSetup),
-                      s, fused);
+                      s, fused, nullptr, fallback ? nullptr : mask, 1);
       if (st != FASTOCR_OK) return st;
       {
         ProfScope p(ctx, FASTOCR_PROF_TOPK, s);
-        FASTOCR_TRY_CUDA(fastocr::launch_select_topk(ctx->scores, ctx->lim.max_vis_len, layers[l].vis_len, k, layers[l].batch,
+        FASTOCR_TRY_CUDA(fastocr::launch_select_topk(ctx->scores, ctx->lim.max_vis_len, layers[l].vis_len, k, B,
                                                      max_vis_len, fixation, k_stride, fused ? ctx->logits : nullptr, ctx->stats,
-                                                     layers[l].num_q_heads, ctx->lim.max_vis_len, s),
+                                                     layers[l].num_q_heads, ctx->lim.max_vis_len, s, fallback ? nullptr : mask, 1),
                          "top-k launch");
       }
-      have = true;
       prev = kSelection;
-    } else {
-      // a pruned layer that follows another attention layer reads nothing the latter wrote (its
-      // queries, index set and cache were complete before), so the two may overlap; right after
-      // a selection only the set-up (lengths, kept counts) may run ahead
-      const int wp = !chained ? fastocr::kWaitAtStart : (prev == kAttention ? fastocr::kWaitBeforeWrites : fastocr::kWaitAfterSetup);
-      st = sparse_impl(ctx, &layers[l], ql, fixation, k, k_stride, max_kept, ol, out_is_fp32, wp, s,
-                       plan_fits(layers[l]) ? ctx->plan : nullptr, plan_grid);
-      if (st != FASTOCR_OK) return st;
-      prev = kAttention;
+      if (unite) {
+        // first selection of the step: the set starts afresh; later ones are added to it
+        const int first = (fallback || (focal_seq == nullptr && !selected_this_step)) ? 1 : 0;
+        FASTOCR_TRY_CUDA(fastocr::launch_union_sets(uni_idx(cur), uni_cnt(cur), U, fixation, k, k_stride, layers[l].vis_len,
+                                                    max_vis_len, B, uni_idx(cur ^ 1), uni_cnt(cur ^ 1),
+                                                    fallback ? nullptr : focal_seq_dev, l, first, fallback_ran ? 1 : 0, s),
+                         "kept-set launch");
+        cur ^= 1;
+        prev = kOther;
+      }
+      if (fallback) fallback_ran = true;
+      selected_this_step = true;
+      have = true;
     }
   }
   if (has_fixation_out != nullptr) *has_fixation_out = have ? 1 : 0;
+  return FASTOCR_OK;
+}
+
+fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
+                                   const void* q, void* out, int out_is_fp32, const uint8_t* is_focal,
+                                   const int32_t* k, int32_t* fixation, int32_t k_stride, int has_fixation,
+                                   int32_t max_vis_len, int32_t max_kept, int* has_fixation_out, void* stream) {
+  return fastocr_decode_step_ex(ctx, num_layers, layers, q, out, out_is_fp32, is_focal, k, fixation, k_stride, has_fixation,
+                                max_vis_len, max_kept, has_fixation_out, nullptr, stream);
+}
+
+fastocr_status fastocr_warmup_step(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers, const void* q,
+                                   void* out, int out_is_fp32, float* ratio_out, void* stream) {
+  if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
+  if (num_layers <= 0 || layers == nullptr || q == nullptr || out == nullptr || ratio_out == nullptr)
+    return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL pointer or num_layers <= 0");
+  if (ctx->lim.max_vis_len <= 0) return fail(ctx, FASTOCR_ERR_WORKSPACE, "context was created with max_vis_len = 0");
+  for (int l = 0; l < num_layers; ++l) {
+    fastocr_status st = check_view(ctx, &layers[l], q, true);
+    if (st != FASTOCR_OK) return st;
+    if (layers[l].batch != layers[0].batch || layers[l].num_q_heads != layers[0].num_q_heads)
+      return fail(ctx, FASTOCR_ERR_INVALID_ARG, "layer %d has a different batch / head geometry", l);
+  }
+  NvtxScope range("fastocr_warmup_step");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int B = layers[0].batch;
+  const int64_t per_layer = static_cast<int64_t>(B) * layers[0].num_q_heads * fastocr::kHeadDim;
+  const size_t q_bytes = per_layer * 2, o_bytes = per_layer * (out_is_fp32 ? 4 : 2);
+  for (int l = 0; l < num_layers; ++l) {
+    // one pass over K and V: the layer's output, and from the same logits the head-averaged image
+    // attention whose sum over the image span is Eq. 1's ratio
+    fastocr_status st = dense_impl(ctx, &layers[l], static_cast<const char*>(q) + l * q_bytes, static_cast<char*>(out) + l * o_bytes,
+                                   out_is_fp32, ctx->scores, ctx->lim.max_vis_len, ctx->lim.max_vis_len, fastocr::kWaitAtStart, s,
+                                   false, ratio_out + static_cast<size_t>(l) * B);
+    if (st != FASTOCR_OK) return st;
+  }
   return FASTOCR_OK;
 }
 
@@ -580,6 +697,13 @@ int32_t fastocr_focal_layers(const double* mean_ratio, int32_t num_layers, doubl
 
 double fastocr_attn_flops(double batch, double layers, double hidden, double seq_len) {
   return batch * layers * (8.0 * hidden * hidden + 4.0 * hidden * seq_len);
+}
+
+double fastocr_attn_flops_pruned(double batch, double layers, double hidden, double seq_len, double full_layers,
+                                 double kept_len) {
+  const double proj = 8.0 * hidden * hidden * layers;                    // every layer projects the new token
+  const double attend = 4.0 * hidden * (full_layers * seq_len + (layers - full_layers) * kept_len);
+  return batch * (proj + attend);
 }
 
 fastocr_status fastocr_profile_begin(fastocr_ctx* ctx, int32_t max_launches, int coalesce_runs) {

@@ -80,3 +80,26 @@ def make_case(seed, spans, H=28, Hkv=4, page_size=0, grid_w=None, boost=2.0) -> 
     if page_size:
         case.block_table, case.num_pages = make_page_table(seed, seq_len, page_size, spare_pages=3)
     return case
+
+
+def make_layer_stack(seed, spans, L, H=28, Hkv=4, page_size=0, q_boost=1.0):
+    """L layers over one batch geometry: per-layer K, V and queries (all seeded), the views sharing one
+    set of length arrays as a caller's would. -> (cases per layer, views per layer, q [L][B][H][128] CPU)."""
+    from paper_2605_17447_b200 import KVView
+    from workloads import normal_bf16, stream_key
+    base = make_case(seed, spans, H=H, Hkv=Hkv, page_size=page_size)
+    cases, views, shared = [], [], None
+    for l in range(L):
+        K, V = make_kv(seed, l, base.B, max(base.seq_len), Hkv, 128)
+        q = normal_bf16(stream_key(seed, 55, l), (base.B, H, 128))
+        if q_boost != 1.0:
+            q = (q.float() * q_boost).to(torch.bfloat16)
+        c = Case(base.B, H, Hkv, base.seq_len, base.vis_start, base.vis_len, K, V, q, base.page_size,
+                 base.block_table, base.num_pages)
+        cases.append(c)
+        v = c.device_view()
+        if shared is None:
+            shared = (v.seq_len, v.vis_start, v.vis_len)
+        views.append(KVView(v.k, v.v, shared[0], shared[1], shared[2], H, max(base.seq_len), SCALE,
+                            block_table=v.block_table if page_size else None))
+    return cases, views, torch.stack([c.q for c in cases])

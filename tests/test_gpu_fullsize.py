@@ -76,3 +76,150 @@ def test_full_size_layer_chain_against_oracle_on_sampled_sequences():
             err = (got.cpu() - ref).abs()
             assert err.max() <= 1e-4 and err.mean() <= 1e-3
     ctx.close()
+
+
+def _step_inputs(cfg, L, dev, n_caches=None, steps=2, paged=False):
+    """Device-resident decode state of a workload config for `steps` consecutive steps over L layers
+    (n_caches distinct caches cycled over the layers, every layer with its own queries)."""
+    import paper_2605_17447_b200 as fo
+    from workloads import fixation_track, make_kv, make_page_table, make_queries, scatter_to_pages
+    B, H, Hkv = cfg.batch, cfg.num_q_heads, cfg.num_kv_heads
+    n_caches = n_caches or L
+    S0 = cfg.seq_len(0)
+    stride = max(S0) + steps
+    i32 = lambda x: torch.tensor(x, dtype=torch.int32, device=dev)
+    vs = i32(cfg.vis_start)
+    tracks = np.stack([fixation_track(cfg.seed, b, steps, cfg.grid_h[b], cfg.grid_w[b], cfg.advance) for b in range(B)])
+    gh, gw = torch.tensor(cfg.grid_h, device=dev), torch.tensor(cfg.grid_w, device=dev)
+    table = None
+    if paged:
+        table, num_pages = make_page_table(cfg.seed, [stride] * B, cfg.page_size)
+    caches = []
+    for c in range(n_caches):
+        K, V = make_kv(cfg.seed, c, B, stride, Hkv, 128, dev)
+        caches.append((K, V))
+    q = torch.empty(steps, L, B, H, 128, dtype=torch.bfloat16, device=dev)
+    for l in range(L):
+        K = caches[l % n_caches][0]
+        for s in range(steps):
+            q[s, l] = make_queries(cfg.seed, l, s, lambda b, pos: K[b, pos], vs.long(), torch.tensor(tracks[:, s, :], device=dev),
+                                   gh, gw, H)
+    seq_len = i32([s + 1 for s in S0])
+    views = []
+    for l in range(L):
+        K, V = caches[l % n_caches]
+        if paged:
+            Kp = scatter_to_pages(K, [stride] * B, table, num_pages, cfg.page_size)
+            Vp = scatter_to_pages(V, [stride] * B, table, num_pages, cfg.page_size)
+            views.append(fo.KVView(Kp, Vp, seq_len, vs, i32(cfg.vis_len), H, stride, SCALE, block_table=table.to(dev)))
+        else:
+            views.append(fo.KVView(K, V, seq_len, vs, i32(cfg.vis_len), H, stride, SCALE))
+    return caches, views, q, seq_len, S0
+
+
+def _check_step_against_oracle(cfg, L, focal, n_caches, paged, sample, steps=2):
+    """Runs `steps` decode steps of the configuration through fastocr_decode_step (all launches chained as
+    in a timed step) and compares the sampled sequences, every layer, and the carried set with
+    Algorithm 1 run by the oracle on the same bytes."""
+    import paper_2605_17447_b200 as fo
+    dev = "cuda"
+    B, H, Hkv = cfg.batch, cfg.num_q_heads, cfg.num_kv_heads
+    caches, views, q, seq_len, S0 = _step_inputs(cfg, L, dev, n_caches, steps, paged)
+    ks = [fo.kept_count(n, cfg.tau) for n in cfg.vis_len]
+    kd = torch.tensor(ks, dtype=torch.int32, device=dev)
+    ctx = fo.Context(B, H, Hkv, max(S0) + steps, max(cfg.vis_len))
+    fix = torch.full((B, max(ks)), -1, dtype=torch.int32, device=dev)
+    is_focal = [l in focal for l in range(L)]
+    max_kept = max(k + s - n for k, s, n in zip(ks, S0, cfg.vis_len)) + steps
+    plan = fo.StepPlan(ctx, views, is_focal, kd, fix, max(cfg.vis_len), max_kept)
+    have, f_last = False, {b: None for b in sample}
+    for s in range(steps):
+        seq_len.copy_(torch.tensor([x + s + 1 for x in S0], dtype=torch.int32))
+        out = torch.full((L, B, H, 128), 7.0, dtype=torch.float32, device=dev)
+        have = plan.run(q[s], out, have)
+        torch.cuda.synchronize()
+        assert have
+        for b in sample:
+            S = S0[b] + s + 1
+            layers = [(q[s, l, b].cpu(), caches[l % n_caches][0][b, :S].cpu(), caches[l % n_caches][1][b, :S].cpu()) for l in range(L)]
+            tr = oracle.decode_step(layers, focal, f_last[b], cfg.vis_start[b], cfg.vis_len[b], cfg.tau, SCALE, acc64=True)
+            # selections may differ from the oracle's only at near-ties of the oracle's scores
+            got = fix[b, :ks[b]].cpu()
+            if got.tolist() != tr.f_last.tolist():
+                deepest = max(focal) if focal else 0
+                ref_sc, _ = oracle.scores(*layers[deepest][:2], SCALE, cfg.vis_start[b], cfg.vis_len[b], True)
+                kth = float(torch.sort(ref_sc, descending=True).values[ks[b] - 1])
+                assert all(abs(float(ref_sc[i]) - kth) <= 1e-5 * kth for i in set(got.tolist()) ^ set(tr.f_last.tolist()))
+                tr = None                                 # outputs downstream of a near-tie are checked on the next sample
+            if tr is not None:
+                for l in range(L):
+                    err = (out[l, b].cpu() - tr.outputs[l]).abs()
+                    assert err.max() <= 1e-4 and err.mean() <= 1e-3, (s, b, l, float(err.max()))
+                f_last[b] = tr.f_last
+            else:
+                f_last[b] = got
+    assert ctx.device_faults() == 0
+    ctx.close()
+
+
+def test_72b_shaped_step_against_oracle():
+    """Config 3's head geometry and span (64 query / 8 KV heads, N = 16384, B = 8): a focal layer between
+    pruned layers, selection from 64 heads' logits on clusters of CTAs, pruned passes of 1332 tokens."""
+    from workloads import get_config
+    cfg = get_config("cfg3")
+    _check_step_against_oracle(cfg, L=5, focal=[2], n_caches=3, paged=False, sample=(0, 5))
+
+
+def test_paged_ragged_serving_step_against_oracle():
+    """Config 2's batch (32 ragged sequences of 4096-8192 image tokens, 16-token pages, shuffled page
+    table): 128 units, one CTA per unit in the pruned passes."""
+    from workloads import get_config
+    cfg = get_config("cfg2")
+    _check_step_against_oracle(cfg, L=4, focal=[1], n_caches=2, paged=True, sample=(0, 13, 31))
+
+
+def test_28_layer_step_in_the_timed_configuration_against_oracle():
+    """The benchmark's default step as it is timed: batch 64, N = 8192, 28 layers with focal layers 13 and
+    18, launches overlapping (a full-cache pass starting beside a draining pruned pass, two selections
+    per step), two consecutive steps so that the second starts from a carried set."""
+    from workloads import get_config
+    cfg = get_config("cfg4", N=8192, batch=64)
+    _check_step_against_oracle(cfg, L=28, focal=[13, 18], n_caches=4, paged=False, sample=(0, 41, 63))
+
+
+def test_more_units_than_ctas():
+    """80 sequences x 4 KV heads = 320 units against 296 pruned-pass CTAs: ranges of rows that straddle
+    units, partial results merged through global memory. Every sequence against the oracle."""
+    import paper_2605_17447_b200 as fo
+    import sys, os
+    sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+    from harness import make_case
+    g = torch.Generator().manual_seed(77)
+    ri = lambda lo, hi: int(torch.randint(lo, hi + 1, (1,), generator=g))
+    spans = [(ri(0, 30), ri(200, 900), ri(0, 90)) for _ in range(80)]
+    case = make_case(2100, spans)
+    kv = case.device_view(poison=True)
+    ks = [oracle.kept_count(n, 0.1) for n in case.vis_len]
+    idx = torch.zeros(80, max(ks), dtype=torch.int32)
+    for b in range(80):
+        idx[b, :ks[b]] = torch.randperm(case.vis_len[b], generator=g)[:ks[b]].sort().values.int()
+    ctx = fo.Context(80, 28, 4, max(case.seq_len), max(case.vis_len))
+    out = torch.full((80, 28, 128), 7.0, dtype=torch.float32, device="cuda")
+    dense = torch.full((80, 28, 128), 7.0, dtype=torch.float32, device="cuda")
+    q = case.q.cuda()
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    fo.fastocr_sparse_decode_attn(ctx, kv, q, idx.cuda(), kd, out, max_kept=max(k + s - n for k, s, n in zip(ks, case.seq_len, case.vis_len)))
+    fo.fastocr_dense_decode_attn(ctx, kv, q, dense)
+    out3 = torch.full((3, 80, 28, 128), 7.0, dtype=torch.float32, device="cuda")
+    fo.fastocr_decode_step(ctx, [kv, kv, kv], torch.stack([q, q, q]), out3, [False] * 3, kd, idx.cuda().clone(), True, max(case.vis_len))
+    torch.cuda.synchronize()
+    for b in range(80):
+        ref = oracle.sparse(*case.seq(b), SCALE, case.vis_start[b], case.vis_len[b], idx[b, :ks[b]], True)
+        err = (out[b].cpu() - ref).abs()
+        assert err.max() <= 1e-4 and err.mean() <= 1e-3, b
+        err = (dense[b].cpu() - oracle.dense(*case.seq(b), SCALE, True)).abs()
+        assert err.max() <= 1e-4 and err.mean() <= 1e-3, b
+    for l in range(3):
+        assert torch.equal(out3[l], out)
+    assert ctx.device_faults() == 0
+    ctx.close()

@@ -13,6 +13,11 @@ from harness import SCALE, make_case
 
 pytestmark = pytest.mark.gpu
 
+# FASTOCR_CLUSTER_MAX_ROWS=0 (a tuning knob read when a context is created) turns the merge inside
+# thread-block clusters off; the tests that assert which path ran follow the knob.
+import os
+CLUSTERS_ON = int(os.environ.get("FASTOCR_CLUSTER_MAX_ROWS", "6")) > 0
+
 MAX_ABS, MEAN_ABS = 1e-2, 1e-3      # stated tolerance for bf16 K/V/Q against the fp32 oracle
 TIGHT = 1e-4                        # what fp32 accumulation on both sides actually delivers
 
@@ -69,7 +74,7 @@ def test_dense_and_fused_scores_match_oracle(fo, ctx, shape, paged):
     # a single sequence leaves most SMs empty anyway: each (sequence, KV head) unit is then one cluster of
     # 16 CTAs and merges inside it (some units have fewer than 16 rows: CTAs without work in the cluster)
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    assert fo.cluster_launch_count() == before + (1 if 2 * 16 * case.B * case.Hkv <= sms else 0)
+    assert fo.cluster_launch_count() == before + (1 if CLUSTERS_ON and 2 * 16 * case.B * case.Hkv <= sms else 0)
     _check_out(out, _oracle_dense(case))
     # fp32-accumulating oracle too (the stated reference)
     err32 = (out.cpu() - _oracle_dense(case, acc64=False)).abs()
@@ -200,14 +205,14 @@ def test_sparse_cluster_merge_matches_oracle(fo, ctx, case_no, paged):
     out = torch.full((case.B, case.H, 128), 7.0, dtype=torch.float32, device="cuda")
     before = fo.cluster_launch_count()
     fo.fastocr_sparse_decode_attn(ctx, kv, q, idx.cuda(), kd, out, max_kept=max_kept)
-    assert fo.cluster_launch_count() == before + 1       # the path under test is the one that ran
+    assert fo.cluster_launch_count() == before + (1 if CLUSTERS_ON else 0)       # the path under test is the one that ran
     _check_out(out, ref)
     # the same inside a decode step (launch plan in use), three pruned layers on last step's set
     out3 = torch.full((3, case.B, case.H, 128), 7.0, dtype=torch.float32, device="cuda")
     before = fo.cluster_launch_count()
     assert fo.fastocr_decode_step(ctx, [kv, kv, kv], torch.stack([q, q, q]), out3, [False, False, False], kd,
                                   idx.cuda().clone(), True, max(case.vis_len), max_kept=max_kept)
-    assert fo.cluster_launch_count() == before + 3
+    assert fo.cluster_launch_count() == before + (3 if CLUSTERS_ON else 0)
     for l in range(3):
         assert torch.equal(out3[l], out)
 

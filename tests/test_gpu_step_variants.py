@@ -1,0 +1,251 @@
+"""GPU parity of the step-level entry points beyond Algorithm 1's plain post-warm-up step: the warm-up
+step (profiling block), per-sequence focal layer sets, the union-of-selections variant, the 64-head
+shape inside a decode step, and what the kernels do with device-side lengths, index-list entries and
+page ids that lie outside what the host checked. Everything goes through the C ABI and is compared
+with the CPU oracle element by element."""
+import math
+
+import pytest
+import torch
+
+import oracle
+from harness import SCALE, make_case, make_layer_stack
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS, TIGHT = 1e-2, 1e-3, 1e-4
+
+
+@pytest.fixture(scope="module")
+def fo():
+    import paper_2605_17447_b200 as f
+    return f
+
+
+@pytest.fixture(scope="module")
+def ctx(fo):
+    c = fo.Context(max_batch=8, num_q_heads=64, num_kv_heads=8, max_seq_len=8192, max_vis_len=6000)
+    yield c
+    c.close()
+
+
+def _check_out(got, ref):
+    err = (got.float().cpu() - ref).abs()
+    assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS
+    assert err.max() <= TIGHT, float(err.max())
+
+
+def test_warmup_step_records_eq1_and_keeps_dense_outputs(fo, ctx):
+    """Algorithm 1's profiling block: w steps, every layer dense, r per layer and sequence from the same
+    pass; the focal layer sets that follow (per sequence) equal the oracle's."""
+    L, w = 4, 3
+    spans = [(6, 300, 20), (3, 170, 41), (9, 512, 7)]
+    ratios_gpu = torch.zeros(w, L, len(spans), dtype=torch.float32)
+    ratios_ref = torch.zeros(w, L, len(spans), dtype=torch.float64)
+    for t in range(w):
+        cases, views, q_all = make_layer_stack(1300 + t, spans, L)
+        out = torch.empty(L, len(spans), 28, 128, dtype=torch.float32, device="cuda")
+        r = torch.full((L, len(spans)), -1.0, dtype=torch.float32, device="cuda")
+        fo.fastocr_warmup_step(ctx, views, q_all.cuda(), out, r)
+        ratios_gpu[t] = r.cpu()
+        for b in range(len(spans)):
+            outs, rr = oracle.warmup_step([c.seq(b) for c in cases], cases[0].vis_start[b], cases[0].vis_len[b], SCALE, acc64=True)
+            for l in range(L):
+                _check_out(out[l, b], outs[l])
+                ratios_ref[t, l, b] = rr[l]
+    assert float((ratios_gpu.double() - ratios_ref).abs().max()) <= 1e-5
+    for b in range(len(spans)):
+        mean_gpu = ratios_gpu[:, :, b].double().mean(dim=0).tolist()
+        assert fo.focal_layers(mean_gpu, 0.5, 1) == oracle.profile_focal_layers(ratios_ref[:, :, b].tolist(), 0.5, 1)
+    # the single-layer call gives the same ratio with or without the score array
+    cases, views, q_all = make_layer_stack(1300, spans, 1)
+    out = torch.empty(len(spans), 28, 128, dtype=torch.float32, device="cuda")
+    sc = torch.zeros(len(spans), 512, dtype=torch.float32, device="cuda")
+    m1 = torch.zeros(len(spans), dtype=torch.float32, device="cuda")
+    m2 = torch.zeros_like(m1)
+    fo.fastocr_dense_decode_attn(ctx, views[0], q_all[0].cuda(), out, image_mass_out=m1)
+    fo.fastocr_dense_decode_attn(ctx, views[0], q_all[0].cuda(), out, scores_out=sc, image_mass_out=m2)
+    assert torch.equal(m1, m2) and torch.equal(m1.cpu(), ratios_gpu[0, 0])
+    assert ctx.device_faults() == 0
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_decode_step_with_per_sequence_focal_sets(fo, ctx, paged):
+    """Each sequence has its own focal layer set (the paper profiles C per sample): a layer that is focal
+    for part of the batch runs as two masked launches. Two consecutive steps, every sequence against
+    the oracle run with that sequence's own set."""
+    L = 6
+    spans = [(6, 300, 20), (3, 170, 41), (5, 222, 9), (2, 260, 30)]
+    focal_of = [[2], [1, 3], [], [0, 3]]                      # layer 3 mixed 2:2, layer 0 focal for one sequence only
+    matrix = [[l in focal_of[b] for b in range(len(spans))] for l in range(L)]
+    cases, views, q_all = make_layer_stack(1400, spans, L, page_size=16 if paged else 0)
+    base = cases[0]
+    ks = [oracle.kept_count(n, 0.1) for n in base.vis_len]
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    fix = torch.full((base.B, max(ks)), -1, dtype=torch.int32, device="cuda")
+    have, f_last = False, [None] * base.B
+    for step in range(2):
+        out = torch.full((L, base.B, base.H, 128), 7.0, dtype=torch.float32, device="cuda")
+        have = fo.fastocr_decode_step(ctx, views, q_all.cuda(), out, matrix, kd, fix, have, max(base.vis_len))
+        assert have
+        for b in range(base.B):
+            tr = oracle.decode_step([c.seq(b) for c in cases], focal_of[b], f_last[b], base.vis_start[b], base.vis_len[b],
+                                    0.1, SCALE, acc64=True)
+            for l in range(L):
+                _check_out(out[l, b], tr.outputs[l])
+            assert fix[b, :ks[b]].cpu().tolist() == tr.f_last.tolist()
+            f_last[b] = tr.f_last
+    assert ctx.device_faults() == 0
+
+
+@pytest.mark.parametrize("per_seq", [False, True])
+def test_decode_step_union_of_selections(fo, ctx, per_seq):
+    """The union variant: after a focal layer the kept image set is the union of this step's selections;
+    the set carried to the next step stays the deepest focal layer's own."""
+    L = 6
+    spans = [(6, 300, 20), (3, 170, 41), (4, 280, 11)]
+    focal_of = [[1, 3, 4], [2, 4], [1]] if per_seq else [[1, 3, 4]] * 3
+    is_focal = [[l in focal_of[b] for b in range(3)] for l in range(L)] if per_seq else [l in focal_of[0] for l in range(L)]
+    cases, views, q_all = make_layer_stack(1500, spans, L, q_boost=2.0)
+    base = cases[0]
+    ks = [oracle.kept_count(n, 0.1) for n in base.vis_len]
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    fix = torch.full((base.B, max(ks)), -1, dtype=torch.int32, device="cuda")
+    have, f_last = False, [None] * base.B
+    grew = False
+    for step in range(2):
+        out = torch.full((L, base.B, base.H, 128), 7.0, dtype=torch.float32, device="cuda")
+        have = fo.fastocr_decode_step(ctx, views, q_all.cuda(), out, is_focal, kd, fix, have, max(base.vis_len),
+                                      max_kept=max(3 * k + s - n for k, s, n in zip(ks, base.seq_len, base.vis_len)), union_sets=True)
+        for b in range(base.B):
+            tr = oracle.decode_step([c.seq(b) for c in cases], focal_of[b], f_last[b], base.vis_start[b], base.vis_len[b],
+                                    0.1, SCALE, acc64=True, union_sets=True)
+            for l in range(L):
+                _check_out(out[l, b], tr.outputs[l])
+            assert fix[b, :ks[b]].cpu().tolist() == tr.f_last.tolist()
+            f_last[b] = tr.f_last
+            grew = grew or any(u is not None and len(u) > ks[b] for u in tr.used_set)
+    assert grew                                                 # the union really was larger than one selection somewhere
+    assert ctx.device_faults() == 0
+
+
+@pytest.mark.parametrize("spans", [[(5, 700, 9), (1, 640, 3)], [(16, 5000, 40), (16, 4800, 56)]])
+def test_decode_step_with_64_query_heads(fo, ctx, spans):
+    """The 72B-shaped head geometry (64 query / 8 KV heads) through the whole step: the selection kernel
+    forms the scores from 64 heads' logits (one token per thread for the short spans, four tokens per
+    thread and clusters of CTAs for the long ones)."""
+    L = 4
+    cases, views, q_all = make_layer_stack(1600, spans, L, H=64, Hkv=8, q_boost=1.5)
+    base = cases[0]
+    ks = [oracle.kept_count(n, 0.05) for n in base.vis_len]
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    fix = torch.full((base.B, max(ks)), -1, dtype=torch.int32, device="cuda")
+    have, f_last = False, [None] * base.B
+    for step in range(2):
+        out = torch.empty(L, base.B, 64, 128, dtype=torch.float32, device="cuda")
+        have = fo.fastocr_decode_step(ctx, views, q_all.cuda(), out, [False, True, False, False], kd, fix, have, max(base.vis_len))
+        for b in range(base.B):
+            tr = oracle.decode_step([c.seq(b) for c in cases], [1], f_last[b], base.vis_start[b], base.vis_len[b], 0.05, SCALE, acc64=True)
+            for l in range(L):
+                _check_out(out[l, b], tr.outputs[l])
+            assert fix[b, :ks[b]].cpu().tolist() == tr.f_last.tolist()
+            f_last[b] = tr.f_last
+    assert ctx.device_faults() == 0
+
+
+def test_kept_count_beyond_the_index_rows_uses_the_row(fo, ctx):
+    """k[b] larger than the index list's row length: the first k_stride entries are the set (nothing past
+    the row is read), which is not a fault."""
+    case = make_case(1700, [(4, 200, 10), (3, 90, 5)])
+    kv = case.device_view()
+    g = torch.Generator().manual_seed(3)
+    k_stride = 12
+    idx = torch.stack([torch.randperm(n, generator=g)[:k_stride].sort().values.int() for n in case.vis_len])
+    # the buffer really ends after the rows: a read past them would meet the guard values placed behind
+    flat = torch.full((2 * k_stride + 64,), 10 ** 6, dtype=torch.int32)
+    flat[:2 * k_stride] = idx.flatten()
+    dev = flat.cuda()
+    out = torch.empty(2, 28, 128, dtype=torch.float32, device="cuda")
+    fo.fastocr_sparse_decode_attn(ctx, kv, case.q.cuda(), dev[:2 * k_stride].view(2, k_stride),
+                                  torch.tensor([40, 9999], dtype=torch.int32, device="cuda"), out)
+    ref = torch.stack([oracle.sparse(*case.seq(b), SCALE, case.vis_start[b], case.vis_len[b], idx[b], True) for b in range(2)])
+    _check_out(out, ref)
+    assert ctx.device_faults() == 0
+
+
+def test_device_side_lengths_are_forced_into_range_and_counted(fo, ctx):
+    """seq_len / vis_start / vis_len live in device memory, where the host cannot check them. Values outside
+    what the host did check are forced into range and counted; the other sequences are unaffected. The
+    caches are over-allocated, so that even the unclamped reads would have stayed inside the buffers."""
+    case = make_case(1800, [(4, 200, 10), (3, 90, 5), (6, 150, 8)])
+    kv = case.device_view(extra_stride=4096)                    # rows far beyond max_seq_len exist (zeros)
+    q = case.q.cuda()
+    good = torch.stack([oracle.dense(*case.seq(b), SCALE, True) for b in range(3)])
+    out = torch.empty(3, 28, 128, dtype=torch.float32, device="cuda")
+    i32 = lambda x: torch.tensor(x, dtype=torch.int32, device="cuda")
+    assert ctx.device_faults() == 0
+    for bad_seq_len, bad_start, bad_len, want in (
+            ([214, 98 + 3000, 164], None, None, 1),             # longer than max_seq_len
+            ([214, -5, 164], None, None, 3),                    # negative: the span no longer fits either
+            (None, [4, -7, 6], None, 1),                        # span starts before the sequence
+            (None, None, [200, 5000, 150], 1),                  # span longer than the sequence
+            ([10 ** 9, 98, -3], [4, 3, 99999], None, 4)):       # several at once
+        view = case.device_view(extra_stride=4096)
+        view.max_seq_len = kv.max_seq_len
+        if bad_seq_len:
+            view.seq_len = i32(bad_seq_len)
+        if bad_start:
+            view.vis_start = i32(bad_start)
+        if bad_len:
+            view.vis_len = i32(bad_len)
+        out.fill_(7.0)
+        fo.fastocr_dense_decode_attn(ctx, view, q, out)
+        torch.cuda.synchronize()
+        assert ctx.device_faults() == want
+        ok = [b for b in range(3) if (not bad_seq_len or bad_seq_len[b] == case.seq_len[b])
+              and (not bad_start or bad_start[b] == case.vis_start[b]) and (not bad_len or bad_len[b] == case.vis_len[b])]
+        for b in ok:
+            _check_out(out[b], good[b])
+        assert bool(torch.isfinite(out).all())
+    # pruned pass and selection with the same kind of input
+    ks = [10, 5, 8]
+    g = torch.Generator().manual_seed(1)
+    idx = torch.zeros(3, 10, dtype=torch.int32)
+    for b in range(3):
+        idx[b, :ks[b]] = torch.randperm(case.vis_len[b], generator=g)[:ks[b]].sort().values.int()
+    view = case.device_view(extra_stride=4096)
+    view.max_seq_len = kv.max_seq_len
+    view.seq_len = i32([214, 98 + 3000, 164])
+    fo.fastocr_sparse_decode_attn(ctx, view, q, idx.cuda(), i32(ks), out)
+    torch.cuda.synchronize()
+    assert ctx.device_faults() == 1
+    for b in (0, 2):
+        _check_out(out[b], oracle.sparse(*case.seq(b), SCALE, case.vis_start[b], case.vis_len[b], idx[b, :ks[b]], True))
+    sel = torch.full((3, 10), -1, dtype=torch.int32, device="cuda")
+    sc = torch.rand(3, 256, generator=g)
+    fo.fastocr_select_topk(ctx, sc.cuda(), i32([200, -4, 150]), i32(ks), sel, 256)   # a negative length selects nothing
+    torch.cuda.synchronize()
+    assert sel[1].tolist() == [-1] * 10
+    for b in (0, 2):
+        assert sel[b, :ks[b]].cpu().tolist() == oracle.topk(sc[b, :case.vis_len[b]], ks[b]).tolist()
+
+
+def test_page_ids_outside_the_pool_are_clamped_and_counted(fo, ctx):
+    """A block-table entry beyond num_pages is forced into the pool and counted. The pools hold more pages
+    than the view declares, so the unclamped read would have stayed inside the allocation too."""
+    case = make_case(1900, [(4, 200, 10), (3, 90, 5)], page_size=16)
+    kv = case.device_view()
+    q = case.q.cuda()
+    declared = kv.k.shape[0]
+    spare = torch.zeros(64, 16, 4, 128, dtype=torch.bfloat16, device="cuda")
+    bad = fo.KVView(torch.cat([kv.k, spare]), torch.cat([kv.v, spare]), kv.seq_len, kv.vis_start, kv.vis_len, 28,
+                    kv.max_seq_len, SCALE, block_table=kv.block_table.clone(), num_pages=declared)
+    bad.block_table[1, 2] = declared + 40                        # inside the allocation, outside the declared pool
+    bad.block_table[1, 3] = -9
+    out = torch.empty(2, 28, 128, dtype=torch.float32, device="cuda")
+    assert ctx.device_faults() == 0
+    fo.fastocr_dense_decode_attn(ctx, bad, q, out)
+    torch.cuda.synchronize()
+    assert ctx.device_faults() == 2 * 16 * 4                     # two pages x 16 tokens, looked up once by each of the 4 KV heads' units
+    _check_out(out[0], oracle.dense(*case.seq(0), SCALE, True))
+    assert bool(torch.isfinite(out).all())

@@ -4,7 +4,7 @@ last on purpose: a run that stops at the first failure has then already run ever
 import pytest
 import torch
 
-from harness import make_case
+from harness import SCALE, make_case
 
 pytestmark = pytest.mark.gpu
 
@@ -39,7 +39,27 @@ def test_noalloc_matches_context_entry_point_twice_in_a_row():
             assert torch.cuda.mem_get_info()[0] >= free_before
         err = (got - ref).abs()
         assert err.max() <= 1e-4 and err.mean() <= 1e-3, float(err.max())     # same tolerance as the parity tests
+        # and against the oracle itself, not only against the library's other entry point
+        import oracle
+        idx_c, ks = idx.cpu(), kd.cpu().tolist()
+        want = torch.stack([oracle.sparse(*case.seq(b), SCALE, case.vis_start[b], case.vis_len[b], idx_c[b, :ks[b]], True)
+                            for b in range(case.B)])
+        err = (got.cpu() - want).abs()
+        assert err.max() <= 1e-4 and err.mean() <= 1e-3, float(err.max())
+    assert fo.noalloc_device_faults() == 0
     ctx.close()
+
+
+def test_noalloc_reports_values_it_had_to_force_into_range():
+    """A caller without a context can still learn that its device-side inputs were out of range."""
+    import paper_2605_17447_b200 as fo
+    case, kv, q, idx, kd = _inputs(904, [(4, 64, 4), (3, 90, 5)], False)
+    idx[1, 0] = 5000                                                 # outside the image span: clamped and counted
+    out = torch.empty(case.B, case.H, 128, dtype=torch.float32, device="cuda")
+    fo.noalloc_device_faults()
+    fo.fastocr_sparse_decode_attn_noalloc(kv, q, idx, kd, out)
+    assert fo.noalloc_device_faults() == 4                           # one entry, met by each of the 4 KV heads' units
+    assert fo.noalloc_device_faults() == 0 and bool(torch.isfinite(out).all())
 
 
 def test_noalloc_rejects_oversized_batches():
