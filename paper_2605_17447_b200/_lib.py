@@ -6,7 +6,8 @@ import ctypes as C
 import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libfastocr.so")
+# FASTOCR_LIB: development knob, another build of the same library (a debug or experimental variant)
+LIB_PATH = os.environ.get("FASTOCR_LIB") or os.path.join(HERE, "libfastocr.so")
 
 
 class KVViewStruct(C.Structure):

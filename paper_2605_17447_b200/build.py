@@ -31,7 +31,8 @@ def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str |
     tag = "" if out is None else "." + os.path.basename(out).replace(".so", "")
     if verbose:
         flags += ["-Xptxas", "-v"]
-    objs = [os.path.join(CSRC, src.replace(".cu", tag + ".o")) for src in SOURCES]
+    obj_dir = CSRC if out is None else os.path.dirname(os.path.abspath(out))      # a variant's objects stay beside the variant
+    objs = [os.path.join(obj_dir, src.replace(".cu", tag + ".o")) for src in SOURCES]
     procs = [subprocess.Popen([nvcc, *flags, "-c", os.path.join(CSRC, src), "-o", obj]) for src, obj in zip(SOURCES, objs)]
     failed = [src for src, p in zip(SOURCES, procs) if p.wait() != 0]      # the files compile side by side
     if failed:

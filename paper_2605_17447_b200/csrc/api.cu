@@ -50,6 +50,11 @@ struct fastocr_ctx {
   // kernel). Such launches are latency-bound and gain 5-60 %; with more rows per CTA the GPU is full,
   // clusters are harder to place and hold their slots until the slowest CTA is done: 8-13 % slower.
   int cluster_max_rows = 6;
+  // Consecutive pruned layers of a decode step that share their lengths and index set run as one launch
+  // (up to kMaxGroupLayers of them): its persistent CTAs stream through equal ranges of all those
+  // layers' rows, so that layer boundaries cost no launch, no set-up and no pipeline ramp.
+  int group_layers = fastocr::kMaxGroupLayers;   // 1 = one launch per layer
+  int group_min_rows = 4;                        // rows a CTA of a group launch should have at least
   bool l2_persist_set = false;      // FASTOCR_L2_PERSIST_MB changed the context's persisting-L2 limit: put it back
   size_t l2_persist_before = 0;
   unsigned long long* trace = nullptr;   // set only by debug builds
@@ -179,17 +184,18 @@ struct ProfScope {
   fastocr_ctx* ctx;
   cudaStream_t s;
   bool armed = false;
-  ProfScope(fastocr_ctx* c, int cls, cudaStream_t st) : ctx(c), s(st) {
+  // n: layers the launch covers (a group launch is timed as that many launches of its class)
+  ProfScope(fastocr_ctx* c, int cls, cudaStream_t st, int n = 1) : ctx(c), s(st) {
     if (!c->prof_on) return;
     if (c->prof_runs) {
       if (c->prof_open && c->prof_class.back() == cls) {       // the run goes on
-        c->prof_count.back() += 1;
+        c->prof_count.back() += n;
         return;
       }
       close_run(c, st);
       if (c->prof_used + 2 > c->prof_ev.size()) return;
       c->prof_class.push_back(cls);
-      c->prof_count.push_back(1);
+      c->prof_count.push_back(n);
       cudaEventRecord(c->prof_ev[c->prof_used], st);
       c->prof_open = true;
       c->prof_stream = st;
@@ -198,7 +204,7 @@ struct ProfScope {
     if (c->prof_used + 2 <= c->prof_ev.size()) {
       armed = true;
       c->prof_class.push_back(cls);
-      c->prof_count.push_back(1);
+      c->prof_count.push_back(n);
       cudaEventRecord(c->prof_ev[c->prof_used], st);
     }
   }
@@ -316,6 +322,47 @@ fastocr_status sparse_impl(fastocr_ctx* ctx, const fastocr_kv_view* kv, const vo
   return FASTOCR_OK;
 }
 
+// Layers [l0, l0 + n) of a decode step, all pruned over the same index set, as one launch.
+fastocr_status group_impl(fastocr_ctx* ctx, const fastocr_kv_view* layers, int n, const void* q, size_t q_bytes, const int32_t* idx,
+                          const int32_t* k, int32_t k_stride, int32_t max_kept, void* out, size_t o_bytes, int out_is_fp32,
+                          int wait_point, cudaStream_t s) {
+  const fastocr_kv_view* kv = &layers[0];
+  const int max_len = (max_kept > 0 && max_kept < kv->max_seq_len) ? max_kept : kv->max_seq_len;
+  AttnLaunch a = make_launch(ctx, kv, q, true, max_len);
+  a.idx = idx;
+  a.kcount = k;
+  a.k_stride = k_stride;
+  a.cluster_ctas = 0;
+  a.n_layers = n;
+  a.q_layer_bytes = static_cast<int64_t>(q_bytes);
+  a.out_layer_bytes = static_cast<int64_t>(o_bytes);
+  for (int i = 0; i < n; ++i) {
+    a.layer_k[i] = layers[i].k;
+    a.layer_v[i] = layers[i].v;
+  }
+  // every CTA slot of the GPU unless the group is so small that a CTA would get fewer than a few rows
+  const int64_t rows = static_cast<int64_t>(kv->batch) * kv->num_kv_heads * ((max_len + 31) / 32) * n;
+  int64_t grid = static_cast<int64_t>(ctx->sm_count) * fastocr::kAttnCtasPerSm;
+  if (rows < grid * ctx->group_min_rows) grid = rows / ctx->group_min_rows;
+  a.grid_ctas = static_cast<int>(grid < 1 ? 1 : grid);
+  a.active_ctas = a.grid_ctas;
+  a.wait_point = wait_point;
+  a.plan = nullptr;
+  a.out = out;
+  a.out_is_fp32 = out_is_fp32;
+  ProfScope p(ctx, FASTOCR_PROF_ATTN_SPARSE, s, n);
+  FASTOCR_TRY_CUDA(fastocr::launch_attn_partial(a, s), "attention launch");
+  return FASTOCR_OK;
+}
+
+// whether two layers' views differ only in their caches (what a group launch requires)
+bool same_geometry(const fastocr_kv_view& x, const fastocr_kv_view& y) {
+  return x.batch == y.batch && x.num_q_heads == y.num_q_heads && x.num_kv_heads == y.num_kv_heads && x.page_size == y.page_size &&
+         x.max_seq_len == y.max_seq_len && x.seq_stride_tokens == y.seq_stride_tokens && x.block_table == y.block_table &&
+         x.max_pages == y.max_pages && x.num_pages == y.num_pages && x.seq_len == y.seq_len && x.vis_start == y.vis_start &&
+         x.vis_len == y.vis_len && x.sm_scale == y.sm_scale;
+}
+
 fastocr_status check_scores_args(fastocr_ctx* ctx, const fastocr_kv_view* kv, const float* scores_out, int32_t n_stride) {
   if (scores_out == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL scores_out");
   if (n_stride <= 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "n_stride must be positive");
@@ -352,6 +399,10 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   if (const char* v = std::getenv("FASTOCR_DENSE_CTAS_PER_SM")) ctx->dense_ctas_per_sm = std::atoi(v);     // tuning knobs,
   if (const char* v = std::getenv("FASTOCR_SPARSE_CTAS_PER_SM")) ctx->sparse_ctas_per_sm = std::atoi(v);   // read once here
   if (const char* v = std::getenv("FASTOCR_CLUSTER_MAX_ROWS")) ctx->cluster_max_rows = std::atoi(v);
+  if (const char* v = std::getenv("FASTOCR_GROUP_LAYERS")) ctx->group_layers = std::atoi(v);
+  if (const char* v = std::getenv("FASTOCR_GROUP_MIN_ROWS")) ctx->group_min_rows = std::atoi(v);
+  if (ctx->group_layers < 1 || ctx->group_layers > fastocr::kMaxGroupLayers) ctx->group_layers = fastocr::kMaxGroupLayers;
+  if (ctx->group_min_rows < 1) ctx->group_min_rows = 1;
   if (const char* v = std::getenv("FASTOCR_L2_PERSIST_MB")) {
     // Experiment, off by default: an L2 set-aside for evict-last lines (the logits of a focal layer).
     // It is a limit of this process's CUDA context and takes that much L2 away from everything else.
@@ -366,7 +417,8 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
   }
   if (ctx->dense_ctas_per_sm < 1 || ctx->dense_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->dense_ctas_per_sm = fastocr::kAttnCtasPerSm;
   if (ctx->sparse_ctas_per_sm < 1 || ctx->sparse_ctas_per_sm > fastocr::kAttnCtasPerSm) ctx->sparse_ctas_per_sm = 2;
-  ctx->cap_items = static_cast<int64_t>(ctx->sm_count) * fastocr::kAttnCtasPerSm +
+  // (a group launch uses two slots per CTA instead)
+  ctx->cap_items = 2 * static_cast<int64_t>(ctx->sm_count) * fastocr::kAttnCtasPerSm +
                    static_cast<int64_t>(lim->max_batch) * lim->num_kv_heads + 64;
   const int64_t nvis = lim->max_vis_len > 0 ? lim->max_vis_len : 1;
   const size_t bytes_acc = static_cast<size_t>(ctx->cap_items) * fastocr::kMaxGroup * fastocr::kHeadDim * sizeof(float);
@@ -379,9 +431,9 @@ fastocr_status fastocr_create(fastocr_ctx** out, int device, const fastocr_limit
       (e = cudaMalloc(&ctx->scores, bytes_scores)) != cudaSuccess ||
       (e = cudaMalloc(&ctx->uni_idx, 2 * static_cast<size_t>(lim->max_batch) * nvis * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->uni_cnt, 2 * static_cast<size_t>(lim->max_batch) * sizeof(int32_t))) != cudaSuccess ||
-      (e = cudaMalloc(&ctx->counters, fastocr::kMaxUnits * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMalloc(&ctx->counters, fastocr::kMaxGroupCounters * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->plan, static_cast<size_t>(kPlanCtas) * 4 * sizeof(int4))) != cudaSuccess ||
-      (e = cudaMemset(ctx->counters, 0, fastocr::kMaxUnits * sizeof(int32_t))) != cudaSuccess ||
+      (e = cudaMemset(ctx->counters, 0, fastocr::kMaxGroupCounters * sizeof(int32_t))) != cudaSuccess ||
       (e = cudaMalloc(&ctx->faults, sizeof(unsigned long long))) != cudaSuccess ||
       (e = cudaMemset(ctx->faults, 0, sizeof(unsigned long long))) != cudaSuccess) {
     fastocr_destroy(ctx);
@@ -560,7 +612,7 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
     }
     have = have0;
   }
-  if (n_pruned >= 2 && overlap && !unite) {
+  if (n_pruned >= 2 && overlap && !unite && ctx->group_layers == 1) {
     AttnLaunch pa = sparse_args(ctx, plan_view, q, fixation, k, k_stride, max_kept);
     if (pa.grid_ctas <= kPlanCtas) {
       plan_grid = pa.grid_ctas;
@@ -581,6 +633,22 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
     const bool mixed = n_focal != 0 && n_focal != B;
     const uint8_t* mask = mixed ? focal_seq_dev + static_cast<size_t>(l) * B : nullptr;
     fastocr_status st;
+    if (n_focal == 0) {
+      // a run of layers that the whole batch attends pruned, over the same set and the same lengths: one launch
+      int n = 1;
+      while (n < ctx->group_layers && l + n < num_layers && focal_count(l + n) == 0 && same_geometry(layers[l], layers[l + n])) ++n;
+      const bool fits = static_cast<int64_t>(B) * layers[l].num_kv_heads <= fastocr::kMaxUnits;
+      if (n > 1 && overlap && fits) {
+        const bool chained = prev != kOther;
+        const int wp = !chained ? fastocr::kWaitAtStart : (prev == kAttention ? fastocr::kWaitBeforeWrites : fastocr::kWaitAfterSetup);
+        st = group_impl(ctx, &layers[l], n, ql, q_bytes, unite ? uni_idx(cur) : fixation, unite ? uni_cnt(cur) : k,
+                        unite ? U : k_stride, max_kept, ol, o_bytes, out_is_fp32, wp, s);
+        if (st != FASTOCR_OK) return st;
+        prev = kAttention;
+        l += n - 1;
+        continue;
+      }
+    }
     if (n_focal != B) {
       // A pruned layer that follows another attention layer reads nothing the latter wrote (its
       // queries, index set and cache were complete before), so the two may overlap; right after

@@ -123,7 +123,7 @@ __device__ __forceinline__ void store_pair(void* out, int is_fp32, int64_t index
 
 // number of attended tokens of sequence b and the pieces needed to enumerate them
 struct SeqGeom {
-  int vs, N, kept_vis, n_tok;                           // n_tok < 0: the sequence takes no part in this launch
+  int vs, N, kept_vis, n_tok;                           // n_tok: attended tokens of this launch (< 0: the sequence takes no part)
 };
 // The lengths come from device memory and cannot be checked by the host without a synchronisation:
 // they are forced into what the host did check (0 <= seq_len <= max_seq_len, the image span inside
@@ -350,10 +350,16 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   // pipeline refill) and a unit that fits one CTA needs no global merge. Otherwise (ragged
   // batches, more units than CTAs, or long ranges where a few merges are negligible): all rows
   // laid end to end and cut into equal ranges.
-  const int parts_rule = planned ? 0 : split_rule(units, grid, total_rows, longest_unit, HAS_IDX);
+  // A group of layers (pruned passes only): the rows of all its layers, layer after layer, are one long
+  // sequence cut into equal ranges. A CTA streams through its range without regard to unit or layer
+  // boundaries; the few units it shares with its neighbours are merged through global partials.
+  const int n_layers = HAS_IDX ? max(a.n_layers, 1) : 1;
+  const bool grouped = n_layers > 1;
+  const int all_rows = n_layers * total_rows;          // rows of the launch
+  const int parts_rule = (planned || grouped) ? 0 : split_rule(units, grid, total_rows, longest_unit, HAS_IDX);
   const bool split_units = planned ? plan1.z != 0 : parts_rule > 0;
   const int parts = planned ? plan1.w : max(parts_rule, 1);     // CTAs per unit
-  const int per_cta = planned ? plan2.x : (total_rows + grid - 1) / grid;   // rows per CTA (equal-range mode)
+  const int per_cta = planned ? plan2.x : (all_rows + grid - 1) / grid;   // rows per CTA (equal-range mode)
   int r0 = 0, r1 = 0, first_unit = 0;
   if (planned) {
     first_unit = plan0.y;
@@ -370,8 +376,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       r1 = min(ue, r0 + per);
     }
   } else {
-    r0 = min(total_rows, blockIdx.x * per_cta);
-    r1 = min(total_rows, r0 + per_cta);
+    r0 = min(all_rows, static_cast<int>(blockIdx.x) * per_cta);
+    r1 = min(all_rows, r0 + per_cta);
   }
 
   const float scale_log2 = a.sm_scale * 1.4426950408889634f;
@@ -411,11 +417,17 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 
   // ---- the CTA's range, one unit segment after the other --------------------------------------
   int u = first_unit;
+  int layer = 0, layer_row0 = 0;                       // layer of the group the walk is in, and its first row
   if (!planned && !split_units && r0 < r1) {
-    int lo = 0, hi = units;                            // largest u with prefix[u] <= r0
+    if (grouped) {
+      layer = r0 / total_rows;
+      layer_row0 = layer * total_rows;
+    }
+    const int local = r0 - layer_row0;
+    int lo = 0, hi = units;                            // largest u with prefix[u] <= local
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (prefix_s[mid] <= r0) lo = mid; else hi = mid;
+      if (prefix_s[mid] <= local) lo = mid; else hi = mid;
     }
     u = lo;
   }
@@ -425,10 +437,26 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     wait_for_prior_grids();
     dependents_may_launch();
   }
+  // State that survives a segment boundary when the look-ahead stages of one segment have already
+  // fetched the first blocks of the next (see `carry_next` below).
+  uint32_t qb[8][2];                                   // B fragments of Q^T of the segment's unit
+  bool carried = false;                                // this segment's first blocks are in flight already, q is loaded
+  int pos_p = 0, row_p = 0;
+  bool idx_p = false;
+  const uint32_t ring_end = ring_warp + kStages * L::kStageBytes;
+  uint32_t src = ring_warp, dst_ahead = ring_warp;     // ring slots of block n and of block n + kDepth
 #pragma unroll 1
   while (seg_begin < r1) {
-    while (prefix_s[u + 1] <= seg_begin) ++u;          // skip empty units
-    const int ubeg = prefix_s[u], uend = prefix_s[u + 1];
+    while (true) {                                     // skip empty units; past the last unit the next layer begins
+      if (grouped && u == units) {
+        u = 0;
+        ++layer;
+        layer_row0 += total_rows;
+      }
+      if (layer_row0 + prefix_s[u + 1] > seg_begin) break;
+      ++u;
+    }
+    const int ubeg = layer_row0 + prefix_s[u], uend = layer_row0 + prefix_s[u + 1];
     const int seg_rows = min(uend, r1) - seg_begin;    // rows of unit u inside this range
     const int b = u / Hkv, g = u - b * Hkv;
     SeqGeom sg;
@@ -441,19 +469,22 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     }
     const int tok0 = (seg_begin - ubeg) * kRowTokens + warp * kBlockTokens;   // this warp's first token of the segment
     // this lane's 16-byte chunk of cache row 0 of the unit (a row is row_bytes long)
-    const char* kptr = reinterpret_cast<const char*>(a.k) + (b * seq_elems + g * kHeadDim + 8 * c16) * 2;
-    const char* vptr = HAS_V ? reinterpret_cast<const char*>(a.v) + (b * seq_elems + g * kHeadDim + 8 * c16) * 2 : nullptr;
+    const void* k_base = grouped ? a.layer_k[layer] : a.k;
+    const void* v_base = grouped ? a.layer_v[layer] : a.v;
+    const char* kptr = reinterpret_cast<const char*>(k_base) + (b * seq_elems + g * kHeadDim + 8 * c16) * 2;
+    const char* vptr = HAS_V ? reinterpret_cast<const char*>(v_base) + (b * seq_elems + g * kHeadDim + 8 * c16) * 2 : nullptr;
 
     // B fragments of Q^T for the eight 16-dim steps: head g8, dims 16 s + {2 t4, 2 t4 + 1} and 16 s + 8 + {2 t4, 2 t4 + 1}
-    uint32_t qb[8][2];
-    {
-      const uint32_t* qp = reinterpret_cast<const uint32_t*>(a.q) + (static_cast<int64_t>(u) * G + g8) * (kHeadDim / 2) + t4;
+    auto load_q = [&](int unit) {
+      const uint32_t* qp = reinterpret_cast<const uint32_t*>(static_cast<const char*>(a.q) + layer * a.q_layer_bytes) +
+                           (static_cast<int64_t>(unit) * G + g8) * (kHeadDim / 2) + t4;
 #pragma unroll
       for (int st = 0; st < 8; ++st) {
         qb[st][0] = head_ok ? __ldg(qp + 8 * st) : 0u;
         qb[st][1] = head_ok ? __ldg(qp + 8 * st + 4) : 0u;
       }
-    }
+    };
+    if (!carried) load_q(u);
     // The lane's share of the state: heads hA = 2 t4 and hB = 2 t4 + 1.
     float o[8][4];                                     // O^T tile j: dims {16 j + g8, 16 j + 8 + g8} x heads {hA, hB}
 #pragma unroll
@@ -474,13 +505,39 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     // A block is named by the list index jr of its first token (tok0 + 32 per block); it exists
     // while jr < lim. All 32 lanes run stages P and R (lanes 16-31 mirror lanes 0-15: no divergence).
     const int lim = min(sg.n_tok, tok0 + seg_rows * kRowTokens);
+    // When the range goes on into the next KV head of the same sequence (same lengths, same index
+    // list, same block table; the cache rows lie 256 bytes further), the look-ahead stages do not idle
+    // over the last blocks of this segment: they fetch the first blocks of the next one, which then
+    // starts with its pipeline full, no prologue, no drain in between. (Other boundaries: next
+    // sequence, next layer, a short segment: the pipeline is drained and refilled.)
+    const int seg_tok_end = tok0 + seg_rows * kRowTokens;          // list index at which this warp leaves the segment
+    bool carry_next = false;
+    int lim_n = 0;                                                 // the next segment's limit; 0: nothing to fetch there
+    if (!planned && !split_units && seg_begin + seg_rows < r1 && seg_rows >= kDepth + 2 && u + 1 < units && (u + 1) / Hkv == b) {
+      const int rows_n = min(layer_row0 + prefix_s[u + 2], r1) - (seg_begin + seg_rows);
+      if (prefix_s[u + 2] > prefix_s[u + 1] && rows_n > 0) {
+        carry_next = true;
+        lim_n = min(sg.n_tok, warp * kBlockTokens + rows_n * kRowTokens);
+      }
+    }
+    const int shift_n = seg_tok_end - warp * kBlockTokens;         // list index in this segment -> list index in the next
     const int tl = lane & (kBlockTokens - 1);
     const int vis_end = sg.vs + sg.kept_vis, text_shift = sg.N - sg.kept_vis;
     const int32_t* idx_row = HAS_IDX ? a.idx + static_cast<int64_t>(b) * a.k_stride - sg.vs : nullptr;
     const int32_t* bt_row = PAGED ? a.block_table + static_cast<int64_t>(b) * a.max_pages : nullptr;
-    auto stage_p = [&](int jr, int& pos, bool& is_idx) {     // is_idx: pos is a raw index-list entry, checked in stage R
+    // A look-ahead block named by a list index past the end of this segment belongs to the next one.
+    auto locate = [&](int& jr, int& lx, int& head_off) {
+      lx = lim;
+      head_off = 0;
+      if (jr >= seg_tok_end) {
+        jr -= shift_n;
+        lx = lim_n;
+        head_off = kHeadDim * 2;
+      }
+    };
+    auto stage_p = [&](int jr, int lx, int& pos, bool& is_idx) {     // is_idx: pos is a raw index-list entry, checked in stage R
       is_idx = false;
-      if (jr < lim) {
+      if (jr < lx) {
         const int j = min(jr + tl, sg.n_tok - 1);
         pos = j;
         if (HAS_IDX) {                                 // kept set: text before | selected image | text after
@@ -493,8 +550,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
         }
       }
     };
-    auto stage_r = [&](int jr, int pos, bool is_idx, int& row) {
-      if (jr < lim) {
+    auto stage_r = [&](int jr, int lx, int pos, bool is_idx, int& row) {
+      if (jr < lx) {
         if (is_idx) {
           const int inside = min(max(pos, 0), sg.N - 1);      // never read outside the image span
           bad_entries += inside != pos;
@@ -515,23 +572,23 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     // The copies of a block: its 16 K rows are one cp.async group, its 16 V rows another (K is
     // needed at the top of the block's iteration, V only after the softmax, and each tile's ring
     // slot is free again as soon as the fragments of the block that used it last are in registers).
-    auto stage_ik = [&](int jr, uint32_t dst, int row) {
-      if (jr < lim) {
+    auto stage_ik = [&](int jr, int lx, int head_off, uint32_t dst, int row) {
+      if (jr < lx) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {                  // rows 2i (lanes 0-15) and 2i + 1 (lanes 16-31)
           const int rr = __shfl_sync(0xffffffffu, row, 2 * i + half);
-          cp_async16(dst + cp_off[i & 3] + (i >> 2) * 2048, kptr + static_cast<int64_t>(rr) * row_bytes, stream_policy);
+          cp_async16(dst + cp_off[i & 3] + (i >> 2) * 2048, kptr + head_off + static_cast<int64_t>(rr) * row_bytes, stream_policy);
         }
       }
       cp_async_commit();
     };
-    auto stage_iv = [&](int jr, uint32_t dst, int row) {
+    auto stage_iv = [&](int jr, int lx, int head_off, uint32_t dst, int row) {
       if (!HAS_V) return;
-      if (jr < lim) {
+      if (jr < lx) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int rr = __shfl_sync(0xffffffffu, row, 2 * i + half);
-          cp_async16(dst + L::kTileBytes + cp_off[i & 3] + (i >> 2) * 2048, vptr + static_cast<int64_t>(rr) * row_bytes, stream_policy);
+          cp_async16(dst + L::kTileBytes + cp_off[i & 3] + (i >> 2) * 2048, vptr + head_off + static_cast<int64_t>(rr) * row_bytes, stream_policy);
         }
       }
       cp_async_commit();
@@ -543,10 +600,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     // sequence's cache span, and the first touch of a page by this SM costs a translation miss in
     // the middle of the stream. Touch every page of the span now, all at once (one line each, L2
     // only): lanes 0-15 of warp 0 for K, lanes 16-31 for V.
-    if (HAS_IDX && !PAGED && warp == 0) {
+    if (HAS_IDX && !PAGED && warp == 0 && !carried) {
       const int64_t span = static_cast<int64_t>(sg.n_tok - sg.kept_vis + sg.N) * row_elems * 2;   // bytes, whole sequence
-      const char* base = reinterpret_cast<const char*>(half ? static_cast<const void*>(a.v) : a.k) +
-                         (b * seq_elems + g * kHeadDim) * 2;
+      const char* base = reinterpret_cast<const char*>(half ? v_base : k_base) + (b * seq_elems + g * kHeadDim) * 2;
       int64_t off = static_cast<int64_t>(c16) << 21;
       if (c16 == 15) off = span - 256;
       if (off >= 0 && off < span && (HAS_V || half == 0)) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
@@ -554,36 +610,35 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     // Filling the stages: the lookups of the first rows are issued together (one round trip for
     // the index-list entries, one for the block-table entries) instead of one after the other,
     // then the copies of the first kDepth rows go out.
-    int pos_p = 0, row_p = 0;
-    bool idx_p = false;
     FASTOCR_TRACE_CYC(11);
-    {
+    if (!carried) {
+      // (a segment shorter than the look-ahead names blocks past its end here: they are looked for in
+      // the next segment only by the main loop, so they must not exist for the prologue)
       int posq[kDepth + 2], rowq[kDepth + 1];
       bool ixq[kDepth + 2];
 #pragma unroll
       for (int r = 0; r < kDepth + 2; ++r) {
         posq[r] = 0;
-        stage_p(tok0 + r * kRowTokens, posq[r], ixq[r]);
+        stage_p(tok0 + r * kRowTokens, lim, posq[r], ixq[r]);
       }
 #pragma unroll
       for (int r = 0; r < kDepth + 1; ++r) {
         rowq[r] = 0;
-        stage_r(tok0 + r * kRowTokens, posq[r], ixq[r], rowq[r]);
+        stage_r(tok0 + r * kRowTokens, lim, posq[r], ixq[r], rowq[r]);
       }
       FASTOCR_TRACE_CYC(12);
 #pragma unroll
       for (int r = 0; r < kDepth; ++r) {
-        stage_ik(tok0 + r * kRowTokens, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
-        stage_iv(tok0 + r * kRowTokens, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
+        stage_ik(tok0 + r * kRowTokens, lim, 0, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
+        stage_iv(tok0 + r * kRowTokens, lim, 0, ring_warp + (r % kStages) * L::kStageBytes, rowq[r]);
       }
       row_p = rowq[kDepth];
       pos_p = posq[kDepth + 1];
       idx_p = ixq[kDepth + 1];
+      src = ring_warp;
+      dst_ahead = ring_warp + (kDepth % kStages) * L::kStageBytes;
       FASTOCR_TRACE_CYC(13);
     }
-    uint32_t src = ring_warp;                                          // ring slot of block n
-    uint32_t dst_ahead = ring_warp + (kDepth % kStages) * L::kStageBytes;   // ring slot of block n + kDepth
-    const uint32_t ring_end = ring_warp + kStages * L::kStageBytes;
 #pragma unroll 1
     for (int j0 = tok0; j0 < tok0 + seg_rows * kRowTokens; j0 += kRowTokens) {   // j0: list index of the block's first token
       FASTOCR_TRACE_CLK(c_top);
@@ -612,10 +667,18 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       // ---- look-ahead: K copies of block n + kDepth into the slot block n's K tile just left, then
       // stages R and P one and two blocks further ---------------------------------------------------
       __syncwarp();                                    // every lane has this block's K fragments
-      stage_ik(j0 + kDepth * kRowTokens, dst_ahead, row_p);
+      int jr_i = j0 + kDepth * kRowTokens, lim_i, off_i;
+      locate(jr_i, lim_i, off_i);
+      stage_ik(jr_i, lim_i, off_i, dst_ahead, row_p);
       const int row_v = row_p;
-      stage_r(j0 + (kDepth + 1) * kRowTokens, pos_p, idx_p, row_p);
-      stage_p(j0 + (kDepth + 2) * kRowTokens, pos_p, idx_p);
+      {
+        int jr = j0 + (kDepth + 1) * kRowTokens, lx, off;
+        locate(jr, lx, off);
+        stage_r(jr, lx, pos_p, idx_p, row_p);
+        jr = j0 + (kDepth + 2) * kRowTokens;
+        locate(jr, lx, off);
+        stage_p(jr, lx, pos_p, idx_p);
+      }
 
       FASTOCR_TRACE_CLK(c_look);
       FASTOCR_TRACE_ADD(trace_look, c_look, c_qk);
@@ -674,7 +737,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
 #pragma unroll
           for (int j = 0; j < 8; ++j) ldsm_x4_trans(va[j], src + L::kTileBytes + v_off[j & 3] + (j >> 2) * 128);
           __syncwarp();                                // the V tile's slot is free: copies of block n + kDepth
-          stage_iv(j0 + kDepth * kRowTokens, dst_ahead, row_v);   // go out while the tensor cores work
+          stage_iv(jr_i, lim_i, off_i, dst_ahead, row_v);         // go out while the tensor cores work
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             mma_bf16(o[j], va[j][0], va[j][1], va[j][2], va[j][3], ph0, ph1);
@@ -682,7 +745,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           }
         }
       }
-      if (HAS_V && !live) stage_iv(j0 + kDepth * kRowTokens, dst_ahead, row_v);   // keeps the group count in step (nothing to copy any more)
+      if (HAS_V && !live) stage_iv(jr_i, lim_i, off_i, dst_ahead, row_v);   // keeps the group count in step
       src += L::kStageBytes;
       if (src == ring_end) src = ring_warp;
       dst_ahead += L::kStageBytes;
@@ -690,7 +753,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       FASTOCR_TRACE_CLK(c_end);
       FASTOCR_TRACE_ADD(trace_pv, c_end, c_look);
     }
-    cp_async_wait<0>();
+    if (carry_next) load_q(u + 1);                     // the next segment's queries arrive while this one is merged
+    else cp_async_wait<0>();
     FASTOCR_TRACE_MARK(4);
     FASTOCR_TRACE_CYC(15);
 
@@ -813,7 +877,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
         cluster.sync();                                // no CTA leaves while its buffer may still be read
       } else if (c_lo != c_hi) {                       // the unit is shared with other CTAs
         wait_for_prior_grids();                        // the split workspace may still be in use by the previous kernel
-        const int64_t slot = static_cast<int64_t>(blockIdx.x) + u;
+        // a group launch: a range has at most two shared pieces, its first and its last segment
+        const int64_t slot = grouped ? 2 * static_cast<int64_t>(blockIdx.x) + (seg_begin == r0 ? 0 : 1) : static_cast<int64_t>(blockIdx.x) + u;
+        int* arrivals = a.counters + (grouped ? layer * units + u : u);
 #pragma unroll
         for (int it = 0; it < kItems; ++it) {
           const int e = it * kThreads + tid, h = e >> 4, d8 = (e & 15) * 8;
@@ -828,9 +894,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
         __threadfence();                               // partial visible before the arrival is counted
         __syncthreads();
         if (tid == 0) {
-          const int prev = atomicAdd(a.counters + u, 1);
+          const int prev = atomicAdd(arrivals, 1);
           const int last = prev == c_hi - c_lo;
-          if (last) a.counters[u] = 0;                 // ready for the next launch
+          if (last) *arrivals = 0;                     // ready for the next launch
           *mrg_flag = last;
         }
         __syncthreads();
@@ -855,7 +921,8 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
               const int hh = h < G ? h : 0;
 #pragma unroll
               for (int r = 0; r < kMergeRound; ++r) {  // a short tail re-reads the last partial (ignored below)
-                const int64_t sl = static_cast<int64_t>(min(c0 + r, c_hi)) + u;
+                const int cc = min(c0 + r, c_hi);        // CTA cc's piece of this unit: its first segment iff its range starts inside the unit
+                const int64_t sl = grouped ? 2 * static_cast<int64_t>(cc) + (cc * per_cta >= ubeg ? 0 : 1) : static_cast<int64_t>(cc) + u;
                 ml[it][r] = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (sl * kMaxGroup + hh) * 2));
                 x0[it][r] = x1[it][r] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (HAS_V) {
@@ -891,8 +958,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
           if (HAS_V) {
             const float inv = den[it] > 0.f ? 1.f / den[it] : 0.f;
             const int64_t oi = (head0 + h) * kHeadDim + d8;
+            void* out_l = static_cast<char*>(a.out) + layer * a.out_layer_bytes;
 #pragma unroll
-            for (int i = 0; i < 8; i += 2) store_pair(a.out, a.out_is_fp32, oi + i, num[it][i] * inv, num[it][i + 1] * inv);
+            for (int i = 0; i < 8; i += 2) store_pair(out_l, a.out_is_fp32, oi + i, num[it][i] * inv, num[it][i + 1] * inv);
           }
           if (LOGITS && (e & 15) == 0) {
             a.stats[(head0 + h) * 2 + 0] = M[it];
@@ -903,7 +971,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     }
     seg_begin += seg_rows;
     ++u;
+    carried = carry_next;
   }
+  cp_async_wait<0>();
   if (r0 >= r1 && merges_in_cluster(split_units, parts)) {
     cg::cluster_group cluster = cg::this_cluster();    // a CTA without rows: the two barriers of the cluster merge
     cluster.sync();
@@ -932,8 +1002,9 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       if (load_geom(a, e / Hkv, HAS_IDX).n_tok != 0) continue;   // not part of this launch: left alone
       wait_for_prior_grids();
       const int64_t head0 = static_cast<int64_t>(e) * G;
-      for (int i = tid; i < G * kHeadDim / 2; i += kThreads)
-        if (HAS_V) store_pair(a.out, a.out_is_fp32, head0 * kHeadDim + 2 * i, 0.f, 0.f);
+      for (int l = 0; l < n_layers; ++l)
+        for (int i = tid; i < G * kHeadDim / 2; i += kThreads)
+          if (HAS_V) store_pair(static_cast<char*>(a.out) + l * a.out_layer_bytes, a.out_is_fp32, head0 * kHeadDim + 2 * i, 0.f, 0.f);
       for (int i = tid; i < G; i += kThreads)
         if (LOGITS) {
           a.stats[(head0 + i) * 2 + 0] = -INFINITY;

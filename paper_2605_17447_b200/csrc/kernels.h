@@ -11,6 +11,8 @@ constexpr int kAttnWarps = 2;         // warps per persistent attention CTA
 constexpr int kAttnCtasPerSm = 4;     // resident CTAs per SM (registers and shared memory)
 constexpr int kMaxUnits = 512;        // sequences x KV heads per launch (their row prefix lives in shared memory)
 constexpr int kMaxPartsPerUnit = 16;  // CTAs sharing one unit in split mode (bounds the last CTA's merge)
+constexpr int kMaxGroupLayers = 32;    // consecutive pruned layers one launch can walk (their cache pointers travel in the launch arguments)
+constexpr int kMaxGroupCounters = kMaxGroupLayers * kMaxUnits;   // arrival counters: one per (layer of the group, unit)
 constexpr int kTopkMaxN = 32768;      // keys of one sequence must fit one CTA's shared memory
 constexpr int kTopkMaxHeads = 128;    // query heads the selection kernel can score by itself
 
@@ -121,12 +123,22 @@ struct AttnLaunch {
   int32_t cluster_ctas;       // CTAs per unit when the grid is units x this many and the launch should run one cluster
                               // of that size per unit (a unit's pieces then merge through distributed shared memory); else 0
   int32_t wait_point;         // where the kernel waits for earlier kernels: kWaitAtStart / kWaitAfterSetup / kWaitBeforeWrites
+  // A group of consecutive pruned layers in one launch (n_layers > 1; pruned mode only): the layers share
+  // lengths, kept counts, index set, block table and geometry and differ in their caches, queries and
+  // outputs. The rows of all layers of the group are laid end to end (layer-major) and cut into equal
+  // ranges, one per CTA.
+  int32_t n_layers;           // 0 or 1: a single layer (k, v, q, out above)
+  int64_t q_layer_bytes;      // distance between consecutive layers' queries / outputs
+  int64_t out_layer_bytes;
+  const void* layer_k[kMaxGroupLayers];
+  const void* layer_v[kMaxGroupLayers];
   const int4* plan;           // NULL or one 64-byte record per CTA written by launch_attn_plan for this very launch
                               // shape (grid, lengths, kept counts): the CTA's range and unit, ready made
   // workspace
-  float* part_acc;            // [slots][8][128], slot = CTA index + unit index (unit = sequence * Hkv + KV head)
+  float* part_acc;            // [slots][8][128], slot = CTA index + unit index (unit = sequence * Hkv + KV head);
+                              // a group launch: slot = 2 x CTA index + (0: the CTA's first piece, 1: its last)
   float* part_ml;             // [slots][8][2]  (max, sum) in the log2 domain
-  int32_t* counters;          // [units] arrival counters, zero between launches
+  int32_t* counters;          // [kMaxGroupCounters] arrival counters per (layer of the group, unit), zero between launches
   // results
   void* out;                  // [B][H][128] bf16 or fp32 (unused when v == nullptr)
   int32_t out_is_fp32;

@@ -27,6 +27,27 @@ namespace cg = cooperative_groups;
 namespace fastocr {
 namespace {
 
+#ifdef FASTOCR_TOPK_TRACE
+// debug builds: cycle stamps of the selection kernel's phases, 8 per CTA
+__device__ long long g_topk_trace[8 * 1024];
+__device__ unsigned long long g_topk_wall[2 * 1024];  // wall-clock nanoseconds at entry (after the wait) and at exit
+__device__ __forceinline__ unsigned long long topk_wall_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
+  return t;
+}
+#define TOPK_STAMP(i)                                                          \
+  do {                                                                         \
+    if (threadIdx.x == 0 && blockIdx.x < 1024) {                               \
+      g_topk_trace[blockIdx.x * 8 + (i)] = clock64();                          \
+      if ((i) == 0) g_topk_wall[blockIdx.x * 2] = topk_wall_now();             \
+      if ((i) == 6) g_topk_wall[blockIdx.x * 2 + 1] = topk_wall_now();         \
+    }                                                                          \
+  } while (0)
+#else
+#define TOPK_STAMP(i) do { } while (0)
+#endif
+
 constexpr int kTopkThreads = 1024;
 constexpr int kTopkWarps = kTopkThreads / 32;
 constexpr int kTopkMaxCluster = 8;
@@ -155,6 +176,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
 
   wait_for_prior_grids();
   dependents_may_launch();
+  TOPK_STAMP(0);
   cg::cluster_group cluster = cg::this_cluster();
   const int C = static_cast<int>(cluster.num_blocks());
   const int c = static_cast<int>(cluster.block_rank());
@@ -201,9 +223,11 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
                     for (int t = 0; t < count; ++t) all_copies(j0 + t, kq[t]);
                   }
                 });
+    TOPK_STAMP(7);
     if (C > 1) cluster.sync();                          // every slice has arrived in every copy
   }
   __syncthreads();
+  TOPK_STAMP(1);
 
   // ---- radix select, three passes over digits of 11, 11 and 10 bits (most significant first) ----
   // Pass p histograms the digit of the keys that match the prefix found so far; thread t then owns
@@ -265,6 +289,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
       sel_remaining = remaining - (first ? before : before + c0);
     }
     __syncthreads();
+    TOPK_STAMP(2 + pass);
   }
   const uint32_t thr = sel_prefix;                      // key of the k-th largest score
   const uint32_t take_eq = sel_remaining;               // how many keys equal to thr are selected
@@ -342,6 +367,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   __syncthreads();
   uint32_t gt_before = warp_gt[warp] + gt_incl - gt;
   uint32_t eq_before = warp_eq[warp] + eq_incl - eq;
+  TOPK_STAMP(5);
   int32_t* op = idx_out + static_cast<int64_t>(b) * k_stride;
   auto emit = [&](int i, uint32_t key) {
     const bool mine = i >= lo_i && i < hi_i;
@@ -373,6 +399,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
       eq_run += __popc(m_eq);
     }
   }
+  TOPK_STAMP(6);
 }
 
 // The same selection with the sequence split over the cluster in every phase, for long sequences:
@@ -661,6 +688,15 @@ static int max_active_clusters(int C, size_t smem) {
   if (used < 16) memo[used++] = Memo{C, smem, n};
   return n;
 }
+
+#ifdef FASTOCR_TOPK_TRACE
+extern "C" int fastocr_debug_topk_trace(long long* host_out, int n) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_topk_trace, sizeof(long long) * n));
+}
+extern "C" int fastocr_debug_topk_wall(unsigned long long* host_out, int n) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_topk_wall, sizeof(unsigned long long) * n));
+}
+#endif
 
 cudaError_t configure_topk() {
   cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkMaxN * 4 + 16);

@@ -59,7 +59,9 @@ def test_full_size_layer_chain_against_oracle_on_sampled_sequences():
     have = fo.fastocr_decode_step(ctx, [kv, kv, kv], torch.stack([q, q, q]), out2, [True, False, False], kd, fix, False, N)
     torch.cuda.synchronize()
     assert have and torch.equal(fix, idx)
-    assert torch.equal(out2[0], dense) and torch.equal(out2[1], out) and torch.equal(out2[2], out)
+    assert torch.equal(out2[0], dense)
+    for l in (1, 2):       # the two pruned layers run as one launch that cuts their rows differently: same sums in another order
+        assert float((out2[l] - out).abs().max()) <= 3e-5
     # sampled sequences against the oracle, element by element
     for b in (0, 17, 63):
         qc, Kc, Vc = q[b].cpu(), K[b].cpu(), V[b].cpu()
@@ -215,11 +217,10 @@ def test_more_units_than_ctas():
     torch.cuda.synchronize()
     for b in range(80):
         ref = oracle.sparse(*case.seq(b), SCALE, case.vis_start[b], case.vis_len[b], idx[b, :ks[b]], True)
-        err = (out[b].cpu() - ref).abs()
-        assert err.max() <= 1e-4 and err.mean() <= 1e-3, b
+        for got in (out[b], out3[0, b], out3[1, b], out3[2, b]):      # one launch per layer, and the three layers as one launch
+            err = (got.cpu() - ref).abs()
+            assert err.max() <= 1e-4 and err.mean() <= 1e-3, b
         err = (dense[b].cpu() - oracle.dense(*case.seq(b), SCALE, True)).abs()
         assert err.max() <= 1e-4 and err.mean() <= 1e-3, b
-    for l in range(3):
-        assert torch.equal(out3[l], out)
     assert ctx.device_faults() == 0
     ctx.close()

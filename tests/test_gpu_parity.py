@@ -207,14 +207,26 @@ def test_sparse_cluster_merge_matches_oracle(fo, ctx, case_no, paged):
     fo.fastocr_sparse_decode_attn(ctx, kv, q, idx.cuda(), kd, out, max_kept=max_kept)
     assert fo.cluster_launch_count() == before + (1 if CLUSTERS_ON else 0)       # the path under test is the one that ran
     _check_out(out, ref)
-    # the same inside a decode step (launch plan in use), three pruned layers on last step's set
-    out3 = torch.full((3, case.B, case.H, 128), 7.0, dtype=torch.float32, device="cuda")
-    before = fo.cluster_launch_count()
-    assert fo.fastocr_decode_step(ctx, [kv, kv, kv], torch.stack([q, q, q]), out3, [False, False, False], kd,
-                                  idx.cuda().clone(), True, max(case.vis_len), max_kept=max_kept)
-    assert fo.cluster_launch_count() == before + (3 if CLUSTERS_ON else 0)
-    for l in range(3):
-        assert torch.equal(out3[l], out)
+    # the same inside a decode step, three pruned layers on last step's set: as one group launch (the
+    # library's default), and, with group launches switched off, as three cluster launches from a launch plan
+    for group_layers in ("32", "1"):
+        saved = os.environ.get("FASTOCR_GROUP_LAYERS")
+        os.environ["FASTOCR_GROUP_LAYERS"] = group_layers        # read when a context is created
+        c2 = fo.Context(max_batch=8, num_q_heads=64, num_kv_heads=8, max_seq_len=40000, max_vis_len=32768)
+        if saved is None:
+            del os.environ["FASTOCR_GROUP_LAYERS"]
+        else:
+            os.environ["FASTOCR_GROUP_LAYERS"] = saved
+        out3 = torch.full((3, case.B, case.H, 128), 7.0, dtype=torch.float32, device="cuda")
+        before = fo.cluster_launch_count()
+        assert fo.fastocr_decode_step(c2, [kv, kv, kv], torch.stack([q, q, q]), out3, [False, False, False], kd,
+                                      idx.cuda().clone(), True, max(case.vis_len), max_kept=max_kept)
+        if group_layers == "1":
+            assert fo.cluster_launch_count() == before + (3 if CLUSTERS_ON else 0)
+        for l in range(3):
+            _check_out(out3[l], ref)
+        assert c2.device_faults() == 0
+        c2.close()
 
 
 @pytest.mark.parametrize("seed", range(12))

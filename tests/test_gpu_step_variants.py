@@ -249,3 +249,35 @@ def test_page_ids_outside_the_pool_are_clamped_and_counted(fo, ctx):
     assert ctx.device_faults() == 2 * 16 * 4                     # two pages x 16 tokens, looked up once by each of the 4 KV heads' units
     _check_out(out[0], oracle.dense(*case.seq(0), SCALE, True))
     assert bool(torch.isfinite(out).all())
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_layers_after_a_selection_with_empty_text_or_empty_selection(fo, ctx, paged):
+    """Pruned layers after a focal layer, run as one launch: sequences without text tokens, sequences that
+    keep no image token, and a sequence with neither (zeros) must come out right; every other sequence is
+    the oracle's pruned attention over the set the focal layer selected."""
+    L = 4
+    spans = [(4, 200, 10), (0, 150, 0), (3, 90, 5), (0, 64, 0), (7, 130, 0)]
+    ks = [20, 15, 0, 0, 13]                                      # sequence 1: no text; 2: nothing kept; 3: neither
+    cases, views, q_all = make_layer_stack(2000, spans, L, page_size=16 if paged else 0, q_boost=1.5)
+    base = cases[0]
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    fix = torch.full((base.B, max(ks)), -1, dtype=torch.int32, device="cuda")
+    out = torch.full((L, base.B, base.H, 128), 7.0, dtype=torch.float32, device="cuda")
+    assert fo.fastocr_decode_step(ctx, views, q_all.cuda(), out, [True, False, False, False], kd, fix, False, max(base.vis_len))
+    torch.cuda.synchronize()
+    for b in range(base.B):
+        q0, K0, V0 = cases[0].seq(b)
+        _check_out(out[0, b], oracle.dense(q0, K0, V0, SCALE, True))
+        sel = fix[b, :ks[b]].cpu()
+        if ks[b]:
+            sc, _ = oracle.scores(q0, K0, SCALE, base.vis_start[b], base.vis_len[b], True)
+            ref_sel = oracle.topk(sc, ks[b])
+            kth = float(torch.sort(sc, descending=True).values[ks[b] - 1])
+            assert all(abs(float(sc[i]) - kth) <= 1e-5 * kth for i in set(sel.tolist()) ^ set(ref_sel.tolist()))
+        for l in range(1, L):
+            if ks[b] + base.seq_len[b] - base.vis_len[b] == 0:
+                assert float(out[l, b].abs().max()) == 0.0
+            else:
+                _check_out(out[l, b], oracle.sparse(*cases[l].seq(b), SCALE, base.vis_start[b], base.vis_len[b], sel, True))
+    assert ctx.device_faults() == 0
