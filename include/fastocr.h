@@ -37,6 +37,10 @@
  *     meaningless; all other sequences are unaffected). Kept counts above
  *     vis_len[b] or above the index list's row length k_stride are clamped
  *     silently (documented behaviour, not a fault).
+ *   - Arithmetic: bf16 inputs, fp32 accumulation; the two contractions of a block (q.K^T, P.V) run
+ *     on the tensor cores (warp-level mma, bf16 x bf16 -> fp32), P split into a bf16 high part and a
+ *     bf16 remainder; exponentials are ex2.approx. Outputs agree with an fp32 CPU evaluation of the
+ *     same formulas to about 1e-4 absolute.
  *   - head_dim must be 128 and num_q_heads / num_kv_heads (the GQA group size)
  *     one of 1, 2, 4, 7, 8; query head h reads KV head h / group size.
  */
