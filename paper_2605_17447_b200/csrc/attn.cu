@@ -407,13 +407,6 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
   for (int i = 0; i < 4; ++i) cp_off[i] = (2 * i + half) * 256 + ((c16 ^ row_swz(2 * i + half)) << 4);
   const uint64_t stream_policy = l2_evict_first_policy();
   const uint64_t keep_policy = LOGITS ? l2_policy_evict_last() : 0;   // logits: read back by the next kernel
-#ifdef FASTOCR_TRACE
-  if (a.trace != nullptr && lane == 0) {               // slot 2: the SM this CTA runs on
-    unsigned smid;
-    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-    a.trace[(blockIdx.x * kAttnWarps + warp) * 16 + 2] = smid + 1;
-  }
-#endif
 
   // ---- the CTA's range, one unit segment after the other --------------------------------------
   int u = first_unit;
@@ -437,6 +430,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
     wait_for_prior_grids();
     dependents_may_launch();
   }
+  FASTOCR_TRACE_MARK(2);                               // (debug builds) the wait, if any, is over
   // State that survives a segment boundary when the look-ahead stages of one segment have already
   // fetched the first blocks of the next (see `carry_next` below).
   uint32_t qb[8][2];                                   // B fragments of Q^T of the segment's unit
@@ -646,7 +640,7 @@ __global__ void __launch_bounds__(kThreads, kAttnCtasPerSm) attn_stream_kernel(c
       __syncwarp();                                    // every lane's K copies of this block have landed
       FASTOCR_TRACE_CLK(c_waited);
       FASTOCR_TRACE_ADD(trace_wait, c_waited, c_top);
-      if (j0 == tok0) { FASTOCR_TRACE_MARK(3); FASTOCR_TRACE_CYC(14); }
+      if (j0 == tok0 && seg_begin == r0) { FASTOCR_TRACE_MARK(3); FASTOCR_TRACE_CYC(14); }   // first data of the CTA's range
       const bool live = j0 < sg.n_tok;                 // the block holds at least one attended token
       // two accumulators (even / odd 16-dim steps): dependent MMA chains of four
       float sc[4] = {0.f, 0.f, 0.f, 0.f}, sc2[4] = {0.f, 0.f, 0.f, 0.f};

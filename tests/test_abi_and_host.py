@@ -38,6 +38,9 @@ def test_host_rules_agree_with_oracle():
         rho, gap = rnd.choice([0.05, 0.1, 0.2, 0.5, 1.0]), rnd.randint(0, 4)
         assert fo.focal_layers(r, rho, gap) == oracle.focal_layers(r, rho, gap)
     assert abs(fo.attn_flops(8, 36, 2048, 4096) - oracle.attn_flops(8, 36, 2048, 4096)) < 1.0
+    for b, l, h, s_, f, sk in ((8, 36, 2048, 4096, 4, 204.8), (4, 36, 2048, 8192, 3, 409.6), (64, 28, 3584, 8449, 2, 666), (1, 5, 64, 100, 0, 0)):
+        want = oracle.attn_flops_pruned(b, l, h, s_, f, sk)
+        assert abs(fo.attn_flops_pruned(b, l, h, s_, f, sk) - want) <= 1e-9 * want
 
 
 def test_product_does_not_import_the_oracle():

@@ -281,3 +281,26 @@ def test_layers_after_a_selection_with_empty_text_or_empty_selection(fo, ctx, pa
             else:
                 _check_out(out[l, b], oracle.sparse(*cases[l].seq(b), SCALE, base.vis_start[b], base.vis_len[b], sel, True))
     assert ctx.device_faults() == 0
+
+
+def test_a_run_of_pruned_layers_longer_than_one_launch_takes(fo, ctx):
+    """35 consecutive pruned layers on a carried set: the run is cut into a launch of 32 layers and one of 3
+    (the second starts while the first drains); every layer against the oracle."""
+    L = 35
+    spans = [(6, 300, 20), (3, 170, 41)]
+    cases, views, q_all = make_layer_stack(2200, spans, L)
+    base = cases[0]
+    ks = [oracle.kept_count(n, 0.1) for n in base.vis_len]
+    g = torch.Generator().manual_seed(4)
+    fix = torch.zeros(base.B, max(ks), dtype=torch.int32)
+    for b in range(base.B):
+        fix[b, :ks[b]] = torch.randperm(base.vis_len[b], generator=g)[:ks[b]].sort().values.int()
+    out = torch.full((L, base.B, base.H, 128), 7.0, dtype=torch.float32, device="cuda")
+    before = fo.launch_count()
+    assert fo.fastocr_decode_step(ctx, views, q_all.cuda(), out, [False] * L, torch.tensor(ks, dtype=torch.int32, device="cuda"),
+                                  fix.cuda(), True, max(base.vis_len))
+    assert fo.launch_count() - before == 2
+    for l in range(L):
+        for b in range(base.B):
+            _check_out(out[l, b], oracle.sparse(*cases[l].seq(b), SCALE, base.vis_start[b], base.vis_len[b], fix[b, :ks[b]], True))
+    assert ctx.device_faults() == 0
