@@ -304,3 +304,27 @@ def test_a_run_of_pruned_layers_longer_than_one_launch_takes(fo, ctx):
         for b in range(base.B):
             _check_out(out[l, b], oracle.sparse(*cases[l].seq(b), SCALE, base.vis_start[b], base.vis_len[b], fix[b, :ks[b]], True))
     assert ctx.device_faults() == 0
+
+
+@pytest.mark.parametrize("H,Hkv", [(3, 3), (4, 2), (16, 4), (8, 1)])
+def test_decode_step_other_group_sizes(fo, ctx, H, Hkv):
+    """GQA groups of 1, 2, 4 and 8 query heads per KV head through the whole step (runs of pruned layers as
+    one launch, a focal layer in between), paged cache, ragged batch."""
+    L = 5
+    spans = [(6, 300, 20), (0, 170, 41), (5, 64, 0)]
+    cases, views, q_all = make_layer_stack(2300 + H, spans, L, H=H, Hkv=Hkv, page_size=16, q_boost=1.5)
+    base = cases[0]
+    ks = [oracle.kept_count(n, 0.1) for n in base.vis_len]
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    fix = torch.full((base.B, max(ks)), -1, dtype=torch.int32, device="cuda")
+    have, f_last = False, [None] * base.B
+    for step in range(2):
+        out = torch.full((L, base.B, H, 128), 7.0, dtype=torch.float32, device="cuda")
+        have = fo.fastocr_decode_step(ctx, views, q_all.cuda(), out, [False, False, True, False, False], kd, fix, have, max(base.vis_len))
+        for b in range(base.B):
+            tr = oracle.decode_step([c.seq(b) for c in cases], [2], f_last[b], base.vis_start[b], base.vis_len[b], 0.1, SCALE, acc64=True)
+            for l in range(L):
+                _check_out(out[l, b], tr.outputs[l])
+            assert fix[b, :ks[b]].cpu().tolist() == tr.f_last.tolist()
+            f_last[b] = tr.f_last
+    assert ctx.device_faults() == 0
