@@ -121,6 +121,9 @@ class Workload:
         if cfg.page_size:
             table, self.num_pages = make_page_table(cfg.seed + rank, [self.S_stride] * B, cfg.page_size)
             self.block_table = table.to(device)
+        # all layers' caches in one allocation per tensor ([L] leading), so that a decode step's new rows go
+        # into every layer's cache with one scatter per tensor; layer l's cache is the view [l]
+        self.K_all = self.V_all = None
         for l in range(self.L):
             K, V = make_kv(cfg.seed, l, B, self.S_stride, self.Hkv, cfg.head_dim, device, seq_offset=self.seq_offset)
             for s in range(n_distinct):
@@ -130,6 +133,12 @@ class Workload:
             if cfg.page_size:
                 K = scatter_to_pages(K, [self.S_stride] * B, self.block_table.cpu(), self.num_pages, cfg.page_size)
                 V = scatter_to_pages(V, [self.S_stride] * B, self.block_table.cpu(), self.num_pages, cfg.page_size)
+            if self.K_all is None:
+                self.K_all = torch.empty((self.L,) + tuple(K.shape), dtype=K.dtype, device=device)
+                self.V_all = torch.empty_like(self.K_all)
+            self.K_all[l].copy_(K)
+            self.V_all[l].copy_(V)
+            K, V = self.K_all[l], self.V_all[l]
             self.K.append(K)
             self.V.append(V)
             if fo:
@@ -556,9 +565,9 @@ def main():
     if not args.no_e2e:
         q_host = w.q_all.cpu().pin_memory()                                         # [nd][L][B][H][d]
         rows = [w.flat_row(s) for s in range(w.nd)]                                 # step s appends position S0+s
-        flatK = [k.view(-1, w.Hkv, cfg.head_dim) for k in w.K]
-        flatV = [v.view(-1, w.Hkv, cfg.head_dim) for v in w.V]
-        newkv_host = torch.stack([torch.stack([torch.stack([flatK[l][rows[s]], flatV[l][rows[s]]]) for l in range(w.L)])
+        flatK = w.K_all.view(w.L, -1, w.Hkv, cfg.head_dim)                          # [L][rows][Hkv][d]
+        flatV = w.V_all.view(w.L, -1, w.Hkv, cfg.head_dim)
+        newkv_host = torch.stack([torch.stack([flatK[:, rows[s]], flatV[:, rows[s]]], dim=1)
                                   for s in range(w.nd)]).cpu().pin_memory()         # [nd][L][2][B][Hkv][d]
         out_host = torch.empty(out.shape, dtype=out.dtype).pin_memory()
         q_dev = torch.empty_like(w.q_all[0])
@@ -582,9 +591,8 @@ def main():
             if n_sl == 1:                               # everything in stream order
                 q_dev.copy_(q_host[s], non_blocking=True)
                 newkv_dev.copy_(newkv_host[s], non_blocking=True)
-                for l in range(w.L):
-                    flatK[l].index_copy_(0, rows[s], newkv_dev[l, 0])
-                    flatV[l].index_copy_(0, rows[s], newkv_dev[l, 1])
+                flatK.index_copy_(1, rows[s], newkv_dev[:, 0])
+                flatV.index_copy_(1, rows[s], newkv_dev[:, 1])
                 state["have"] = plans[0].run(q_dev, out, state["have"])
                 out_host.copy_(out, non_blocking=True)
                 return
@@ -596,9 +604,8 @@ def main():
                     ev_in[i].record(s_in)
             for i, (a, b) in enumerate(slices):
                 cur.wait_event(ev_in[i])
-                for l in range(a, b):                   # append the current token's K/V rows to every layer's cache
-                    flatK[l].index_copy_(0, rows[s], newkv_dev[l, 0])
-                    flatV[l].index_copy_(0, rows[s], newkv_dev[l, 1])
+                flatK[a:b].index_copy_(1, rows[s], newkv_dev[a:b, 0])      # append the current token's K/V rows to the
+                flatV[a:b].index_copy_(1, rows[s], newkv_dev[a:b, 1])      # caches of the slice's layers
                 state["have"] = plans[i].run(q_dev[a:b], out[a:b], state["have"])
                 ev_out[i].record(cur)
                 with torch.cuda.stream(s_out):
