@@ -171,6 +171,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   extern __shared__ __align__(16) uint32_t keys[];      // all keys of the sequence
   __shared__ float head_st[2 * kTopkMaxHeads];          // scoring mode: per head (max, 1 / sum)
   __shared__ uint32_t hist[kTopkBins];
+  __shared__ uint32_t hist_first[kTopkBins];            // scoring mode: first-digit histogram of the CTA's own slice, built while scoring
   __shared__ uint32_t warp_gt[kTopkWarps], warp_eq[kTopkWarps];
   __shared__ uint32_t sel_prefix, sel_remaining;
 
@@ -194,12 +195,14 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   const int n_loc = hi_i - lo_i;
   // A peer's shared memory may be written only once that CTA is known to be running: every CTA
   // signals here and checks for the others just before its first remote store.
-  if (C > 1) cluster.barrier_arrive();
   hist[2 * tid] = hist[2 * tid + 1] = 0u;
+  hist_first[2 * tid] = hist_first[2 * tid + 1] = 0u;
   if (tid == 0) {
     sel_prefix = 0u;
     sel_remaining = static_cast<uint32_t>(k);
   }
+  __syncthreads();                                      // the histograms are clear before anybody counts into them
+  if (C > 1) cluster.barrier_arrive();
   if (logits == nullptr) {
     const float* sp = scores + static_cast<int64_t>(b) * n_stride;
     for (int i = tid; i < N; i += kTopkThreads) keys[i] = score_key(sp[i]);
@@ -207,7 +210,11 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
     // The CTA scores its slice and writes the keys into every CTA's copy of the key array
     // (distributed shared memory). Before the first remote store all threads, together, make sure
     // that the peers are running (the second half of the barrier begun above).
+    // The first radix pass's histogram (top 11 bits) is counted here, key by key as the scores are formed
+    // (the threads spend this phase waiting for logits anyway), each CTA for its own slice; the pass itself
+    // then only adds up the CTAs' histograms instead of walking all keys.
     auto all_copies = [&](int j, uint32_t key) {
+      atomicAdd(&hist_first[key >> 21], 1u);
       for (int r = 0; r < C; ++r) cluster.map_shared_rank(keys, r)[lo_i + j] = key;
     };
     score_slice(logits, stats, head_st, b, num_q_heads, n_stride_logits, lo_i, n_loc, per_cta, drop_logits,
@@ -217,6 +224,8 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
                 all_copies,
                 [&](int j0, const uint32_t* kq, int count) {
                   if (count == 4) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) atomicAdd(&hist_first[kq[t] >> 21], 1u);
                     for (int r = 0; r < C; ++r)
                       *reinterpret_cast<uint4*>(cluster.map_shared_rank(keys, r) + lo_i + j0) = make_uint4(kq[0], kq[1], kq[2], kq[3]);
                   } else {
@@ -239,7 +248,8 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
     const uint32_t hi_mask = pass == 0 ? 0u : (0xffffffffu << (pass == 1 ? 21 : 10));
     const uint32_t prefix = sel_prefix;
     const uint32_t remaining = sel_remaining;
-    for (int base = warp * 32; base < N; base += kTopkThreads) {   // warp-uniform trip count
+    const bool counted = pass == 0 && logits != nullptr;   // the first digit was counted while scoring
+    for (int base = warp * 32; base < N && !counted; base += kTopkThreads) {   // warp-uniform trip count
       const int i = base + lane;
       const uint32_t key = i < N ? keys[i] : 0u;
       const bool in = i < N && (key & hi_mask) == prefix;
@@ -258,9 +268,18 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
     }
     __syncthreads();
     const int d0 = kTopkBins - 1 - 2 * tid, d1 = d0 - 1;   // bins in descending digit order
-    const uint32_t c0 = hist[d0], c1 = hist[d1];
+    uint32_t c0 = hist[d0], c1 = hist[d1];
     hist[d0] = 0u;                                      // ready for the next pass
     hist[d1] = 0u;
+    if (counted) {                                      // every CTA of the cluster counted its slice (complete since the barrier above)
+      c0 = c1 = 0u;
+      for (int r = 0; r < C; ++r) {
+        const uint32_t* h = C > 1 ? cluster.map_shared_rank(hist_first, r) : hist_first;
+        c0 += h[d0];
+        c1 += h[d1];
+      }
+      if (C > 1) cluster.barrier_arrive();              // (waited for at the end: no CTA leaves while a peer may still read its histogram)
+    }
     const uint32_t local = c0 + c1;
     uint32_t incl = local;
 #pragma unroll
@@ -399,6 +418,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
       eq_run += __popc(m_eq);
     }
   }
+  if (C > 1 && logits != nullptr) cluster.barrier_wait();
   TOPK_STAMP(6);
 }
 
@@ -450,10 +470,16 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_split_kernel(const f
     const float* sp = scores + static_cast<int64_t>(b) * n_stride + lo_i;
     for (int i = tid; i < n_loc; i += kTopkThreads) keys[i] = score_key(sp[i]);
   } else {
+    // (the first pass's histogram is counted on the way, as in select_topk_kernel; score_slice has a block
+    // barrier between the clearing above and the first key)
     score_slice(logits, stats, head_st, b, num_q_heads, n_stride_logits, lo_i, n_loc, per_cta, drop_logits,
                 []() {},
-                [&](int j, uint32_t key) { keys[j] = key; },
+                [&](int j, uint32_t key) {
+                  atomicAdd(&hist[0][key >> 21], 1u);
+                  keys[j] = key;
+                },
                 [&](int j0, const uint32_t* kq, int count) {
+                  for (int t = 0; t < count; ++t) atomicAdd(&hist[0][kq[t] >> 21], 1u);
                   if (count == 4) {
                     *reinterpret_cast<uint4*>(keys + j0) = make_uint4(kq[0], kq[1], kq[2], kq[3]);
                   } else {
@@ -475,7 +501,8 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_split_kernel(const f
     const uint32_t hi_mask = pass == 0 ? 0u : (0xffffffffu << (pass == 1 ? 21 : 10));
     const uint32_t prefix = sel_prefix;
     const uint32_t remaining = sel_remaining;
-    for (int base = warp * 32; base < n_loc; base += kTopkThreads) {   // warp-uniform trip count
+    const bool counted = pass == 0 && logits != nullptr;   // the first digit was counted while scoring
+    for (int base = warp * 32; base < n_loc && !counted; base += kTopkThreads) {   // warp-uniform trip count
       const int i = base + lane;
       const uint32_t key = i < n_loc ? keys[i] : 0u;
       const bool in = i < n_loc && (key & hi_mask) == prefix;
