@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-slices", type=int, default=4, help="layer slices per end-to-end step (copies of one overlap the arithmetic of the next)")
     ap.add_argument("--workload", default="cfg4", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--N", type=int, default=8192, help="image tokens (cfg4 only)")
     ap.add_argument("--batch", type=int, default=64, help="sequences (cfg4 only)")
@@ -576,7 +577,7 @@ def main():
         # The step runs as a few slices of consecutive layers (one library call each), so that the
         # copies overlap the arithmetic: slice i's inputs arrive while slice i - 1 computes, its
         # outputs leave while slice i + 1 computes. Steps themselves stay serial (autoregressive).
-        n_sl = 4 if (w.L >= 8 and w.B * w.Hkv >= 64) else 1   # small batches are bound by the host's calls: one slice
+        n_sl = args.e2e_slices if (w.L >= 8 and w.B * w.Hkv >= 64) else 1   # small batches are bound by the host's calls: one slice
         cuts = [round(i * w.L / n_sl) for i in range(n_sl + 1)]
         slices = list(zip(cuts[:-1], cuts[1:]))
         plans = [fo.StepPlan(w.ctx, w.views[a:b], is_focal[a:b], w.k_d, w.fix, max(w.vis_len), w.max_kept) for a, b in slices]
