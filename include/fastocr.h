@@ -202,11 +202,30 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
  *       the previous step. `fixation` still receives every focal layer's own selection, so that what
  *       is carried to the next step is the deepest focal layer's set as in Algorithm 1. The union
  *       lives in the context's workspace; max_kept must bound text + union size.
+ *   scores_exchange  for a cache that is sharded by KV head over several processes (each holds
+ *       num_q_heads / n query heads and their KV heads of every sequence): the focal score of
+ *       Section 3.1.1 averages the attention weight over ALL heads, so the per-rank partial
+ *       averages must be added up before the selection; nothing else in the step crosses ranks.
+ *       When the callback is set, a focal layer runs as: full-cache pass over the local heads,
+ *       local score = mean over the local heads, scores_exchange(...), selection from the exchanged
+ *       scores. The callback is called on the host, between those launches, once per focal layer
+ *       (the fallback at layer 0 included), in layer order; it must enqueue on `stream` an
+ *       in-place sum over the ranks of scores[batch][n_stride] (device fp32, the context's
+ *       workspace; entries beyond a sequence's vis_len, and rows of sequences for which the layer
+ *       is not focal, hold garbage and may be summed or not) and return 0, or non-zero on failure
+ *       (the step then returns FASTOCR_ERR_CUDA with nothing further launched). All ranks must run
+ *       the same schedule (same focal sets, same has_fixation) and see the same k and spans; with
+ *       equal head counts per rank the sum of the local means ranks the tokens as the global mean
+ *       does, and every rank then selects the same set from identical scores.
  */
+typedef int (*fastocr_scores_exchange_fn)(float* scores, int32_t batch, int32_t n_stride, int32_t layer,
+                                          void* stream, void* user);
 typedef struct fastocr_step_options {
   const uint8_t* is_focal_seq;     /* host uint8 [L][B], or NULL   */
   const uint8_t* is_focal_seq_dev; /* device uint8 [L][B], or NULL */
   int32_t union_sets;              /* 0 = Algorithm 1              */
+  fastocr_scores_exchange_fn scores_exchange;   /* NULL = all heads are local */
+  void* scores_exchange_user;      /* passed through to the callback */
 } fastocr_step_options;
 fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
                                       const void* q, void* out, int out_is_fp32, const uint8_t* is_focal,

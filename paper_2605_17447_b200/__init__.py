@@ -6,4 +6,4 @@ from .api import (  # noqa: F401
     fastocr_dense_decode_attn, fastocr_focal_scores, fastocr_select_topk, fastocr_sparse_decode_attn,
     fastocr_decode_step, fastocr_warmup_step, fastocr_sparse_decode_attn_noalloc, noalloc_device_faults, StepPlan, PROF_CLASSES,
 )
-from .sharding import shard_sequences  # noqa: F401
+from .sharding import make_scores_exchange, mean_ratio_over_ranks, shard_heads, shard_sequences  # noqa: F401

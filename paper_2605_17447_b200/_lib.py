@@ -22,8 +22,13 @@ class KVViewStruct(C.Structure):
     ]
 
 
+# int (*)(float* scores, int32 batch, int32 n_stride, int32 layer, void* stream, void* user)
+ScoresExchangeFn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p)
+
+
 class StepOptionsStruct(C.Structure):
-    _fields_ = [("is_focal_seq", C.c_void_p), ("is_focal_seq_dev", C.c_void_p), ("union_sets", C.c_int32)]
+    _fields_ = [("is_focal_seq", C.c_void_p), ("is_focal_seq_dev", C.c_void_p), ("union_sets", C.c_int32),
+                ("scores_exchange", ScoresExchangeFn), ("scores_exchange_user", C.c_void_p)]
 
 
 class LimitsStruct(C.Structure):

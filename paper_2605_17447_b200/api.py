@@ -226,16 +226,40 @@ def fastocr_sparse_decode_attn_noalloc(kv: KVView, q: torch.Tensor, idx: torch.T
         raise FastOCRError(rc, lib.fastocr_noalloc_last_error().decode())
 
 
+class _DeviceFloats:
+    """A span of device fp32 memory owned by the library, described through the CUDA array interface."""
+
+    def __init__(self, ptr: int, shape):
+        self.__cuda_array_interface__ = {"shape": tuple(int(x) for x in shape), "typestr": "<f4", "data": (int(ptr), False),
+                                         "strides": None, "version": 2}
+
+
 class _StepArgs:
     """Marshalled arguments of fastocr_decode_step_ex that do not change between steps."""
 
     def __init__(self, layers: Sequence[KVView], is_focal, k: torch.Tensor, fixation: torch.Tensor, max_vis_len: int,
-                 max_kept: int, union_sets: bool):
+                 max_kept: int, union_sets: bool, scores_exchange=None):
         self.L = len(layers)
         self.keep = (list(layers), k, fixation)
         self.arr = (_lib.KVViewStruct * self.L)(*[kv.struct() for kv in layers])
         focal = np.ascontiguousarray(np.asarray(is_focal, dtype=np.uint8))
         self.opt = _lib.StepOptionsStruct(None, None, int(bool(union_sets)))
+        self.exchange_error = None
+        if scores_exchange is not None:
+            device = k.device
+
+            def hook(ptr, batch, n_stride, layer, stream, user):
+                # the library's score workspace as a tensor (no copy); the callable enqueues on the current stream
+                try:
+                    scores = torch.as_tensor(_DeviceFloats(ptr, (batch, n_stride)), device=device)
+                    scores_exchange(scores, layer)
+                    return 0
+                except BaseException as e:      # must not propagate through the C frames
+                    self.exchange_error = e
+                    return 1
+
+            self._hook = _lib.ScoresExchangeFn(hook)   # kept alive with the arguments
+            self.opt.scores_exchange = self._hook
         self.focal = focal
         self.focal_ptr = focal.ctypes.data
         if focal.ndim == 2:                       # per-sequence focal layer sets [L][B]: host copy + device copy
@@ -254,10 +278,14 @@ class _StepArgs:
         self.have = C.c_int(0)
 
     def run(self, ctx: Context, q: torch.Tensor, out: torch.Tensor, has_fixation: bool, stream=None) -> bool:
-        ctx.check(ctx._lib.fastocr_decode_step_ex(ctx._h, self.L, self.arr, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()),
-                                                  int(out.dtype == torch.float32), self.focal_ptr, self.k, self.fix,
-                                                  self.k_stride, int(bool(has_fixation)), self.max_vis, self.max_kept,
-                                                  C.byref(self.have), C.byref(self.opt), _stream(stream)))
+        rc = ctx._lib.fastocr_decode_step_ex(ctx._h, self.L, self.arr, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()),
+                                             int(out.dtype == torch.float32), self.focal_ptr, self.k, self.fix,
+                                             self.k_stride, int(bool(has_fixation)), self.max_vis, self.max_kept,
+                                             C.byref(self.have), C.byref(self.opt), _stream(stream))
+        if self.exchange_error is not None:             # what the exchange callable raised, not the library's summary of it
+            e, self.exchange_error = self.exchange_error, None
+            raise e
+        ctx.check(rc)
         return bool(self.have.value)
 
 
@@ -268,11 +296,16 @@ def noalloc_device_faults() -> int:
 
 def fastocr_decode_step(ctx: Context, layers: Sequence[KVView], q: torch.Tensor, out: torch.Tensor,
                         is_focal, k: torch.Tensor, fixation: torch.Tensor, has_fixation: bool,
-                        max_vis_len: int, max_kept: int = 0, union_sets: bool = False, stream=None) -> bool:
+                        max_vis_len: int, max_kept: int = 0, union_sets: bool = False, stream=None,
+                        scores_exchange=None) -> bool:
     """q/out: [L][B][H][128]. is_focal: [L] (one focal layer set for the batch) or [L][B] (per-sequence
-    sets). Returns whether `fixation` is valid after the step."""
+    sets). scores_exchange: for heads sharded over processes, a callable (scores [B][n_stride] device
+    fp32, layer) that sums the scores over the ranks in place on the current stream (see
+    sharding.make_scores_exchange); the step must then run on the current stream. Returns whether
+    `fixation` is valid after the step."""
     _dev(q, torch.bfloat16, "q")
-    return _StepArgs(layers, is_focal, k, fixation, max_vis_len, max_kept, union_sets).run(ctx, q, out, has_fixation, stream)
+    return _StepArgs(layers, is_focal, k, fixation, max_vis_len, max_kept, union_sets, scores_exchange).run(
+        ctx, q, out, has_fixation, stream)
 
 
 def fastocr_warmup_step(ctx: Context, layers: Sequence[KVView], q: torch.Tensor, out: torch.Tensor,
@@ -291,10 +324,11 @@ class StepPlan:
     (the per-step Python cost is then a single foreign call)."""
 
     def __init__(self, ctx: Context, layers: Sequence[KVView], is_focal, k: torch.Tensor,
-                 fixation: torch.Tensor, max_vis_len: int, max_kept: int = 0, union_sets: bool = False):
+                 fixation: torch.Tensor, max_vis_len: int, max_kept: int = 0, union_sets: bool = False,
+                 scores_exchange=None):
         self.ctx = ctx
         self.L = len(layers)
-        self._args = _StepArgs(layers, is_focal, k, fixation, max_vis_len, max_kept, union_sets)
+        self._args = _StepArgs(layers, is_focal, k, fixation, max_vis_len, max_kept, union_sets, scores_exchange)
 
     def run(self, q: torch.Tensor, out: torch.Tensor, has_fixation: bool, stream=None) -> bool:
         return self._args.run(self.ctx, q, out, has_fixation, stream)

@@ -550,6 +550,7 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
   const uint8_t* focal_seq = opt != nullptr ? opt->is_focal_seq : nullptr;           // host [L][B]
   const uint8_t* focal_seq_dev = opt != nullptr ? opt->is_focal_seq_dev : nullptr;   // the same on the device
   const bool unite = opt != nullptr && opt->union_sets != 0;
+  const fastocr_scores_exchange_fn exchange = opt != nullptr ? opt->scores_exchange : nullptr;
   if (num_layers <= 0 || layers == nullptr || q == nullptr || out == nullptr || (is_focal == nullptr && focal_seq == nullptr) ||
       k == nullptr || fixation == nullptr)
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL pointer or num_layers <= 0");
@@ -668,13 +669,20 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
       // attention kernel lies in between, that kernel waited for the selection before it let
       // anything else start, so this launch may stream at once, beside the draining pruned pass.
       // The selection kernel forms the scores from the logits itself (no score array, one launch
-      // less) unless there are more heads than it has room for.
+      // less) unless there are more heads than it has room for, or the scores are to be summed over
+      // ranks first (heads sharded over processes).
       const bool chained = prev != kOther && overlap;
-      const bool fused = layers[l].num_q_heads <= fastocr::kTopkMaxHeads;
+      const bool fused = layers[l].num_q_heads <= fastocr::kTopkMaxHeads && exchange == nullptr;
       st = dense_impl(ctx, &layers[l], ql, ol, out_is_fp32, fused ? nullptr : ctx->scores, ctx->lim.max_vis_len, max_vis_len,
                       !chained ? fastocr::kWaitAtStart : (prev == kAttention ? fastocr::kWaitBeforeWrites : fastocr::kWaitAfterSetup),
                       s, fused, nullptr, fallback ? nullptr : mask, 1);
       if (st != FASTOCR_OK) return st;
+      if (exchange != nullptr) {
+        // heads sharded over processes: the local partial scores are added up over the ranks (the
+        // caller's collective, enqueued on this stream) before anything is selected
+        if (exchange(ctx->scores, B, ctx->lim.max_vis_len, l, stream, opt->scores_exchange_user) != 0)
+          return fail(ctx, FASTOCR_ERR_CUDA, "the scores exchange of layer %d failed", l);
+      }
       {
         ProfScope p(ctx, FASTOCR_PROF_TOPK, s);
         FASTOCR_TRY_CUDA(fastocr::launch_select_topk(ctx->scores, ctx->lim.max_vis_len, layers[l].vis_len, k, B,

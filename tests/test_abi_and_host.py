@@ -87,3 +87,67 @@ def test_shard_sequences_edges():
     assert shard_sequences(64, 3, 8) == (24, 32)
     with pytest.raises(ValueError):
         shard_sequences(4, 2, 2)
+
+
+_GLOO_HEADS_WORKER = r"""
+import os, sys, math, torch, torch.distributed as dist
+sys.path.insert(0, os.environ["FASTOCR_ROOT"])
+import oracle
+from paper_2605_17447_b200.sharding import shard_heads, make_scores_exchange, mean_ratio_over_ranks
+dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%s" % os.environ["PORT"],
+                        rank=int(os.environ["RANK"]), world_size=int(os.environ["WORLD_SIZE"]))
+rank, world = dist.get_rank(), dist.get_world_size()
+# one sequence, 8 query heads over 4 KV heads; the same seeded tensors on every rank
+H, Hkv, d, vs, N, T = 8, 4, 128, 5, 300, 40
+S = vs + N + T
+g = torch.Generator().manual_seed(77)
+K = torch.randn(S, Hkv, d, generator=g).bfloat16()
+q = (torch.randn(H, d, generator=g) * 1.5).bfloat16()
+sm = 1 / math.sqrt(d)
+want_scores, want_mass = oracle.scores(q, K, sm, vs, N)            # all heads
+q0, q1, k0, k1 = shard_heads(H, Hkv, rank, world)
+assert (q1 - q0) * world == H and (k1 - k0) * world == Hkv
+local, mass = oracle.scores(q[q0:q1], K[:, k0:k1].contiguous(), sm, vs, N)   # this rank's heads only
+summed = local.clone().view(1, N)
+make_scores_exchange()(summed, 0)                                   # the product's exchange, over gloo
+# the sum of the local means is world x the mean over all heads (up to rounding): same ranking
+assert torch.allclose(summed[0] / world, want_scores, rtol=2e-6, atol=1e-9), (summed[0] / world - want_scores).abs().max()
+k = 15
+got, want = set(oracle.topk(summed[0], k).tolist()), set(oracle.topk(want_scores, k).tolist())
+if got != want:                                                     # only tokens tied with the k-th score to rounding may differ
+    kth = torch.sort(want_scores, descending=True).values[k - 1].item()
+    for i in got ^ want:
+        assert abs(want_scores[i].item() - kth) <= 1e-5 * abs(kth), (i, want_scores[i].item(), kth)
+# every rank ends with the same bits, hence the same selection
+mine = summed.clone(); other = [torch.empty_like(mine) for _ in range(world)]
+dist.all_gather(other, mine)
+assert all(torch.equal(o, mine) for o in other)
+r = mean_ratio_over_ranks(torch.tensor([[mass]], dtype=torch.float32))
+assert abs(r.item() - want_mass) <= 1e-5
+dist.barrier(); dist.destroy_process_group()
+"""
+
+
+def test_head_sharding_world_size_two_gloo(tmp_path):
+    """Heads sharded over two ranks: the exchanged local score means select what the all-head scores
+    select (Section 3.1.1 averages over all heads), identically on both ranks."""
+    import socket
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    script = tmp_path / "h.py"
+    script.write_text(_GLOO_HEADS_WORKER)
+    procs = []
+    for r in range(2):
+        env = dict(os.environ, RANK=str(r), WORLD_SIZE="2", PORT=str(port), FASTOCR_ROOT=ROOT)
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env))
+    for p in procs:
+        assert p.wait(timeout=180) == 0
+
+
+def test_shard_heads_edges():
+    from paper_2605_17447_b200.sharding import shard_heads
+    assert [shard_heads(64, 8, r, 4) for r in range(4)] == [(0, 16, 0, 2), (16, 32, 2, 4), (32, 48, 4, 6), (48, 64, 6, 8)]
+    assert shard_heads(28, 4, 0, 1) == (0, 28, 0, 4)
+    with pytest.raises(ValueError):
+        shard_heads(28, 4, 0, 3)        # 4 KV heads do not divide over 3 ranks
+    with pytest.raises(ValueError):
+        shard_heads(30, 4, 0, 2)

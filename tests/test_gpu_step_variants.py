@@ -328,3 +328,157 @@ def test_decode_step_other_group_sizes(fo, ctx, H, Hkv):
             assert fix[b, :ks[b]].cpu().tolist() == tr.f_last.tolist()
             f_last[b] = tr.f_last
     assert ctx.device_faults() == 0
+
+
+def _head_shard(cases, r, world):
+    """Rank r's share of a layer stack: its KV heads (and the query heads that read them) of every layer."""
+    from harness import Case
+    import paper_2605_17447_b200 as f
+    base = cases[0]
+    q0, q1, k0, k1 = f.shard_heads(base.H, base.Hkv, r, world)
+    local, views, shared = [], [], None
+    for c in cases:
+        lc = Case(c.B, q1 - q0, k1 - k0, c.seq_len, c.vis_start, c.vis_len, c.K[:, :, k0:k1].contiguous(),
+                  c.V[:, :, k0:k1].contiguous(), c.q[:, q0:q1].contiguous(), c.page_size, c.block_table, c.num_pages)
+        v = lc.device_view()
+        if shared is None:
+            shared = (v.seq_len, v.vis_start, v.vis_len)
+        views.append(f.KVView(v.k, v.v, shared[0], shared[1], shared[2], q1 - q0, max(c.seq_len), SCALE,
+                              block_table=v.block_table if c.page_size else None))
+        local.append(lc)
+    return local, views, torch.stack([c.q for c in local]), (q0, q1)
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_decode_step_with_heads_sharded_over_two_ranks(fo, paged):
+    """Heads sharded over two processes, emulated one rank after the other on one GPU: each rank runs the
+    whole step over its 14 query / 2 KV heads, and at every focal layer its exchange callback adds the other
+    rank's local scores (what the all-reduce would deliver) before the selection. Both ranks must select
+    the oracle's all-head sets and produce the oracle's outputs for their heads."""
+    L, world = 5, 2
+    spans = [(6, 300, 20), (3, 170, 41), (9, 512, 7)]
+    focal = [1, 3]
+    cases, _, _ = make_layer_stack(2500, spans, L, page_size=16 if paged else 0, q_boost=1.5)
+    base = cases[0]
+    ks = [oracle.kept_count(n, 0.1) for n in base.vis_len]
+    n_max = max(base.vis_len)
+    ranks = []
+    for r in range(world):
+        local, views, q_all, (q0, q1) = _head_shard(cases, r, world)
+        c = fo.Context(max_batch=base.B, num_q_heads=q1 - q0, num_kv_heads=base.Hkv // world, max_seq_len=max(base.seq_len),
+                       max_vis_len=n_max + 13)
+        # what this rank would contribute to the exchange at each layer: the mean over its heads
+        part = torch.zeros(L, base.B, n_max, dtype=torch.float32, device="cuda")
+        scratch = torch.empty(base.B, q1 - q0, 128, dtype=torch.float32, device="cuda")
+        for l in range(L):
+            fo.fastocr_dense_decode_attn(c, views[l], q_all[l].cuda(), scratch, scores_out=part[l])
+        ranks.append(dict(ctx=c, views=views, q=q_all.cuda(), heads=(q0, q1), part=part,
+                          fix=torch.full((base.B, max(ks)), -1, dtype=torch.int32, device="cuda"), have=False, calls=[]))
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    f_last = [None] * base.B
+    for step in range(2):
+        traces = [oracle.decode_step([c.seq(b) for c in cases], focal, f_last[b], base.vis_start[b], base.vis_len[b], 0.1, SCALE,
+                                     acc64=True) for b in range(base.B)]
+        for r, me in enumerate(ranks):
+            other = ranks[1 - r]
+
+            def exchange(scores, layer, me=me, other=other):
+                assert scores.shape == (base.B, n_max + 13) and scores.dtype == torch.float32 and scores.is_cuda
+                me["calls"].append(layer)
+                # the library's local scores are what the stand-alone call gave for this rank
+                for b in range(base.B):
+                    assert torch.equal(scores[b, :base.vis_len[b]], me["part"][layer, b, :base.vis_len[b]])
+                scores[:, :n_max] += other["part"][layer]
+
+            out = torch.full((L, base.B, me["heads"][1] - me["heads"][0], 128), 7.0, dtype=torch.float32, device="cuda")
+            me["have"] = fo.fastocr_decode_step(me["ctx"], me["views"], me["q"], out, [l in focal for l in range(L)], kd, me["fix"],
+                                                me["have"], n_max, scores_exchange=exchange)
+            assert me["have"]
+            for b in range(base.B):
+                for l in range(L):
+                    _check_out(out[l, b], traces[b].outputs[l][me["heads"][0]:me["heads"][1]])
+                assert me["fix"][b, :ks[b]].cpu().tolist() == traces[b].f_last.tolist()
+            assert me["ctx"].device_faults() == 0
+        assert torch.equal(ranks[0]["fix"], ranks[1]["fix"])
+        for b in range(base.B):
+            f_last[b] = traces[b].f_last
+    # one exchange per focal layer, in layer order; the first step's fallback at layer 0 included
+    assert ranks[0]["calls"] == [0, 1, 3, 1, 3] and ranks[1]["calls"] == ranks[0]["calls"]
+    for me in ranks:
+        me["ctx"].close()
+
+
+def test_a_failing_scores_exchange_ends_the_step(fo, ctx):
+    """What the exchange callable raises reaches the caller, and nothing is selected after it."""
+    L = 3
+    cases, views, q_all = make_layer_stack(2600, [(4, 200, 10)], L)
+    base = cases[0]
+    kd = torch.tensor([20], dtype=torch.int32, device="cuda")
+    fix = torch.full((1, 20), -1, dtype=torch.int32, device="cuda")
+    out = torch.empty(L, 1, 28, 128, dtype=torch.float32, device="cuda")
+
+    def boom(scores, layer):
+        raise RuntimeError("exchange failed on purpose (host side)")
+
+    with pytest.raises(RuntimeError, match="exchange failed on purpose"):
+        fo.fastocr_decode_step(ctx, views, q_all.cuda(), out, [False, True, False], kd, fix, False, base.vis_len[0], scores_exchange=boom)
+    torch.cuda.synchronize()
+    assert fix.cpu().tolist() == [[-1] * 20]
+    # the context is usable afterwards
+    assert fo.fastocr_decode_step(ctx, views, q_all.cuda(), out, [False, True, False], kd, fix, False, base.vis_len[0])
+    tr = oracle.decode_step([c.seq(0) for c in cases], [1], None, base.vis_start[0], base.vis_len[0], 0.1, SCALE, acc64=True)
+    assert fix[0].cpu().tolist() == tr.f_last.tolist()
+
+
+_NCCL_WORKER = r"""
+import os, sys, torch, torch.distributed as dist
+root = os.environ["FASTOCR_ROOT"]
+sys.path.insert(0, root); sys.path.insert(0, os.path.join(root, "tests"))
+import oracle
+import paper_2605_17447_b200 as fo
+from harness import SCALE, make_layer_stack
+torch.cuda.set_device(0)
+dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%s" % os.environ["PORT"], rank=0, world_size=1)
+L, spans, focal = 4, [(6, 300, 20), (3, 170, 41)], [2]
+cases, views, q_all = make_layer_stack(2700, spans, L, q_boost=1.5)
+base = cases[0]
+ks = [oracle.kept_count(n, 0.1) for n in base.vis_len]
+kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+fix = torch.full((base.B, max(ks)), -1, dtype=torch.int32, device="cuda")
+ctx = fo.Context(max_batch=base.B, num_q_heads=28, num_kv_heads=4, max_seq_len=max(base.seq_len), max_vis_len=max(base.vis_len))
+out = torch.empty(L, base.B, 28, 128, dtype=torch.float32, device="cuda")
+have, f_last = False, [None] * base.B
+for step in range(2):
+    have = fo.fastocr_decode_step(ctx, views, q_all.cuda(), out, [l in focal for l in range(L)], kd, fix, have, max(base.vis_len),
+                                  scores_exchange=fo.make_scores_exchange())
+    torch.cuda.synchronize()
+    for b in range(base.B):
+        tr = oracle.decode_step([c.seq(b) for c in cases], focal, f_last[b], base.vis_start[b], base.vis_len[b], 0.1, SCALE, acc64=True)
+        for l in range(L):
+            assert float((out[l, b].cpu() - tr.outputs[l]).abs().max()) <= 1e-4
+        assert fix[b, :ks[b]].cpu().tolist() == tr.f_last.tolist()
+        f_last[b] = tr.f_last
+ratio = torch.tensor([[0.25, 0.5]], device="cuda")
+assert fo.mean_ratio_over_ranks(ratio).cpu().tolist() == [[0.25, 0.5]]
+assert ctx.device_faults() == 0
+ctx.close()
+dist.destroy_process_group()
+print("ok")
+"""
+
+
+def test_scores_exchange_over_nccl_single_rank(tmp_path):
+    """The exchange helper as a user would pass it, over the NCCL backend (one rank: the only size one GPU
+    allows): the library's score workspace reaches torch.distributed as a tensor, the collective is ordered
+    between the library's launches on the current stream, and the step matches the oracle."""
+    import os
+    import socket
+    import subprocess
+    import sys
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    script = tmp_path / "n.py"
+    script.write_text(_NCCL_WORKER)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, PORT=str(port), FASTOCR_ROOT=root, NCCL_NVLS_ENABLE="0")
+    p = subprocess.run([sys.executable, str(script)], env=env, capture_output=True, text=True, timeout=300)
+    assert p.returncode == 0 and p.stdout.strip().endswith("ok"), p.stdout[-2000:] + p.stderr[-4000:]
