@@ -77,6 +77,11 @@ typedef struct fastocr_limits {
  * The image tokens of sequence b occupy the contiguous position span
  * [vis_start[b], vis_start[b] + vis_len[b]); every other position is text
  * (system, prompt, generated and the current token) and is always attended.
+ * One kernel launch covers up to 512 (sequence, KV head) pairs; a larger batch is processed by
+ * every entry point as chunks of whole sequences, launch after launch on the stream (sequences
+ * are independent of one another, so the results are those of one call; in a decode step each
+ * chunk runs all its layers before the next chunk starts, and a scores_exchange callback is
+ * called once per chunk and focal layer).
  */
 typedef struct fastocr_kv_view {
   int32_t batch;        /* B                                                                     */
@@ -209,7 +214,7 @@ fastocr_status fastocr_decode_step(fastocr_ctx* ctx, int32_t num_layers, const f
  *       When the callback is set, a focal layer runs as: full-cache pass over the local heads,
  *       local score = mean over the local heads, scores_exchange(...), selection from the exchanged
  *       scores. The callback is called on the host, between those launches, once per focal layer
- *       (the fallback at layer 0 included), in layer order; it must enqueue on `stream` an
+ *       (the fallback at layer 0 included; per chunk of the batch, see fastocr_kv_view), in layer order; it must enqueue on `stream` an
  *       in-place sum over the ranks of scores[batch][n_stride] (device fp32, the context's
  *       workspace; entries beyond a sequence's vis_len, and rows of sequences for which the layer
  *       is not focal, hold garbage and may be summed or not) and return 0, or non-zero on failure

@@ -111,8 +111,8 @@ fastocr_status check_view(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "seq_stride_tokens < max_seq_len");
   }
   if (!(kv->sm_scale > 0.f) || !std::isfinite(kv->sm_scale)) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "sm_scale must be positive");
-  if (static_cast<int64_t>(kv->batch) * kv->num_kv_heads > fastocr::kMaxUnits)
-    return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "batch x num_kv_heads exceeds %d", fastocr::kMaxUnits);
+  if (kv->num_kv_heads > fastocr::kMaxUnits)
+    return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "num_kv_heads exceeds %d", fastocr::kMaxUnits);
   if (kv->batch > ctx->lim.max_batch || kv->num_q_heads > ctx->lim.num_q_heads ||
       kv->num_kv_heads > ctx->lim.num_kv_heads || kv->max_seq_len > ctx->lim.max_seq_len)
     return fail(ctx, FASTOCR_ERR_WORKSPACE, "view (B=%d H=%d Hkv=%d S<=%d) exceeds the context limits (B=%d H=%d Hkv=%d S<=%d)",
@@ -370,6 +370,30 @@ fastocr_status check_scores_args(fastocr_ctx* ctx, const fastocr_kv_view* kv, co
   return FASTOCR_OK;
 }
 
+// A launch covers at most kMaxUnits (sequence, KV head) pairs: larger batches run as chunks of whole
+// sequences, one after the other on the stream (sequences are independent of one another).
+int chunk_sequences(const fastocr_kv_view* kv) {
+  const int per = fastocr::kMaxUnits / kv->num_kv_heads;
+  return kv->batch <= per ? kv->batch : per;
+}
+
+// sequences [b0, b0 + nb) of a view
+fastocr_kv_view sub_view(const fastocr_kv_view& v, int b0, int nb) {
+  fastocr_kv_view s = v;
+  s.batch = nb;
+  if (v.page_size == 0) {
+    const int64_t off = static_cast<int64_t>(b0) * v.seq_stride_tokens * v.num_kv_heads * fastocr::kHeadDim * 2;
+    s.k = static_cast<const char*>(v.k) + off;
+    if (v.v != nullptr) s.v = static_cast<const char*>(v.v) + off;
+  } else {
+    s.block_table = v.block_table + static_cast<int64_t>(b0) * v.max_pages;
+  }
+  s.seq_len = v.seq_len + b0;
+  s.vis_start = v.vis_start + b0;
+  s.vis_len = v.vis_len + b0;
+  return s;
+}
+
 }  // namespace
 
 extern "C" {
@@ -496,8 +520,18 @@ fastocr_status fastocr_dense_decode_attn(fastocr_ctx* ctx, const fastocr_kv_view
     if ((st = check_scores_args(ctx, kv, scores_out, n_stride)) != FASTOCR_OK) return st;
     max_vis = n_stride < ctx->lim.max_vis_len ? n_stride : ctx->lim.max_vis_len;
   }
-  return dense_impl(ctx, kv, q, out, out_is_fp32, scores_out, n_stride, max_vis, fastocr::kWaitAtStart,
-                    static_cast<cudaStream_t>(stream), false, image_mass_out);
+  const bool scratch_scores = scores_out == ctx->scores;   // every chunk reuses the scratch
+  const int64_t per_seq = static_cast<int64_t>(kv->num_q_heads) * fastocr::kHeadDim;
+  const int cb = chunk_sequences(kv);
+  for (int b0 = 0; b0 < kv->batch; b0 += cb) {
+    const fastocr_kv_view sv = sub_view(*kv, b0, kv->batch - b0 < cb ? kv->batch - b0 : cb);
+    st = dense_impl(ctx, &sv, static_cast<const char*>(q) + b0 * per_seq * 2, static_cast<char*>(out) + b0 * per_seq * (out_is_fp32 ? 4 : 2),
+                    out_is_fp32, (scores_out != nullptr && !scratch_scores) ? scores_out + static_cast<int64_t>(b0) * n_stride : scores_out,
+                    n_stride, max_vis, fastocr::kWaitAtStart, static_cast<cudaStream_t>(stream), false,
+                    image_mass_out != nullptr ? image_mass_out + b0 : nullptr);
+    if (st != FASTOCR_OK) return st;
+  }
+  return FASTOCR_OK;
 }
 
 fastocr_status fastocr_focal_scores(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, float* scores_out,
@@ -508,8 +542,16 @@ fastocr_status fastocr_focal_scores(fastocr_ctx* ctx, const fastocr_kv_view* kv,
   if ((st = check_scores_args(ctx, kv, scores_out, n_stride)) != FASTOCR_OK) return st;
   if (ctx->lim.max_vis_len <= 0) return fail(ctx, FASTOCR_ERR_WORKSPACE, "context was created with max_vis_len = 0");
   const int32_t max_vis = n_stride < ctx->lim.max_vis_len ? n_stride : ctx->lim.max_vis_len;
-  return dense_impl(ctx, kv, q, nullptr, 0, scores_out, n_stride, max_vis, fastocr::kWaitAtStart,
-                    static_cast<cudaStream_t>(stream), false, image_mass_out);
+  const int64_t per_seq = static_cast<int64_t>(kv->num_q_heads) * fastocr::kHeadDim;
+  const int cb = chunk_sequences(kv);
+  for (int b0 = 0; b0 < kv->batch; b0 += cb) {
+    const fastocr_kv_view sv = sub_view(*kv, b0, kv->batch - b0 < cb ? kv->batch - b0 : cb);
+    st = dense_impl(ctx, &sv, static_cast<const char*>(q) + b0 * per_seq * 2, nullptr, 0, scores_out + static_cast<int64_t>(b0) * n_stride,
+                    n_stride, max_vis, fastocr::kWaitAtStart, static_cast<cudaStream_t>(stream), false,
+                    image_mass_out != nullptr ? image_mass_out + b0 : nullptr);
+    if (st != FASTOCR_OK) return st;
+  }
+  return FASTOCR_OK;
 }
 
 fastocr_status fastocr_select_topk(fastocr_ctx* ctx, const float* scores, int32_t n_stride, const int32_t* vis_len,
@@ -538,7 +580,16 @@ fastocr_status fastocr_sparse_decode_attn(fastocr_ctx* ctx, const fastocr_kv_vie
   if (idx == nullptr || k == nullptr || out == nullptr) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "NULL idx, k or out");
   if (k_stride <= 0 || max_kept < 0) return fail(ctx, FASTOCR_ERR_INVALID_ARG, "k_stride must be positive, max_kept non-negative");
   NvtxScope range("fastocr_sparse_decode_attn");
-  return sparse_impl(ctx, kv, q, idx, k, k_stride, max_kept, out, out_is_fp32, fastocr::kWaitAtStart, static_cast<cudaStream_t>(stream));
+  const int64_t per_seq = static_cast<int64_t>(kv->num_q_heads) * fastocr::kHeadDim;
+  const int cb = chunk_sequences(kv);
+  for (int b0 = 0; b0 < kv->batch; b0 += cb) {
+    const fastocr_kv_view sv = sub_view(*kv, b0, kv->batch - b0 < cb ? kv->batch - b0 : cb);
+    st = sparse_impl(ctx, &sv, static_cast<const char*>(q) + b0 * per_seq * 2, idx + static_cast<int64_t>(b0) * k_stride, k + b0, k_stride,
+                     max_kept, static_cast<char*>(out) + b0 * per_seq * (out_is_fp32 ? 4 : 2), out_is_fp32, fastocr::kWaitAtStart,
+                     static_cast<cudaStream_t>(stream));
+    if (st != FASTOCR_OK) return st;
+  }
+  return FASTOCR_OK;
 }
 
 fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, const fastocr_kv_view* layers,
@@ -567,9 +618,16 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
   }
   NvtxScope range("fastocr_decode_step");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int B_all = layers[0].batch;
+  const int64_t per_seq = static_cast<int64_t>(layers[0].num_q_heads) * fastocr::kHeadDim;
+  const size_t q_bytes = B_all * per_seq * 2, o_bytes = B_all * per_seq * (out_is_fp32 ? 4 : 2);   // from one layer to the next
+  const int focal_stride = B_all;                      // row length of the per-sequence focal matrix
+  // The step over one chunk of the batch (the whole batch unless it has more than kMaxUnits
+  // (sequence, KV head) pairs); all arguments are the chunk's own (views, first query / output /
+  // index row, first column of the focal matrix).
+  auto step_chunk = [&](const fastocr_kv_view* layers, const void* q, void* out, const uint8_t* focal_seq,
+                        const uint8_t* focal_seq_dev, const int32_t* k, int32_t* fixation, bool& have_out) -> fastocr_status {
   const int B = layers[0].batch;
-  const int64_t per_layer = static_cast<int64_t>(B) * layers[0].num_q_heads * fastocr::kHeadDim;
-  const size_t q_bytes = per_layer * 2, o_bytes = per_layer * (out_is_fp32 ? 4 : 2);
   bool have = has_fixation != 0;
   // How many sequences treat layer l as a focal layer: all or none with one focal set for the batch;
   // anything in between with per-sequence sets (Section 3.1.1 profiles C per sample). Layer 0 without
@@ -578,7 +636,7 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
     if (l == 0 && !have) return B;
     if (focal_seq == nullptr) return is_focal[l] != 0 ? B : 0;
     int n = 0;
-    for (int b = 0; b < B; ++b) n += focal_seq[static_cast<size_t>(l) * B + b] != 0;
+    for (int b = 0; b < B; ++b) n += focal_seq[static_cast<size_t>(l) * focal_stride + b] != 0;
     return n;
   };
   // What the launch issued just before the next one was: nothing of this step yet, a pruned or
@@ -595,7 +653,7 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
   auto uni_cnt = [&](int i) { return ctx->uni_cnt + static_cast<size_t>(i) * ctx->lim.max_batch; };
   if (unite && have) {      // what the previous step left is the kept set until this step's first selection
     FASTOCR_TRY_CUDA(fastocr::launch_union_sets(nullptr, nullptr, U, fixation, k, k_stride, layers[0].vis_len, max_vis_len, B,
-                                                uni_idx(0), uni_cnt(0), nullptr, 0, 1, 0, s), "kept-set launch");
+                                                uni_idx(0), uni_cnt(0), nullptr, 0, focal_stride, 1, 0, s), "kept-set launch");
   }
   // The pruned layers of a step see the same lengths and kept counts: what every CTA of theirs
   // would work out from those (its range, its unit) is computed once, by a small kernel at the
@@ -632,7 +690,7 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
     const int n_focal = focal_count(l);
     const bool fallback = l == 0 && !have;
     const bool mixed = n_focal != 0 && n_focal != B;
-    const uint8_t* mask = mixed ? focal_seq_dev + static_cast<size_t>(l) * B : nullptr;
+    const uint8_t* mask = mixed ? focal_seq_dev + static_cast<size_t>(l) * focal_stride : nullptr;
     fastocr_status st;
     if (n_focal == 0) {
       // a run of layers that the whole batch attends pruned, over the same set and the same lengths: one launch
@@ -696,7 +754,7 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
         const int first = (fallback || (focal_seq == nullptr && !selected_this_step)) ? 1 : 0;
         FASTOCR_TRY_CUDA(fastocr::launch_union_sets(uni_idx(cur), uni_cnt(cur), U, fixation, k, k_stride, layers[l].vis_len,
                                                     max_vis_len, B, uni_idx(cur ^ 1), uni_cnt(cur ^ 1),
-                                                    fallback ? nullptr : focal_seq_dev, l, first, fallback_ran ? 1 : 0, s),
+                                                    fallback ? nullptr : focal_seq_dev, l, focal_stride, first, fallback_ran ? 1 : 0, s),
                          "kept-set launch");
         cur ^= 1;
         prev = kOther;
@@ -704,6 +762,26 @@ fastocr_status fastocr_decode_step_ex(fastocr_ctx* ctx, int32_t num_layers, cons
       if (fallback) fallback_ran = true;
       selected_this_step = true;
       have = true;
+    }
+  }
+  have_out = have;
+  return FASTOCR_OK;
+  };
+  bool have = has_fixation != 0;
+  const int cb = chunk_sequences(&layers[0]);
+  if (cb >= B_all) {
+    const fastocr_status st = step_chunk(layers, q, out, focal_seq, focal_seq_dev, k, fixation, have);
+    if (st != FASTOCR_OK) return st;
+  } else {
+    std::vector<fastocr_kv_view> part(static_cast<size_t>(num_layers));
+    for (int b0 = 0; b0 < B_all; b0 += cb) {
+      for (int l = 0; l < num_layers; ++l) part[l] = sub_view(layers[l], b0, B_all - b0 < cb ? B_all - b0 : cb);
+      const fastocr_status st = step_chunk(part.data(), static_cast<const char*>(q) + b0 * per_seq * 2,
+                                           static_cast<char*>(out) + b0 * per_seq * (out_is_fp32 ? 4 : 2),
+                                           focal_seq != nullptr ? focal_seq + b0 : nullptr,
+                                           focal_seq_dev != nullptr ? focal_seq_dev + b0 : nullptr, k + b0,
+                                           fixation + static_cast<int64_t>(b0) * k_stride, have);
+      if (st != FASTOCR_OK) return st;
     }
   }
   if (has_fixation_out != nullptr) *has_fixation_out = have ? 1 : 0;
@@ -735,13 +813,19 @@ fastocr_status fastocr_warmup_step(fastocr_ctx* ctx, int32_t num_layers, const f
   const int B = layers[0].batch;
   const int64_t per_layer = static_cast<int64_t>(B) * layers[0].num_q_heads * fastocr::kHeadDim;
   const size_t q_bytes = per_layer * 2, o_bytes = per_layer * (out_is_fp32 ? 4 : 2);
+  const int64_t per_seq = static_cast<int64_t>(layers[0].num_q_heads) * fastocr::kHeadDim;
+  const int cb = chunk_sequences(&layers[0]);
   for (int l = 0; l < num_layers; ++l) {
     // one pass over K and V: the layer's output, and from the same logits the head-averaged image
-    // attention whose sum over the image span is Eq. 1's ratio
-    fastocr_status st = dense_impl(ctx, &layers[l], static_cast<const char*>(q) + l * q_bytes, static_cast<char*>(out) + l * o_bytes,
-                                   out_is_fp32, ctx->scores, ctx->lim.max_vis_len, ctx->lim.max_vis_len, fastocr::kWaitAtStart, s,
-                                   false, ratio_out + static_cast<size_t>(l) * B);
-    if (st != FASTOCR_OK) return st;
+    // attention whose sum over the image span is Eq. 1's ratio (batches beyond a launch's reach: in chunks)
+    for (int b0 = 0; b0 < B; b0 += cb) {
+      const fastocr_kv_view sv = sub_view(layers[l], b0, B - b0 < cb ? B - b0 : cb);
+      fastocr_status st = dense_impl(ctx, &sv, static_cast<const char*>(q) + l * q_bytes + b0 * per_seq * 2,
+                                     static_cast<char*>(out) + l * o_bytes + b0 * per_seq * (out_is_fp32 ? 4 : 2), out_is_fp32, ctx->scores,
+                                     ctx->lim.max_vis_len, ctx->lim.max_vis_len, fastocr::kWaitAtStart, s, false,
+                                     ratio_out + static_cast<size_t>(l) * B + b0);
+      if (st != FASTOCR_OK) return st;
+    }
   }
   return FASTOCR_OK;
 }

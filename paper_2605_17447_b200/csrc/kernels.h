@@ -176,12 +176,13 @@ cudaError_t launch_select_topk(const float* scores, int32_t n_stride, const int3
                                cudaStream_t s, const uint8_t* seq_mask = nullptr, int32_t mask_want = 0);
 
 // Kept set of the union variant: out = selected (first selection of a step), current u selected (later
-// ones) or current (sequences that are not focal at `layer` when focal_matrix [L][B] is given). Sets are
+// ones) or current (sequences that are not focal at `layer` when focal_matrix, [L] rows of focal_stride
+// entries, is given). Sets are
 // ascending index lists [B][stride] with counts [B]; cur_idx may be NULL (nothing to carry over).
 cudaError_t launch_union_sets(const int32_t* cur_idx, const int32_t* cur_cnt, int32_t u_stride, const int32_t* sel_idx,
                               const int32_t* sel_cnt, int32_t k_stride, const int32_t* vis_len, int32_t max_vis_len,
                               int32_t batch, int32_t* out_idx, int32_t* out_cnt, const uint8_t* focal_matrix, int32_t layer,
-                              int32_t force_first, int32_t fallback_ran, cudaStream_t s);
+                              int32_t focal_stride, int32_t force_first, int32_t fallback_ran, cudaStream_t s);
 
 cudaError_t configure_kernels();   // one-time cudaFuncSetAttribute calls (current device)
 

@@ -22,18 +22,18 @@ __global__ void __launch_bounds__(kSetThreads) union_sets_kernel(
     const int32_t* __restrict__ cur_idx, const int32_t* __restrict__ cur_cnt, int u_stride,
     const int32_t* __restrict__ sel_idx, const int32_t* __restrict__ sel_cnt, int k_stride,
     const int32_t* __restrict__ vis_len, int n_cap, int32_t* __restrict__ out_idx, int32_t* __restrict__ out_cnt,
-    const uint8_t* __restrict__ focal_matrix, int layer, int batch, int force_first, int fallback_ran) {
+    const uint8_t* __restrict__ focal_matrix, int layer, int focal_stride, int force_first, int fallback_ran) {
   __shared__ uint32_t bits[kSetThreads];
   __shared__ uint32_t warp_tot[kSetThreads / 32];
   wait_for_prior_grids();                              // the selection kernel wrote sel_idx just before
   dependents_may_launch();
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = max(min(vis_len[b], n_cap), 0);
-  const bool focal_here = focal_matrix == nullptr || focal_matrix[static_cast<int64_t>(layer) * batch + b] != 0;
+  const bool focal_here = focal_matrix == nullptr || focal_matrix[static_cast<int64_t>(layer) * focal_stride + b] != 0;
   bool first = force_first != 0;
   if (!first && focal_matrix != nullptr && !fallback_ran) {    // no earlier focal layer of this sequence in this step
     first = true;
-    for (int l = 0; l < layer; ++l) first = first && focal_matrix[static_cast<int64_t>(l) * batch + b] == 0;
+    for (int l = 0; l < layer; ++l) first = first && focal_matrix[static_cast<int64_t>(l) * focal_stride + b] == 0;
   }
   const int n_cur = (cur_idx != nullptr && !(focal_here && first)) ? min(max(cur_cnt[b], 0), min(N, u_stride)) : 0;
   const int n_sel = focal_here ? min(max(sel_cnt[b], 0), min(N, k_stride)) : 0;
@@ -81,11 +81,11 @@ __global__ void __launch_bounds__(kSetThreads) union_sets_kernel(
 cudaError_t launch_union_sets(const int32_t* cur_idx, const int32_t* cur_cnt, int32_t u_stride, const int32_t* sel_idx,
                               const int32_t* sel_cnt, int32_t k_stride, const int32_t* vis_len, int32_t max_vis_len,
                               int32_t batch, int32_t* out_idx, int32_t* out_cnt, const uint8_t* focal_matrix, int32_t layer,
-                              int32_t force_first, int32_t fallback_ran, cudaStream_t s) {
+                              int32_t focal_stride, int32_t force_first, int32_t fallback_ran, cudaStream_t s) {
   if (batch <= 0) return cudaSuccess;
   if (max_vis_len > kTopkMaxN) return cudaErrorInvalidValue;
   const cudaError_t e = launch_pdl(union_sets_kernel, dim3(batch), dim3(kSetThreads), 0, s, cur_idx, cur_cnt, u_stride, sel_idx,
-                                   sel_cnt, k_stride, vis_len, max_vis_len, out_idx, out_cnt, focal_matrix, layer, batch,
+                                   sel_cnt, k_stride, vis_len, max_vis_len, out_idx, out_cnt, focal_matrix, layer, focal_stride,
                                    force_first, fallback_ran);
   count_launches(1);
   return e;

@@ -486,3 +486,75 @@ def test_scores_exchange_over_nccl_single_rank(tmp_path):
     if "backend up" not in p.stdout:                    # the machine's NCCL set-up, not this library
         pytest.skip("the NCCL backend did not come up here: " + p.stderr[-300:])
     assert p.returncode == 0 and p.stdout.strip().endswith("ok"), p.stdout[-2000:] + p.stderr[-4000:]
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_batches_beyond_one_launch_run_in_chunks(fo, paged):
+    """140 sequences x 4 KV heads = 560 (sequence, KV head) pairs, more than a launch covers (512): every entry
+    point processes the batch as chunks of whole sequences (128 + 12 here). Every sequence is compared with the
+    oracle: single-layer calls, the warm-up step, and the decode step with per-sequence focal sets (so that the
+    focal matrix, the index rows and the outputs are all addressed per chunk), plain and as the union variant."""
+    g = torch.Generator().manual_seed(91)
+    B, L = 140, 4
+    spans = [(int(torch.randint(0, 7, (1,), generator=g)), int(torch.randint(40, 121, (1,), generator=g)),
+              int(torch.randint(0, 21, (1,), generator=g))) for _ in range(B)]
+    cases, views, q_all = make_layer_stack(2800, spans, L, page_size=16 if paged else 0, q_boost=1.5)
+    base = cases[0]
+    n_max = max(base.vis_len)
+    c = fo.Context(max_batch=B, num_q_heads=28, num_kv_heads=4, max_seq_len=max(base.seq_len), max_vis_len=n_max)
+    ks = [oracle.kept_count(n, 0.1) for n in base.vis_len]
+    kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+    qd = q_all.cuda()
+
+    # single-layer entry points
+    out = torch.empty(B, 28, 128, dtype=torch.float32, device="cuda")
+    sc = torch.zeros(B, n_max, dtype=torch.float32, device="cuda")
+    mass = torch.zeros(B, dtype=torch.float32, device="cuda")
+    fo.fastocr_dense_decode_attn(c, views[0], qd[0], out, scores_out=sc, image_mass_out=mass)
+    sc2 = torch.zeros_like(sc)
+    fo.fastocr_focal_scores(c, views[0], qd[0], sc2)
+    idx = torch.full((B, max(ks)), -1, dtype=torch.int32, device="cuda")
+    fo.fastocr_select_topk(c, sc, views[0].vis_len, kd, idx, n_max)
+    out_s = torch.empty_like(out)
+    fo.fastocr_sparse_decode_attn(c, views[0], qd[0], idx, kd, out_s)
+    assert torch.equal(sc, sc2)
+    for b in range(B):
+        qb, Kb, Vb = cases[0].seq(b)
+        _check_out(out[b], oracle.dense(qb, Kb, Vb, SCALE, True))
+        ref_sc, ref_mass = oracle.scores(qb, Kb, SCALE, base.vis_start[b], base.vis_len[b], True)
+        assert float((sc[b, :base.vis_len[b]].cpu() - ref_sc).abs().max()) <= 1e-6
+        assert abs(float(mass[b]) - ref_mass) <= 1e-5
+        want = oracle.topk(sc[b, :base.vis_len[b]].cpu(), ks[b])
+        assert idx[b, :ks[b]].cpu().tolist() == want.tolist()
+        _check_out(out_s[b], oracle.sparse(qb, Kb, Vb, SCALE, base.vis_start[b], base.vis_len[b], want, True))
+
+    # warm-up step: Eq. 1's ratio per layer and sequence
+    outw = torch.empty(L, B, 28, 128, dtype=torch.float32, device="cuda")
+    r = torch.full((L, B), -1.0, dtype=torch.float32, device="cuda")
+    fo.fastocr_warmup_step(c, views, qd, outw, r)
+    for b in (0, 1, 126, 127, 128, 129, 139):           # both sides of the chunk boundary
+        outs, rr = oracle.warmup_step([cs.seq(b) for cs in cases], base.vis_start[b], base.vis_len[b], SCALE, acc64=True)
+        for l in range(L):
+            _check_out(outw[l, b], outs[l])
+            assert abs(float(r[l, b]) - rr[l]) <= 1e-5
+
+    # decode steps with per-sequence focal layer sets
+    focal_of = [[1] if b % 3 == 0 else ([2] if b % 3 == 1 else [1, 3]) for b in range(B)]
+    matrix = [[l in focal_of[b] for b in range(B)] for l in range(L)]
+    for union in (False, True):
+        fix = torch.full((B, max(ks)), -1, dtype=torch.int32, device="cuda")
+        have, f_last = False, [None] * B
+        for step in range(2):
+            outd = torch.full((L, B, 28, 128), 7.0, dtype=torch.float32, device="cuda")
+            have = fo.fastocr_decode_step(c, views, qd, outd, matrix, kd, fix, have, n_max, union_sets=union,
+                                          max_kept=max(3 * k + s - n for k, s, n in zip(ks, base.seq_len, base.vis_len)) if union else 0)
+            assert have
+            for b in range(B):
+                tr = oracle.decode_step([cs.seq(b) for cs in cases], focal_of[b], f_last[b], base.vis_start[b], base.vis_len[b],
+                                        0.1, SCALE, acc64=True, union_sets=union)
+                for l in range(L):
+                    _check_out(outd[l, b], tr.outputs[l])
+                assert fix[b, :ks[b]].cpu().tolist() == tr.f_last.tolist()
+                f_last[b] = tr.f_last
+    assert c.device_faults() == 0
+    c.close()
