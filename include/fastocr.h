@@ -42,7 +42,7 @@
  *     bf16 remainder; exponentials are ex2.approx. Outputs agree with an fp32 CPU evaluation of the
  *     same formulas to about 1e-4 absolute.
  *   - head_dim must be 128 and num_q_heads / num_kv_heads (the GQA group size)
- *     one of 1, 2, 4, 7, 8; query head h reads KV head h / group size.
+ *     1 to 8; query head h reads KV head h / group size.
  */
 #ifndef FASTOCR_H_
 #define FASTOCR_H_

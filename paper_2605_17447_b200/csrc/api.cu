@@ -85,7 +85,7 @@ fastocr_status fail(fastocr_ctx* ctx, fastocr_status code, const char* fmt, ...)
   return code;
 }
 
-bool group_supported(int G) { return G == 1 || G == 2 || G == 4 || G == 7 || G == 8; }
+bool group_supported(int G) { return G >= 1 && G <= fastocr::kMaxGroup; }
 
 fastocr_status check_view(fastocr_ctx* ctx, const fastocr_kv_view* kv, const void* q, bool need_v) {
   if (ctx == nullptr) return FASTOCR_ERR_INVALID_ARG;
@@ -99,7 +99,7 @@ fastocr_status check_view(fastocr_ctx* ctx, const fastocr_kv_view* kv, const voi
   if (kv->num_q_heads % kv->num_kv_heads != 0)
     return fail(ctx, FASTOCR_ERR_INVALID_ARG, "num_q_heads %d not a multiple of num_kv_heads %d", kv->num_q_heads, kv->num_kv_heads);
   if (!group_supported(kv->num_q_heads / kv->num_kv_heads))
-    return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "GQA group size %d (supported: 1, 2, 4, 7, 8)", kv->num_q_heads / kv->num_kv_heads);
+    return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "GQA group size %d (supported: 1 to 8)", kv->num_q_heads / kv->num_kv_heads);
   if (kv->page_size < 0 || (kv->page_size & (kv->page_size - 1)) != 0)
     return fail(ctx, FASTOCR_ERR_UNSUPPORTED, "page_size %d is not 0 or a power of two", kv->page_size);
   if (kv->page_size > 0) {

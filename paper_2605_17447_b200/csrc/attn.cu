@@ -1236,7 +1236,7 @@ cudaError_t configure_t() {
 
 }  // namespace
 
-#define FASTOCR_FOR_EACH_GROUP(X) X(1) X(2) X(4) X(7) X(8)
+#define FASTOCR_FOR_EACH_GROUP(X) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8)
 
 cudaError_t launch_attn_plan(const AttnLaunch& a, int4* plan_out, cudaStream_t s) {
   if (a.batch * a.num_kv_heads > kMaxUnits || a.grid_ctas <= 0) return cudaErrorInvalidValue;

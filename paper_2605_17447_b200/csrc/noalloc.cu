@@ -97,7 +97,7 @@ fastocr_status fastocr_sparse_decode_attn_noalloc(const fastocr_kv_view* kv, con
   if (kv->head_dim != fastocr::kHeadDim) return fail(FASTOCR_ERR_UNSUPPORTED, "head_dim must be 128");
   if (kv->num_q_heads % kv->num_kv_heads != 0) return fail(FASTOCR_ERR_INVALID_ARG, "num_q_heads must be a multiple of num_kv_heads");
   const int G = kv->num_q_heads / kv->num_kv_heads;
-  if (!(G == 1 || G == 2 || G == 4 || G == 7 || G == 8)) return fail(FASTOCR_ERR_UNSUPPORTED, "GQA group size must be 1, 2, 4, 7 or 8");
+  if (G < 1 || G > fastocr::kMaxGroup) return fail(FASTOCR_ERR_UNSUPPORTED, "GQA group size must be 1 to 8");
   if (kv->page_size < 0 || (kv->page_size & (kv->page_size - 1)) != 0) return fail(FASTOCR_ERR_UNSUPPORTED, "page_size must be 0 or a power of two");
   if (kv->page_size > 0 && (kv->block_table == nullptr || static_cast<int64_t>(kv->max_pages) * kv->page_size < kv->max_seq_len))
     return fail(FASTOCR_ERR_INVALID_ARG, "paged view needs a block_table covering max_seq_len");

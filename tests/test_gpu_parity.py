@@ -451,7 +451,7 @@ def test_argument_errors_are_reported_not_launched(fo, ctx):
     assert e.value.code == 3
     small.close()
     bad = case.device_view()
-    bad.num_q_heads = 12                                        # group of 3: unsupported
+    bad.num_q_heads = 36                                        # group of 9: unsupported
     with pytest.raises(fo.FastOCRError) as e:
         fo.fastocr_dense_decode_attn(ctx, bad, q, out)
     assert e.value.code == 2

@@ -306,9 +306,9 @@ def test_a_run_of_pruned_layers_longer_than_one_launch_takes(fo, ctx):
     assert ctx.device_faults() == 0
 
 
-@pytest.mark.parametrize("H,Hkv", [(3, 3), (4, 2), (16, 4), (8, 1)])
+@pytest.mark.parametrize("H,Hkv", [(3, 3), (4, 2), (16, 4), (8, 1), (6, 2), (10, 2), (12, 2)])
 def test_decode_step_other_group_sizes(fo, ctx, H, Hkv):
-    """GQA groups of 1, 2, 4 and 8 query heads per KV head through the whole step (runs of pruned layers as
+    """GQA groups of 1, 2, 4, 8, 3, 5 and 6 (12 / 2: the 1.7B OCR model's shape) query heads per KV head through the whole step (runs of pruned layers as
     one launch, a focal layer in between), paged cache, ragged batch."""
     L = 5
     spans = [(6, 300, 20), (0, 170, 41), (5, 64, 0)]
