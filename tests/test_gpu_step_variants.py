@@ -558,3 +558,60 @@ def test_batches_beyond_one_launch_run_in_chunks(fo, paged):
                 f_last[b] = tr.f_last
     assert c.device_faults() == 0
     c.close()
+
+
+def test_two_contexts_on_two_streams_and_a_captured_step(fo):
+    """Launches go to the stream they are given: two contexts, each on a stream of its own, run their steps
+    at the same time on different data; then one step is captured into a CUDA graph and replayed on fresh
+    queries (the pointers are the same, the contents new). All of it against the oracle."""
+    L, focal = 4, [1]
+    spans = [(6, 300, 20), (3, 170, 41)]
+    jobs = []
+    for seed in (2900, 2901):
+        cases, views, q_all = make_layer_stack(seed, spans, L, q_boost=1.5)
+        base = cases[0]
+        ks = [oracle.kept_count(n, 0.1) for n in base.vis_len]
+        jobs.append(dict(cases=cases, views=views, q=q_all.cuda(), base=base, ks=ks,
+                         ctx=fo.Context(max_batch=base.B, num_q_heads=28, num_kv_heads=4, max_seq_len=max(base.seq_len),
+                                        max_vis_len=max(base.vis_len)),
+                         kd=torch.tensor(ks, dtype=torch.int32, device="cuda"),
+                         fix=torch.full((base.B, max(ks)), -1, dtype=torch.int32, device="cuda"),
+                         out=torch.full((L, base.B, 28, 128), 7.0, dtype=torch.float32, device="cuda"),
+                         stream=torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    for rep in range(3):                                 # interleaved issue: the two streams overlap on the device
+        for j in jobs:
+            fo.fastocr_decode_step(j["ctx"], j["views"], j["q"], j["out"], [l in focal for l in range(L)], j["kd"], j["fix"],
+                                   rep > 0, max(j["base"].vis_len), stream=j["stream"])
+    torch.cuda.synchronize()
+    for j in jobs:
+        base = j["base"]
+        for b in range(base.B):
+            tr = oracle.decode_step([c.seq(b) for c in j["cases"]], focal, None, base.vis_start[b], base.vis_len[b], 0.1, SCALE, acc64=True)
+            tr2 = oracle.decode_step([c.seq(b) for c in j["cases"]], focal, tr.f_last, base.vis_start[b], base.vis_len[b], 0.1, SCALE, acc64=True)
+            for l in range(L):
+                _check_out(j["out"][l, b], tr2.outputs[l])
+            assert j["fix"][b, :j["ks"][b]].cpu().tolist() == tr2.f_last.tolist()
+            j.setdefault("f_last", []).append(tr2.f_last)
+
+    # capture one step of the first job, replay it on new queries written into the same buffer
+    j = jobs[0]
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.graph(g, stream=side):
+        fo.fastocr_decode_step(j["ctx"], j["views"], j["q"], j["out"], [l in focal for l in range(L)], j["kd"], j["fix"], True,
+                               max(j["base"].vis_len))                  # the current stream is the capturing one
+    cases2, _, q2 = make_layer_stack(2900, spans, L, q_boost=1.1)       # same caches (same seed), other queries
+    j["q"].copy_(q2.cuda())
+    j["out"].fill_(7.0)
+    g.replay()
+    torch.cuda.synchronize()
+    base = j["base"]
+    for b in range(base.B):
+        tr = oracle.decode_step([c.seq(b) for c in cases2], focal, j["f_last"][b], base.vis_start[b], base.vis_len[b], 0.1, SCALE, acc64=True)
+        for l in range(L):
+            _check_out(j["out"][l, b], tr.outputs[l])
+        assert j["fix"][b, :j["ks"][b]].cpu().tolist() == tr.f_last.tolist()
+    for j in jobs:
+        assert j["ctx"].device_faults() == 0
+        j["ctx"].close()
