@@ -615,3 +615,62 @@ def test_two_contexts_on_two_streams_and_a_captured_step(fo):
     for j in jobs:
         assert j["ctx"].device_faults() == 0
         j["ctx"].close()
+
+
+def _random_step_case(seed):
+    """One seeded random decode-step problem: head geometry, batch, depth, spans (empty image, empty text,
+    single tokens, ragged), cache layout, tau, focal sets (one per batch or per sequence), plain or union."""
+    import random
+    rnd = random.Random(seed)
+    H, Hkv = rnd.choice([(28, 4), (16, 2), (12, 2), (8, 8), (64, 8), (10, 2), (6, 2), (4, 1), (7, 1), (32, 4)])
+    B, L = rnd.choice([1, 2, 3, 5, 9]), rnd.choice([1, 2, 3, 5, 7])
+    paged, big = rnd.random() < 0.5, rnd.random() < 0.15
+    tau = rnd.choice([0.0, 0.004, 0.05, 0.1, 0.3, 1.0])
+    spans = []
+    for _ in range(B):
+        n = rnd.choice([3000, 5000]) if big else rnd.choice([0, 1, 7, 33, 64, 100, 257, 700, 1500])
+        a, t = rnd.choice([0, 1, 5, 16, 40]), rnd.choice([0, 1, 3, 20, 70, 200])
+        if a + t == 0 and oracle.kept_count(n, tau) == 0:
+            a = 1                                        # the oracle refuses an empty kept set
+        spans.append((a, n, t))
+    if rnd.random() < 0.4:
+        focal_of = [[l for l in range(L) if rnd.random() < 0.35] for _ in range(B)]
+        is_focal = [[l in focal_of[b] for b in range(B)] for l in range(L)]
+    else:
+        f = [l for l in range(L) if rnd.random() < 0.35]
+        focal_of, is_focal = [f] * B, [l in f for l in range(L)]
+    return dict(H=H, Hkv=Hkv, L=L, paged=paged, tau=tau, spans=spans, focal_of=focal_of, is_focal=is_focal,
+                union=rnd.random() < 0.3, steps=rnd.choice([1, 2, 3]), boost=rnd.choice([1.0, 1.5, 2.5]))
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_randomised_decode_steps(fo, block):
+    """Forty seeded random decode-step problems (ten per block), each run for one to three steps and
+    compared with the oracle's Algorithm 1 trace: every output, and the carried set exactly."""
+    for seed in range(10 * block, 10 * block + 10):
+        p = _random_step_case(seed)
+        cases, views, q_all = make_layer_stack(100000 + seed, p["spans"], p["L"], H=p["H"], Hkv=p["Hkv"],
+                                               page_size=16 if p["paged"] else 0, q_boost=p["boost"])
+        base = cases[0]
+        B, L = base.B, p["L"]
+        ks = [oracle.kept_count(n, p["tau"]) for n in base.vis_len]
+        kd = torch.tensor(ks, dtype=torch.int32, device="cuda")
+        fix = torch.full((B, max(1, max(ks))), -1, dtype=torch.int32, device="cuda")
+        n_max = max(1, max(base.vis_len))
+        c = fo.Context(max_batch=B, num_q_heads=p["H"], num_kv_heads=p["Hkv"], max_seq_len=max(base.seq_len), max_vis_len=n_max)
+        have, f_last = False, [None] * B
+        for step in range(p["steps"]):
+            out = torch.full((L, B, p["H"], 128), 7.0, dtype=torch.float32, device="cuda")
+            mk = max(L * k + s - n for k, s, n in zip(ks, base.seq_len, base.vis_len)) if p["union"] else 0
+            have = fo.fastocr_decode_step(c, views, q_all.cuda(), out, p["is_focal"], kd, fix, have, n_max, max_kept=mk, union_sets=p["union"])
+            for b in range(B):
+                tr = oracle.decode_step([cs.seq(b) for cs in cases], p["focal_of"][b], f_last[b], base.vis_start[b], base.vis_len[b],
+                                        p["tau"], SCALE, acc64=True, union_sets=p["union"])
+                for l in range(L):
+                    err = float((out[l, b].cpu() - tr.outputs[l]).abs().max())
+                    assert err <= TIGHT, (seed, step, l, b, err, p)
+                if tr.f_last is not None:
+                    assert fix[b, :ks[b]].cpu().tolist() == tr.f_last.tolist(), (seed, step, b, p)
+                f_last[b] = tr.f_last
+        assert c.device_faults() == 0, (seed, p)
+        c.close()
